@@ -1,0 +1,183 @@
+/*
+ * hma.h -- C ABI of the decode-side BFP8 KV path (deferred dequantization, paper section 3.3).
+ *
+ * The prefill accelerator ships each layer's KV cache as raw Blocked-FP8 bytes; the decode GPU
+ * keeps them as raw BFP8 pages in HBM and rebuilds BF16 values inside the paged attention kernel
+ * (paper Fig. 2 step 3 and section 3.3).  This library is that decode-side path:
+ *
+ *   hma_kv_ingest_layer     scatter one layer of arriving wire bytes into the paged cache
+ *                           (consumer half of the compute-transfer pipeline, section 3.2)
+ *   hma_decode_attention    GQA paged decode attention reading raw BFP8 pages (section 3.3)
+ *   hma_bfp8_dequant_bf16   one-shot BFP8 -> BF16 rebuild of a request's KV (section 3.3, the
+ *                           "fused kernel rebuilds a whole request's KV")
+ *
+ * BFP8 as read here (the paper gives only "per-block shared exponent" and "7-bit mantissa"):
+ * a block is 16 consecutive head-dim channels of one (token, kv head); it has one exponent byte E
+ * (bias 127) and 16 element bytes b = s<<7 | m;  value = (-1)^s * m * 2^(E-133).  Every such
+ * value with E <= 254 is exactly a BF16 number.
+ *
+ * Conventions for every call
+ *   - plain C; all pointers are raw addresses; "device" = CUDA device memory of the current
+ *     device, "host" = ordinary host memory, "pinned" = page-locked host memory mapped into the
+ *     device address space.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - ownership: the caller owns every buffer (cache layers, wire, Q, output, tables, workspace);
+ *     the library allocates one 4-byte device flag word per cache handle and nothing else.
+ *   - asynchrony: a call validates its arguments on the host, enqueues work on `stream`, and
+ *     returns; no call synchronises the device except hma_error_flags.
+ *   - errors: invalid arguments return a status and enqueue nothing.  Device-side anomalies never
+ *     trap: a page id outside [0, num_pages) is skipped and a bit is set in the cache's flag word.
+ *   - supported geometry: head_dim 128, 16 tokens per page, 16-element blocks,
+ *     num_q_heads / num_kv_heads in 1..8.
+ */
+#ifndef HMA_H
+#define HMA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HMA_OK = 0,
+    HMA_ERR_INVALID_ARG = 1,
+    HMA_ERR_UNSUPPORTED_SHAPE = 2,
+    HMA_ERR_ALIGNMENT = 3,
+    HMA_ERR_WORKSPACE_TOO_SMALL = 4,
+    HMA_ERR_CUDA = 5,
+    HMA_ERR_DEVICE_FLAGGED = 6
+} hma_status_t;
+
+typedef enum { HMA_KV_BFP8 = 0, HMA_KV_BF16 = 1 } hma_kv_format_t;
+typedef enum { HMA_WIRE_TILE32 = 0, HMA_WIRE_ROWMAJOR = 1 } hma_wire_layout_t;
+typedef enum { HMA_OUT_BF16 = 0, HMA_OUT_F32 = 1 } hma_out_dtype_t;
+
+/* bits of the device flag word (hma_error_flags) */
+#define HMA_FLAG_BAD_PAGE_ATTENTION 1u  /* block table entry outside [0, num_pages): page skipped */
+#define HMA_FLAG_BAD_PAGE_INGEST    2u  /* page id outside [0, num_pages): page not written      */
+#define HMA_FLAG_BAD_PAGE_DEQUANT   4u  /* page id outside [0, num_pages): output rows zeroed    */
+#define HMA_FLAG_WAIT_TIMEOUT       8u  /* a bounded wait inside a kernel ran out                */
+
+typedef struct {
+    int32_t num_layers;
+    int32_t num_q_heads;
+    int32_t num_kv_heads;
+    int32_t head_dim;      /* must be 128 */
+    int32_t page_tokens;   /* must be 16  */
+    int32_t bfp_block;     /* must be 16  */
+    int64_t num_pages;     /* physical pages per layer */
+    int32_t format;        /* hma_kv_format_t */
+} hma_cache_desc_t;
+
+typedef struct hma_cache hma_cache_t;   /* opaque; host-side metadata only */
+
+/*
+ * Paged KV cache (paper Fig. 2 step 3: "raw BFP8 pages in HBM").
+ *
+ * One layer is `num_pages` pages; a page holds 16 tokens of every kv head; the record of one
+ * (page, kv head) is contiguous: K part then V part.
+ *   HMA_KV_BFP8: record = 4352 B = K[128 exponent bytes | 2048 element bytes] V[128 | 2048].
+ *                The bytes are the wire bytes unchanged; only their positions inside the record
+ *                are permuted so that one 16-byte shared-memory load feeds one tensor-core
+ *                operand fragment:
+ *                  K exponent (tok, blk j)  at  (tok%8)*16 + (tok/8)*8 + j
+ *                  K element  (tok, ch)     at  128 + ((tok/8) + 2*(j/4))*512 + ((tok%8)*4 + (ch%16)/4)*16
+ *                                               + (j%4)*4 + ch%4,              j = ch/16
+ *                  V exponent (tok, blk j)  at  2176 + ((tok%8)/2)*32 + j*4 + k
+ *                  V element  (tok, ch)     at  2304 + (j/2)*512 + ((ch%8)*4 + (tok%8)/2)*16
+ *                                               + ((j%2)*2 + (ch%16)/8)*4 + k
+ *                                               with k = tok%2 + 2*(tok/8)
+ *   HMA_KV_BF16: record = 8192 B = K[16 x 128 BF16] V[16 x 128 BF16], positions permuted likewise
+ *                (the dequant-free baseline cache, section 3.3 last sentence).
+ * hma_cache_layer_bytes returns num_pages * num_kv_heads * record size, or 0 for a bad descriptor.
+ * The caller allocates each layer (device memory, 256-byte aligned) and passes the pointers;
+ * the handle copies the pointer array.  Layers are not touched by create/destroy.
+ */
+size_t hma_cache_layer_bytes(const hma_cache_desc_t *desc);
+hma_status_t hma_cache_create(const hma_cache_desc_t *desc, void *const *layer_ptrs /* host array of device pointers */,
+                              hma_cache_t **out);
+void hma_cache_destroy(hma_cache_t *cache);
+
+/*
+ * Ingest one layer of one request (sections 3.2 and 3.3: host-to-device copy and the
+ * tiled -> paged layout conversion that merges per-chip shards).  Pure byte movement on a BFP8
+ * cache; on a BF16 cache the same call decodes while scattering (the "standalone consumer pass"
+ * of section 2.3, used to fill the baseline cache with identical values).
+ *
+ *   k_wire, v_wire  device or pinned: raw wire bytes of heads [head_begin, head_begin+head_count)
+ *                   for tokens [token_begin, token_begin+n_tokens), wire token 0 = token_begin.
+ *                   HMA_WIRE_ROWMAJOR: [head][token][8 exponent bytes | 128 element bytes]
+ *                   HMA_WIRE_TILE32:   [head][ceil(n_tokens/32)][4][1088 B]: a 32-token x 32-channel
+ *                     tile = four 16x16 faces ordered (row half, column half); exponents at
+ *                     face*16 + row%16, elements at 64 + face*256 + (row%16)*16 + col%16.
+ *                   Both pointers 16-byte aligned.
+ *   page_ids        device int32: page_ids[i] = physical page of the request's logical page
+ *                   floor(token_begin/16) + i; ceil((token_begin%16 + n_tokens)/16) entries.
+ * Token slots outside the range, other heads and other pages keep their bytes.  Pages being
+ * written must not be read by a concurrent hma_decode_attention; order with stream events.
+ */
+hma_status_t hma_kv_ingest_layer(hma_cache_t *cache, int32_t layer,
+                                 const void *k_wire, const void *v_wire, int32_t wire_layout,
+                                 int32_t head_begin, int32_t head_count,
+                                 const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
+                                 void *stream);
+
+/*
+ * Decode attention over block tables (section 3.3; one query token per sequence, section 1).
+ * For sequence b, q head h, kv head g = h / (num_q_heads/num_kv_heads), T = context_lens[b]:
+ *   s_t = sm_scale * <q[b][h], K_t>,  p = softmax_t(s),  out[b][h] = sum_t p_t V_t,  t < T,
+ * K_t, V_t being the exact BFP8 values of the cached bytes.  T = 0 gives zeros.  Tokens >= T are
+ * masked whatever bytes the last page holds; table entries past ceil(T/16) are never read.
+ *
+ *   q            device, BF16 [batch][num_q_heads][128], 16-byte aligned
+ *   out          device, [batch][num_q_heads][128] BF16 or F32 per out_dtype
+ *   block_table  device int32 [batch][max_pages_per_seq]
+ *   context_lens device int32 [batch]; every entry <= max_pages_per_seq*16
+ *   workspace    device, 256-byte aligned, >= hma_decode_attention_workspace_bytes(...) bytes;
+ *                contents need no initialisation and are clobbered
+ * Accuracy: fp32 accumulation; element exponents above 250 are outside the supported range.
+ */
+size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *desc, int32_t batch);
+hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,
+                                  const void *q, void *out, int32_t out_dtype,
+                                  const int32_t *block_table, int32_t max_pages_per_seq,
+                                  const int32_t *context_lens, int32_t batch, float sm_scale,
+                                  void *workspace, size_t workspace_bytes, void *stream);
+
+/* Same contract, computed by a plain one-CTA-per-(sequence, kv head) CUDA-core kernel that decodes
+ * every element to BF16 first (the elementwise reconstruction section 3.3 compares against).
+ * Needs no workspace.  Kept as an on-device cross-check of the fast kernel. */
+hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer,
+                                         const void *q, void *out, int32_t out_dtype,
+                                         const int32_t *block_table, int32_t max_pages_per_seq,
+                                         const int32_t *context_lens, int32_t batch, float sm_scale,
+                                         void *stream);
+
+/*
+ * One-shot reconstruction (section 3.3): tokens [token_begin, token_begin+n_tokens) of a request,
+ * tensor `which` (0 = K, 1 = V), all kv heads -> row-major BF16 [n_tokens][num_kv_heads][128].
+ * Bit-exact: each output is the BFP8 value rounded to BF16 (exact for E <= 254; E = 255 with
+ * m >= 64 gives +-Inf; m = 0 keeps its sign).  page_ids as in hma_kv_ingest_layer.
+ * On a BF16 cache the call is a gather.  out_bf16: device, 16-byte aligned.
+ */
+hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t layer, int32_t which,
+                                   const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
+                                   void *out_bf16, void *stream);
+
+/* Flat variant: n_blocks blocks, exps[i] with mants[16*i .. 16*i+15] -> out_bf16[16*i ..] (device pointers). */
+hma_status_t hma_bfp8_dequant_blocks_bf16(const uint8_t *exps, const uint8_t *mants, int64_t n_blocks,
+                                          void *out_bf16, void *stream);
+
+/* Copies the cache's device flag word to *host_out and clears it.  Synchronises `stream`. */
+hma_status_t hma_error_flags(const hma_cache_t *cache, uint32_t *host_out, void *stream);
+
+const char *hma_status_string(int32_t status);
+
+/* Number of kernels this library has launched in the calling process (for launch accounting). */
+int64_t hma_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HMA_H */

@@ -1,0 +1,176 @@
+"""ctypes binding of libhma.so: the same entry points as include/hma.h, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch provides device memory and streams); every step of the
+path runs inside the library's kernels.  Loading fails loudly when the library has not been
+built: there is no fallback of any kind.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libhma.so")
+
+HMA_OK = 0
+HMA_ERR_INVALID_ARG, HMA_ERR_UNSUPPORTED_SHAPE, HMA_ERR_ALIGNMENT = 1, 2, 3
+HMA_ERR_WORKSPACE_TOO_SMALL, HMA_ERR_CUDA, HMA_ERR_DEVICE_FLAGGED = 4, 5, 6
+HMA_KV_BFP8, HMA_KV_BF16 = 0, 1
+HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR = 0, 1
+HMA_OUT_BF16, HMA_OUT_F32 = 0, 1
+HMA_FLAG_BAD_PAGE_ATTENTION, HMA_FLAG_BAD_PAGE_INGEST, HMA_FLAG_BAD_PAGE_DEQUANT, HMA_FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
+
+
+class CacheDesc(ctypes.Structure):
+    _fields_ = [("num_layers", ctypes.c_int32), ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("page_tokens", ctypes.c_int32), ("bfp_block", ctypes.c_int32),
+                ("num_pages", ctypes.c_int64), ("format", ctypes.c_int32)]
+
+
+class HmaError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if libhma.so is missing (build it with build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError("libhma.so is not built: run `python -m paper_2606_29986_b200.build`")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+        L.hma_cache_layer_bytes.restype = sz
+        L.hma_cache_layer_bytes.argtypes = [ctypes.POINTER(CacheDesc)]
+        L.hma_cache_create.restype = i32
+        L.hma_cache_create.argtypes = [ctypes.POINTER(CacheDesc), ctypes.POINTER(vp), ctypes.POINTER(vp)]
+        L.hma_cache_destroy.restype = None
+        L.hma_cache_destroy.argtypes = [vp]
+        L.hma_kv_ingest_layer.restype = i32
+        L.hma_kv_ingest_layer.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, i64, i64, vp]
+        L.hma_decode_attention_workspace_bytes.restype = sz
+        L.hma_decode_attention_workspace_bytes.argtypes = [ctypes.POINTER(CacheDesc), i32]
+        L.hma_decode_attention.restype = i32
+        L.hma_decode_attention.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp, sz, vp]
+        L.hma_decode_attention_simple.restype = i32
+        L.hma_decode_attention_simple.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
+        L.hma_bfp8_dequant_bf16.restype = i32
+        L.hma_bfp8_dequant_bf16.argtypes = [vp, i32, i32, vp, i64, i64, vp, vp]
+        L.hma_bfp8_dequant_blocks_bf16.restype = i32
+        L.hma_bfp8_dequant_blocks_bf16.argtypes = [vp, vp, i64, vp, vp]
+        L.hma_error_flags.restype = i32
+        L.hma_error_flags.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+        L.hma_status_string.restype = ctypes.c_char_p
+        L.hma_status_string.argtypes = [i32]
+        L.hma_launch_count.restype = i64
+        L.hma_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(status):
+    return lib().hma_status_string(int(status)).decode()
+
+
+def _check(status, where):
+    if status != HMA_OK:
+        raise HmaError(status, where)
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else ctypes.c_void_p(0)
+
+
+def make_desc(num_layers, num_q_heads, num_kv_heads, num_pages, fmt=HMA_KV_BFP8, head_dim=128, page_tokens=16, bfp_block=16):
+    return CacheDesc(num_layers, num_q_heads, num_kv_heads, head_dim, page_tokens, bfp_block, num_pages, fmt)
+
+
+def hma_cache_layer_bytes(desc):
+    return int(lib().hma_cache_layer_bytes(ctypes.byref(desc)))
+
+
+class KVCache:
+    """Owns the torch uint8 layer buffers and the library's cache handle."""
+
+    def __init__(self, desc, device="cuda", fill=None):
+        self.desc = desc
+        nbytes = hma_cache_layer_bytes(desc)
+        if nbytes == 0:
+            raise HmaError(HMA_ERR_UNSUPPORTED_SHAPE, "hma_cache_layer_bytes")
+        self.layers = []
+        for _ in range(desc.num_layers):
+            t = torch.empty(nbytes, dtype=torch.uint8, device=device)
+            if fill is not None:
+                t.fill_(fill)
+            self.layers.append(t)
+        ptrs = (ctypes.c_void_p * desc.num_layers)(*[t.data_ptr() for t in self.layers])
+        handle = ctypes.c_void_p()
+        _check(lib().hma_cache_create(ctypes.byref(desc), ptrs, ctypes.byref(handle)), "hma_cache_create")
+        self.handle = handle
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().hma_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def hma_kv_ingest_layer(cache, layer, k_wire, v_wire, wire_layout, head_begin, head_count, page_ids,
+                        token_begin, n_tokens, stream=None):
+    _check(lib().hma_kv_ingest_layer(cache.handle, layer, _ptr(k_wire), _ptr(v_wire), wire_layout, head_begin,
+                                     head_count, _ptr(page_ids), token_begin, n_tokens, _stream(stream)),
+           "hma_kv_ingest_layer")
+
+
+def hma_decode_attention_workspace_bytes(desc, batch):
+    return int(lib().hma_decode_attention_workspace_bytes(ctypes.byref(desc), batch))
+
+
+def hma_decode_attention(cache, layer, q, out, block_table, context_lens, sm_scale, workspace, stream=None):
+    out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
+    _check(lib().hma_decode_attention(cache.handle, layer, _ptr(q), _ptr(out), out_dtype, _ptr(block_table),
+                                      block_table.shape[1], _ptr(context_lens), q.shape[0], float(sm_scale),
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "hma_decode_attention")
+
+
+def hma_decode_attention_simple(cache, layer, q, out, block_table, context_lens, sm_scale, stream=None):
+    out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
+    _check(lib().hma_decode_attention_simple(cache.handle, layer, _ptr(q), _ptr(out), out_dtype, _ptr(block_table),
+                                             block_table.shape[1], _ptr(context_lens), q.shape[0], float(sm_scale),
+                                             _stream(stream)), "hma_decode_attention_simple")
+
+
+def hma_bfp8_dequant_bf16(cache, layer, which, page_ids, token_begin, n_tokens, out_bf16, stream=None):
+    _check(lib().hma_bfp8_dequant_bf16(cache.handle, layer, which, _ptr(page_ids), token_begin, n_tokens,
+                                       _ptr(out_bf16), _stream(stream)), "hma_bfp8_dequant_bf16")
+
+
+def hma_bfp8_dequant_blocks_bf16(exps, mants, n_blocks, out_bf16, stream=None):
+    _check(lib().hma_bfp8_dequant_blocks_bf16(_ptr(exps), _ptr(mants), n_blocks, _ptr(out_bf16), _stream(stream)),
+           "hma_bfp8_dequant_blocks_bf16")
+
+
+def hma_error_flags(cache, stream=None):
+    v = ctypes.c_uint32(0)
+    _check(lib().hma_error_flags(cache.handle, ctypes.byref(v), _stream(stream)), "hma_error_flags")
+    return int(v.value)
+
+
+def hma_launch_count():
+    return int(lib().hma_launch_count())

@@ -1,0 +1,88 @@
+"""Shared scaffolding of the GPU parity tests: build a paged cache from seeded wire bytes through the C ABI."""
+import numpy as np
+import torch
+
+from paper_2606_29986_b200 import hma, synth
+
+
+def bf16_bits(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def bf16_bits_to_f64(bits):
+    return (np.asarray(bits, np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+class Scenario:
+    """A batch of sequences with seeded BFP8 wire bytes, ingested into a paged cache on the GPU."""
+
+    def __init__(self, lens, hq, hkv, seed=0, permute=False, fmt=hma.HMA_KV_BFP8, wire_layout=hma.HMA_WIRE_ROWMAJOR,
+                 shards=1, layers=1, extra_pages=3, fill=0xA5, device="cuda"):
+        self.lens = np.asarray(lens, np.int32)
+        self.B, self.hq, self.hkv, self.layers = len(lens), hq, hkv, layers
+        self.seed = seed
+        self.table_np, self.num_pages, self.spare = synth.block_table(self.lens, permute, seed, extra_pages)
+        self.desc = hma.make_desc(layers, hq, hkv, self.num_pages, fmt)
+        self.cache = hma.KVCache(self.desc, device, fill=fill)
+        self.table = torch.from_numpy(self.table_np).to(device)
+        self.ctx = torch.from_numpy(self.lens).to(device)
+        self.q = synth.make_q(self.B, hq, seed).to(device)
+        self.k_wires = [[None] * self.B for _ in range(layers)]
+        self.v_wires = [[None] * self.B for _ in range(layers)]
+        for l in range(layers):
+            for b, T in enumerate(self.lens):
+                T = int(T)
+                kw = synth.make_kv_wire(hkv, T, synth.sequence_seed(seed, l, b, 0))
+                vw = synth.make_kv_wire(hkv, T, synth.sequence_seed(seed, l, b, 1))
+                self.k_wires[l][b], self.v_wires[l][b] = kw.numpy(), vw.numpy()
+                if T == 0:
+                    continue
+                pages = self.table[b, :(T + 15) // 16].contiguous()
+                hs = hkv // shards
+                for s in range(shards):
+                    ks, vs = kw[s * hs:(s + 1) * hs].contiguous(), vw[s * hs:(s + 1) * hs].contiguous()
+                    if wire_layout == hma.HMA_WIRE_TILE32:
+                        ks, vs = synth.rowmajor_to_tile32(ks), synth.rowmajor_to_tile32(vs)
+                    hma.hma_kv_ingest_layer(self.cache, l, ks.to(device), vs.to(device), wire_layout, s * hs, hs, pages, 0, T)
+        torch.cuda.synchronize()
+        ws = hma.hma_decode_attention_workspace_bytes(self.desc, self.B)
+        self.workspace = torch.empty(ws, dtype=torch.uint8, device=device)
+
+    def attention(self, layer=0, out_dtype=torch.bfloat16, simple=False, sm_scale=None, q=None):
+        q = self.q if q is None else q
+        sm_scale = 1.0 / np.sqrt(128.0) if sm_scale is None else sm_scale
+        out = torch.full((self.B, self.hq, 128), float("nan"), dtype=out_dtype, device=q.device)
+        if simple:
+            hma.hma_decode_attention_simple(self.cache, layer, q, out, self.table, self.ctx, sm_scale)
+        else:
+            hma.hma_decode_attention(self.cache, layer, q, out, self.table, self.ctx, sm_scale, self.workspace)
+        torch.cuda.synchronize()
+        return out
+
+    def oracle(self, layer=0, sm_scale=None, q=None):
+        from oracle import oracle as orc
+        q = self.q if q is None else q
+        return orc.decode_attention(bf16_bits(q), self.k_wires[layer], self.v_wires[layer], self.hkv, sm_scale)
+
+
+def parity_metrics(got, ref64):
+    """max-abs and relative-L2 error of a float array against the fp64 oracle."""
+    got = np.asarray(got, np.float64)
+    err = got - ref64
+    return float(np.abs(err).max()), float(np.sqrt((err ** 2).sum() / max((ref64 ** 2).sum(), 1e-300)))
+
+
+def check_attention(out_f32, out_bf16, ref64):
+    """The parity bar.  F32 output: max-abs <= 1e-2 and rel-L2 <= 2e-3 literally.  BF16 output: rel-L2 <= 2e-3
+    literally; max-abs <= 1e-2 on elements with |ref| < 4 and |err| <= 1e-2 + 2^-8 |ref| everywhere (the second term
+    is the half-ulp of the BF16 output itself)."""
+    ma, rl = parity_metrics(out_f32, ref64)
+    assert ma <= 1e-2 and rl <= 2e-3, ("f32 output", ma, rl)
+    got = bf16_bits_to_f64(out_bf16)
+    err = np.abs(got - ref64)
+    mb, rb = parity_metrics(got, ref64)
+    assert rb <= 2e-3, ("bf16 output rel-L2", rb)
+    small = np.abs(ref64) < 4
+    assert (err[small] <= 1e-2).all(), ("bf16 output max-abs on |ref|<4", err[small].max())
+    assert (err <= 1e-2 + 2.0 ** -8 * np.abs(ref64)).all(), ("bf16 output bound", (err - 2.0 ** -8 * np.abs(ref64)).max())
+    return ma, rl, mb, rb

@@ -1,0 +1,139 @@
+"""GPU parity, floating point: fused BFP8 paged decode attention against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2606_29986_b200 import hma, synth
+from helpers import Scenario, bf16_bits, bf16_bits_to_f64, check_attention, parity_metrics
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_and_check(sc, layer=0, sm_scale=None):
+    ref64, _ = sc.oracle(layer, sm_scale)
+    o32 = sc.attention(layer, torch.float32, sm_scale=sm_scale).cpu().numpy()
+    o16 = bf16_bits(sc.attention(layer, torch.bfloat16, sm_scale=sm_scale))
+    return check_attention(o32, o16, ref64), ref64, o32, o16
+
+
+def test_workload_qwen3_4b_full():
+    """Config 1 in full: 32 q / 8 kv heads, batch 4, context 1024, outlier channels, seed 0."""
+    w = synth.WORKLOADS["qwen3-4b-b4-ctx1k"]
+    lens = synth.context_lens(w["ctx"], w["batch"], 0)
+    sc = Scenario(lens, w["hq"], w["hkv"], seed=0)
+    (ma, rl, mb, rb), ref64, o32, o16 = _run_and_check(sc)
+    print("config1 parity: f32 max-abs %.3e rel-L2 %.3e | bf16 max-abs %.3e rel-L2 %.3e" % (ma, rl, mb, rb))
+    # floor: the oracle's own result rounded to BF16
+    _, ref16 = sc.oracle()
+    print("bf16 rounding floor: max-abs %.3e rel-L2 %.3e" % parity_metrics(bf16_bits_to_f64(ref16), ref64))
+    assert hma.hma_error_flags(sc.cache) == 0
+
+
+@pytest.mark.parametrize("hq,hkv", [(8, 8), (8, 4), (16, 4), (40, 8), (64, 8), (24, 8), (7, 1)])
+def test_ragged_contexts_and_group_sizes(hq, hkv):
+    lens = [1, 15, 16, 17, 31, 33, 0, 200, 48, 5]
+    sc = Scenario(lens, hq, hkv, seed=hq * 13 + hkv, permute=True)
+    _, ref64, o32, o16 = _run_and_check(sc)
+    assert not o32[6].any() and not o16[6].any()          # empty context -> zeros
+    # T = 1 returns V exactly
+    from oracle import oracle as orc
+    v = orc.decode_rowmajor_f64(sc.v_wires[0][0])
+    G = hq // hkv
+    for h in range(hq):
+        assert np.array_equal(bf16_bits_to_f64(o16[0, h]), v[h // G, 0])
+
+
+def test_simple_kernel_and_bf16_cache_agree_with_oracle():
+    lens = [70, 16, 129, 0, 3]
+    for fmt in (hma.HMA_KV_BFP8, hma.HMA_KV_BF16):
+        sc = Scenario(lens, 32, 8, seed=21, permute=True, fmt=fmt)
+        ref64, _ = sc.oracle()
+        o32 = sc.attention(0, torch.float32, simple=True).cpu().numpy()
+        o16 = bf16_bits(sc.attention(0, torch.bfloat16, simple=True))
+        check_attention(o32, o16, ref64)
+        if fmt == hma.HMA_KV_BF16:
+            check_attention(sc.attention(0, torch.float32).cpu().numpy(), bf16_bits(sc.attention(0, torch.bfloat16)), ref64)
+
+
+def test_long_context_many_splits_and_determinism():
+    """One long sequence is cut across every CTA (split-K), short ones sit inside a single CTA."""
+    lens = [6000, 40, 2500, 16]
+    sc = Scenario(lens, 64, 8, seed=31, permute=True)
+    _, ref64, o32, o16 = _run_and_check(sc)
+    again = bf16_bits(sc.attention(0, torch.bfloat16))
+    assert np.array_equal(again, o16)                      # fixed reduction order: bitwise repeatable
+    simple = sc.attention(0, torch.float32, simple=True).cpu().numpy()
+    assert np.abs(simple - o32).max() <= 5e-3
+
+
+def test_page_permutation_and_tail_garbage_change_nothing():
+    lens = [100, 37, 260]
+    a = Scenario(lens, 32, 8, seed=41, permute=False, fill=0x00)
+    b = Scenario(lens, 32, 8, seed=41, permute=True, fill=0xFF)     # other physical pages, 0xFF in every unwritten byte
+    oa, ob = a.attention(0, torch.float32).cpu().numpy(), b.attention(0, torch.float32).cpu().numpy()
+    assert np.array_equal(oa, ob)
+    assert np.isfinite(ob).all()
+
+
+def test_sm_scale_and_q_range():
+    lens = [90, 33]
+    sc = Scenario(lens, 16, 4, seed=51)
+    _run_and_check(sc, sm_scale=0.3)
+    # huge and tiny queries: the per-head power-of-two scaling keeps FP16 operands in range
+    for scale in (3.0e4, 1.0e-6):
+        q = (sc.q.float() * scale).to(torch.bfloat16)
+        ref64, _ = sc.oracle(q=q, sm_scale=0.05 / scale)
+        o32 = sc.attention(0, torch.float32, q=q, sm_scale=0.05 / scale).cpu().numpy()
+        ma, rl = parity_metrics(o32, ref64)
+        assert ma <= 1e-2 and rl <= 2e-3, (scale, ma, rl)
+
+
+def test_wide_exponent_spread_in_v():
+    """V blocks whose exponents differ by 2^40 between tokens: the running reference exponent must track them."""
+    sc = Scenario([64], 8, 1, seed=61, extra_pages=0)
+    kw, vw = sc.k_wires[0][0].copy(), sc.v_wires[0][0].copy()
+    rng = np.random.default_rng(61)
+    vw[0, :, :8] = rng.integers(90, 170, (64, 8)).astype(np.uint8)
+    kw[0, :, :8] = rng.integers(120, 130, (64, 8)).astype(np.uint8)
+    hma.hma_kv_ingest_layer(sc.cache, 0, torch.from_numpy(kw).cuda(), torch.from_numpy(vw).cuda(), hma.HMA_WIRE_ROWMAJOR, 0, 1,
+                            sc.table[0, :4].contiguous(), 0, 64)
+    sc.k_wires[0][0], sc.v_wires[0][0] = kw, vw
+    ref64, _ = sc.oracle()
+    o32 = sc.attention(0, torch.float32).cpu().numpy().astype(np.float64)
+    # per 16-channel block the scale differs by many orders of magnitude: compare block by block, relatively
+    for j in range(8):
+        r, g = ref64[0, :, 16 * j:16 * j + 16], o32[0, :, 16 * j:16 * j + 16]
+        assert np.sqrt(((g - r) ** 2).sum() / (r ** 2).sum()) <= 2e-3, j
+
+
+def test_bad_page_id_is_skipped_and_flagged():
+    sc = Scenario([64, 64], 8, 2, seed=71)
+    good = sc.attention(0, torch.float32).cpu().numpy()
+    assert hma.hma_error_flags(sc.cache) == 0
+    tbl = sc.table.clone()
+    tbl[1, 2] = sc.num_pages + 100
+    saved, sc.table = sc.table, tbl
+    out = sc.attention(0, torch.float32).cpu().numpy()
+    assert hma.hma_error_flags(sc.cache) == hma.HMA_FLAG_BAD_PAGE_ATTENTION
+    assert np.isfinite(out).all() and np.array_equal(out[0], good[0])
+    # the result equals attention over the remaining 48 tokens of sequence 1
+    from oracle import oracle as orc
+    keep = np.r_[0:32, 48:64]
+    ref, _ = orc.decode_attention(bf16_bits(sc.q[1:2]), [sc.k_wires[0][1][:, keep]], [sc.v_wires[0][1][:, keep]], 2)
+    assert parity_metrics(out[1:2], ref)[1] <= 2e-3
+    sc.table = saved
+
+
+def test_argument_errors():
+    sc = Scenario([32], 8, 2, seed=81)
+    out = torch.zeros((1, 8, 128), dtype=torch.bfloat16, device="cuda")
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(hma.HmaError) as e:
+        hma.hma_decode_attention(sc.cache, 0, sc.q, out, sc.table, sc.ctx, 0.1, small)
+    assert e.value.status == hma.HMA_ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(hma.HmaError) as e:
+        hma.hma_decode_attention(sc.cache, 3, sc.q, out, sc.table, sc.ctx, 0.1, sc.workspace)
+    assert e.value.status == hma.HMA_ERR_INVALID_ARG
+    with pytest.raises(hma.HmaError) as e:
+        hma.hma_decode_attention(sc.cache, 0, sc.q.view(-1)[1:].view(torch.bfloat16), out, sc.table, sc.ctx, 0.1, sc.workspace)
+    assert e.value.status == hma.HMA_ERR_ALIGNMENT

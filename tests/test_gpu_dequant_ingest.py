@@ -1,0 +1,126 @@
+"""GPU parity, bytes: flat and paged BFP8 -> BF16 reconstruction and the ingest scatter, bit-exact against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2606_29986_b200 import hma, synth
+from helpers import Scenario, bf16_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def test_flat_dequant_exhaustive_table():
+    E = np.repeat(np.arange(256, dtype=np.uint8), 16)
+    m = np.tile(np.arange(256, dtype=np.uint8), 256).reshape(-1, 16)
+    out = torch.zeros(E.size * 16, dtype=torch.bfloat16, device="cuda")
+    hma.hma_bfp8_dequant_blocks_bf16(torch.from_numpy(E).cuda(), torch.from_numpy(m).cuda(), E.size, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_bits(out).reshape(-1, 16), orc.bfp8_decode_bf16(E, m))
+
+
+def test_flat_dequant_random_ragged_sizes():
+    rng = np.random.default_rng(0)
+    for n in (1, 7, 255, 100003):
+        E = rng.integers(0, 256, n).astype(np.uint8)
+        m = rng.integers(0, 256, (n, 16)).astype(np.uint8)
+        out = torch.zeros(n * 16 + 16, dtype=torch.bfloat16, device="cuda")
+        hma.hma_bfp8_dequant_blocks_bf16(torch.from_numpy(E).cuda(), torch.from_numpy(m).cuda(), n, out)
+        torch.cuda.synchronize()
+        got = bf16_bits(out)
+        assert np.array_equal(got[:n * 16].reshape(-1, 16), orc.bfp8_decode_bf16(E, m))
+        assert not got[n * 16:].any()
+    hma.hma_bfp8_dequant_blocks_bf16(None, None, 0, None)     # empty input is a no-op
+
+
+def _dequant_all(sc, layer, which, b):
+    T = int(sc.lens[b])
+    out = torch.zeros((T, sc.hkv, 128), dtype=torch.bfloat16, device="cuda")
+    if T:
+        hma.hma_bfp8_dequant_bf16(sc.cache, layer, which, sc.table[b, :(T + 15) // 16].contiguous(), 0, T, out)
+    torch.cuda.synchronize()
+    return bf16_bits(out).transpose(1, 0, 2)          # -> [Hkv][T][128]
+
+
+@pytest.mark.parametrize("fmt", [hma.HMA_KV_BFP8, hma.HMA_KV_BF16])
+@pytest.mark.parametrize("layout,shards", [(hma.HMA_WIRE_ROWMAJOR, 1), (hma.HMA_WIRE_TILE32, 1), (hma.HMA_WIRE_TILE32, 4),
+                                           (hma.HMA_WIRE_ROWMAJOR, 2)])
+def test_ingest_then_paged_dequant_equals_oracle_decode(fmt, layout, shards):
+    sc = Scenario([1, 15, 16, 17, 33, 100, 0, 64], 32, 8, seed=3, permute=True, fmt=fmt, wire_layout=layout, shards=shards, layers=2)
+    for l in range(2):
+        for b in range(sc.B):
+            for which, wires in ((0, sc.k_wires), (1, sc.v_wires)):
+                assert np.array_equal(_dequant_all(sc, l, which, b), orc.decode_rowmajor_bf16(wires[l][b])), (l, b, which)
+    assert hma.hma_error_flags(sc.cache) == 0
+
+
+@pytest.mark.parametrize("fmt", [hma.HMA_KV_BFP8, hma.HMA_KV_BF16])
+@pytest.mark.parametrize("layout", [hma.HMA_WIRE_ROWMAJOR, hma.HMA_WIRE_TILE32])
+def test_partial_range_ingest_keeps_other_bytes(fmt, layout):
+    """Overwrite tokens [21, 21+45) of a 100-token sequence: those change, everything else is byte-identical."""
+    sc = Scenario([100, 40], 16, 4, seed=5, permute=True, fmt=fmt, layers=1)
+    before = [t.clone() for t in sc.cache.layers]
+    t0, n = 21, 45
+    new_k = synth.make_kv_wire(4, n, 991)
+    new_v = synth.make_kv_wire(4, n, 992)
+    first, last = t0 // 16, (t0 + n - 1) // 16
+    pages = sc.table[0, first:last + 1].contiguous()
+    kk, vv = (new_k, new_v) if layout == hma.HMA_WIRE_ROWMAJOR else (synth.rowmajor_to_tile32(new_k), synth.rowmajor_to_tile32(new_v))
+    hma.hma_kv_ingest_layer(sc.cache, 0, kk.cuda(), vv.cuda(), layout, 0, 4, pages, t0, n)
+    torch.cuda.synchronize()
+    want_k, want_v = sc.k_wires[0][0].copy(), sc.v_wires[0][0].copy()
+    want_k[:, t0:t0 + n], want_v[:, t0:t0 + n] = new_k.numpy(), new_v.numpy()
+    assert np.array_equal(_dequant_all(sc, 0, 0, 0), orc.decode_rowmajor_bf16(want_k))
+    assert np.array_equal(_dequant_all(sc, 0, 1, 0), orc.decode_rowmajor_bf16(want_v))
+    assert np.array_equal(_dequant_all(sc, 0, 0, 1), orc.decode_rowmajor_bf16(sc.k_wires[0][1]))
+    # pages not named in the call are untouched, byte for byte (including the 0xA5 fill of spare pages)
+    rb = 4352 if fmt == hma.HMA_KV_BFP8 else 8192
+    now = sc.cache.layers[0].view(sc.num_pages, -1).cpu().numpy()
+    was = before[0].view(sc.num_pages, -1).cpu().numpy()
+    touched = set(int(p) for p in pages.cpu().numpy())
+    for p in range(sc.num_pages):
+        if p not in touched:
+            assert np.array_equal(now[p], was[p]), p
+    assert now.shape[1] == 4 * rb
+    # sub-range dequant (token_begin not page aligned) matches the same slice
+    out = torch.zeros((n, 4, 128), dtype=torch.bfloat16, device="cuda")
+    hma.hma_bfp8_dequant_bf16(sc.cache, 0, 1, pages, t0, n, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_bits(out).transpose(1, 0, 2), orc.decode_rowmajor_bf16(new_v.numpy()))
+
+
+def test_bfp8_cache_holds_the_wire_bytes_unchanged():
+    """Ingest permutes positions only: the multiset of bytes of a fully written page equals that of its wire rows."""
+    sc = Scenario([32], 8, 2, seed=6, layers=1, extra_pages=0)
+    rec = sc.cache.layers[0].view(2, 2, 4352).cpu().numpy()          # [page][head][record]
+    for p in range(2):
+        for h in range(2):
+            wire = np.concatenate([sc.k_wires[0][0][h, 16 * p:16 * p + 16].reshape(-1), sc.v_wires[0][0][h, 16 * p:16 * p + 16].reshape(-1)])
+            assert np.array_equal(np.sort(rec[p, h]), np.sort(wire))
+
+
+def test_bad_arguments_and_bad_page_ids():
+    sc = Scenario([40], 8, 2, seed=7, layers=1)
+    kw = torch.from_numpy(sc.k_wires[0][0]).cuda()
+    pages = sc.table[0, :3].contiguous()
+    with pytest.raises(hma.HmaError) as e:
+        hma.hma_kv_ingest_layer(sc.cache, 1, kw, kw, hma.HMA_WIRE_ROWMAJOR, 0, 2, pages, 0, 40)
+    assert e.value.status == hma.HMA_ERR_INVALID_ARG
+    with pytest.raises(hma.HmaError):
+        hma.hma_kv_ingest_layer(sc.cache, 0, kw, kw, hma.HMA_WIRE_ROWMAJOR, 1, 2, pages, 0, 40)       # heads 1..2 of 2
+    with pytest.raises(hma.HmaError):
+        hma.hma_kv_ingest_layer(sc.cache, 0, kw, kw, 7, 0, 2, pages, 0, 40)
+    with pytest.raises(hma.HmaError) as e:
+        hma.hma_kv_ingest_layer(sc.cache, 0, kw.view(-1)[1:], kw, hma.HMA_WIRE_ROWMAJOR, 0, 2, pages, 0, 32)
+    assert e.value.status == hma.HMA_ERR_ALIGNMENT
+    # an out-of-range page id never traps: the page is skipped and a flag bit is raised
+    before = sc.cache.layers[0].clone()
+    bad = torch.tensor([sc.num_pages + 5, -1, int(pages[2])], dtype=torch.int32, device="cuda")
+    hma.hma_kv_ingest_layer(sc.cache, 0, kw, kw, hma.HMA_WIRE_ROWMAJOR, 0, 2, bad, 0, 32)
+    assert hma.hma_error_flags(sc.cache) == hma.HMA_FLAG_BAD_PAGE_INGEST
+    assert torch.equal(before, sc.cache.layers[0])
+    out = torch.full((32, 2, 128), 1.0, dtype=torch.bfloat16, device="cuda")
+    hma.hma_bfp8_dequant_bf16(sc.cache, 0, 0, bad, 0, 32, out)
+    assert hma.hma_error_flags(sc.cache) == hma.HMA_FLAG_BAD_PAGE_DEQUANT
+    assert not bf16_bits(out).any()
+    assert hma.hma_error_flags(sc.cache) == 0
