@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-side BFP8 KV path (one JSON line on stdout).
+
+A step is one decode pass of the whole batch: for every layer one hma_decode_attention call
+(fused BFP8 paged attention + cross-split reduction) on the main stream while, for the
+Qwen3-32B workload, one new 8192-token request's raw BFP8 bytes are ingested layer by layer
+on a side stream (hma_kv_ingest_layer, TILE32 wire, 4 producer shards).  `value` is decode
+tokens per second (batch / step time) with every input resident in HBM; `e2e` repeats the
+step with Q, the arriving wire bytes and the outputs in pinned host memory.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+"""
+import argparse
+import json
+import os
+import shutil
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2606_29986_b200 import synth  # noqa: E402
+
+DEFAULT_WORKLOAD = "qwen3-32b-b32-ctx8k"
+BFP8_ROW = 272      # bytes per (token, kv head): K 136 + V 136
+BF16_ROW = 512
+# DRAM bytes per launch of attn_bfp8_kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
+# see profiles/.  Keyed by workload; None where no capture exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        exe = shutil.which("nvidia-smi")
+        if not exe:
+            return
+        self.proc = subprocess.Popen([exe, "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                      "--format=csv,noheader,nounits", "-lms", "100"],
+                                     stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["not recorded: nvidia-smi absent"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 7 and r[3 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- workload on the GPU
+class Workload:
+    def __init__(self, name, device, seed=0, with_bf16=True, with_ingest=True, layers=None):
+        from paper_2606_29986_b200 import hma
+        self.hma, self.name, self.device = hma, name, device
+        w = synth.WORKLOADS[name]
+        self.hq, self.hkv, self.B, self.L = w["hq"], w["hkv"], w["batch"], layers or w["layers"]
+        self.lens = synth.context_lens(w["ctx"], self.B, seed)
+        self.sum_t = int(self.lens.sum())
+        self.ingest_tokens = 8192 if (with_ingest and name == DEFAULT_WORKLOAD) else 0
+        extra = (self.ingest_tokens + 15) // 16
+        table, self.num_pages, spare = synth.block_table(self.lens, w["permute"], seed, extra)
+        self.table = torch.from_numpy(table).to(device)
+        self.ctx = torch.from_numpy(self.lens).to(device)
+        self.spare = torch.from_numpy(np.ascontiguousarray(spare)).to(device)
+        self.sm_scale = 1.0 / np.sqrt(128.0)
+        self.caches = {"bfp8": hma.KVCache(hma.make_desc(self.L, self.hq, self.hkv, self.num_pages, hma.HMA_KV_BFP8), device)}
+        if with_bf16:
+            self.caches["bf16"] = hma.KVCache(hma.make_desc(self.L, self.hq, self.hkv, self.num_pages, hma.HMA_KV_BF16), device)
+        self.q = [synth.make_q(self.B, self.hq, seed + l, device) for l in range(self.L)]
+        self.out = torch.empty((self.L, self.B, self.hq, 128), dtype=torch.bfloat16, device=device)
+        ws = hma.hma_decode_attention_workspace_bytes(self.caches["bfp8"].desc, self.B)
+        self.workspace = torch.empty(ws, dtype=torch.uint8, device=device)
+        self.sample_wires = {}       # (layer, b) -> (k_wire, v_wire) numpy, kept for the parity sample and the CPU baseline
+        keep = {(0, 0), (self.L - 1, self.B - 1)}
+        for l in range(self.L):
+            for b in range(self.B):
+                T = int(self.lens[b])
+                kw = synth.make_kv_wire(self.hkv, T, synth.sequence_seed(seed, l, b, 0), device, synth.channel_seed(seed, l, 0))
+                vw = synth.make_kv_wire(self.hkv, T, synth.sequence_seed(seed, l, b, 1), device, synth.channel_seed(seed, l, 1))
+                pages = self.table[b, :(T + 15) // 16].contiguous()
+                for c in self.caches.values():
+                    hma.hma_kv_ingest_layer(c, l, kw, vw, hma.HMA_WIRE_ROWMAJOR, 0, self.hkv, pages, 0, T)
+                if (l, b) in keep:
+                    self.sample_wires[(l, b)] = (kw.cpu().numpy(), vw.cpu().numpy())
+            torch.cuda.synchronize(device)
+        # the arriving request: TILE32 wire, 4 shards x (hkv/4) heads, every layer, K and V
+        self.side = torch.cuda.Stream(device)
+        if self.ingest_tokens:
+            hs = self.hkv // 4
+            one = synth.rowmajor_to_tile32(synth.make_kv_wire(hs, self.ingest_tokens, 4242, device)).reshape(-1)
+            self.shard_bytes = one.numel()
+            self.wire_dev = torch.empty((self.L, 2, 4, self.shard_bytes), dtype=torch.uint8, device=device)
+            for l in range(self.L):
+                for t in range(2):
+                    for s in range(4):
+                        seed_ls = 4242 + ((l * 2 + t) * 4 + s)
+                        self.wire_dev[l, t, s] = synth.rowmajor_to_tile32(
+                            synth.make_kv_wire(hs, self.ingest_tokens, seed_ls, device)).reshape(-1)
+            self.wire_host = torch.empty(self.wire_dev.shape, dtype=torch.uint8, pin_memory=True)
+            self.wire_host.copy_(self.wire_dev)
+        self.q_host = torch.empty((self.L, self.B, self.hq, 128), dtype=torch.bfloat16, pin_memory=True)
+        for l in range(self.L):
+            self.q_host[l].copy_(self.q[l])
+        self.out_host = torch.empty(self.out.shape, dtype=torch.bfloat16, pin_memory=True)
+        self.q_stage = torch.empty((self.L, self.B, self.hq, 128), dtype=torch.bfloat16, device=device)
+        torch.cuda.synchronize(device)
+
+    def kv_bytes_per_layer(self, fmt):
+        return self.sum_t * self.hkv * (BFP8_ROW if fmt == "bfp8" else BF16_ROW)
+
+    def _ingest_all(self, wire, stream):
+        hma = self.hma
+        hs = self.hkv // 4
+        for l in range(self.L):
+            for s in range(4):
+                hma.hma_kv_ingest_layer(self.caches["bfp8"], l, wire[l, 0, s], wire[l, 1, s], hma.HMA_WIRE_TILE32,
+                                        s * hs, hs, self.spare, 0, self.ingest_tokens, stream)
+
+    def step(self, fmt="bfp8", ingest=True, host=False):
+        """One decode pass over all layers (+ the concurrent ingest).  Everything is enqueued; nothing syncs."""
+        hma = self.hma
+        main = torch.cuda.current_stream(self.device)
+        do_ingest = ingest and self.ingest_tokens and fmt == "bfp8"
+        if do_ingest:
+            self.side.wait_stream(main)
+            self._ingest_all(self.wire_host if host else self.wire_dev, self.side)
+        cache = self.caches[fmt]
+        for l in range(self.L):
+            q = self.q[l]
+            if host:
+                self.q_stage[l].copy_(self.q_host[l], non_blocking=True)
+                q = self.q_stage[l]
+            hma.hma_decode_attention(cache, l, q, self.out[l], self.table, self.ctx, self.sm_scale, self.workspace, main)
+            if host:
+                self.out_host[l].copy_(self.out[l], non_blocking=True)
+        if do_ingest:
+            main.wait_stream(self.side)
+
+    def time_steps(self, steps, warmup, **kw):
+        for _ in range(warmup):
+            self.step(**kw)
+        torch.cuda.synchronize(self.device)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(self.device)
+        e0.record()
+        for _ in range(steps):
+            self.step(**kw)
+        e1.record()
+        torch.cuda.synchronize(self.device)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1) / 1e3) / steps      # seconds per step
+
+    def time_layer_calls(self, fmt, reps):
+        """Average duration of one hma_decode_attention call, CUDA events around every call on its stream."""
+        cache = self.caches[fmt]
+        evs = []
+        for r in range(reps):
+            for l in range(self.L):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                self.hma.hma_decode_attention(cache, l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, self.workspace)
+                b.record()
+                evs.append((a, b))
+        torch.cuda.synchronize(self.device)
+        t = np.array([a.elapsed_time(b) for a, b in evs]) / 1e3
+        return float(t.mean()), float(np.median(t)), float(t.min())
+
+    def parity_sample(self):
+        """GPU output of sampled sequences against the oracle on the same wire bytes (full-size launch configuration)."""
+        from oracle import oracle as orc
+        res = []
+        for (l, b), (kw, vw) in self.sample_wires.items():
+            self.hma.hma_decode_attention(self.caches["bfp8"], l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, self.workspace)
+            torch.cuda.synchronize(self.device)
+            qb = self.q[l][b:b + 1].contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+            ref64, _ = orc.decode_attention(qb, [kw], [vw], self.hkv, self.sm_scale)
+            got = self.out[l][b].float().cpu().numpy().astype(np.float64)
+            err = got - ref64[0]
+            res.append({"layer": l, "seq": b, "max_abs": float(np.abs(err).max()),
+                        "rel_l2": float(np.sqrt((err ** 2).sum() / (ref64 ** 2).sum()))})
+        return res
+
+
+# ----------------------------------------------------------------------------- ranks
+def world():
+    return int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def barrier():
+    if torch.distributed.is_available() and torch.distributed.is_initialized():
+        torch.distributed.barrier()
+
+
+def max_over_ranks(x):
+    """Largest value of x over all ranks (the step time of the slowest rank)."""
+    if torch.distributed.is_available() and torch.distributed.is_initialized():
+        dev = "cuda" if torch.distributed.get_backend() == "nccl" else "cpu"
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        return float(t.item())
+    return x
+
+
+def aggregate_value(tokens_per_rank, seconds_per_step, n_ranks):
+    """Whole-job tokens/s: every rank decodes its own batch (no data-path collective), time = slowest rank."""
+    return tokens_per_rank * n_ranks / seconds_per_step
+
+
+# ----------------------------------------------------------------------------- CPU oracle timing
+def time_oracle(name, n_seq, seed=0, repeats=1):
+    """Seconds the CPU oracle needs for one layer of `n_seq` sequences of the workload; returns (seconds, threads, tokens)."""
+    from oracle import oracle as orc
+    w = synth.WORKLOADS[name]
+    lens = synth.context_lens(w["ctx"], w["batch"], seed)[:n_seq]
+    q = synth.make_q(n_seq, w["hq"], seed).view(torch.int16).numpy().view(np.uint16)
+    kw = [synth.make_kv_wire(w["hkv"], int(t), synth.sequence_seed(seed, 0, b, 0), channel_seed=synth.channel_seed(seed, 0, 0)).numpy() for b, t in enumerate(lens)]
+    vw = [synth.make_kv_wire(w["hkv"], int(t), synth.sequence_seed(seed, 0, b, 1), channel_seed=synth.channel_seed(seed, 0, 1)).numpy() for b, t in enumerate(lens)]
+    orc.decode_attention(q[:1], [kw[0][:, :64]], [vw[0][:, :64]], w["hkv"])      # load the library
+    best = 1e30
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        orc.decode_attention(q, kw, vw, w["hkv"])
+        best = min(best, time.perf_counter() - t0)
+    return best, orc.num_threads(), int(lens.sum())
+
+
+def reference_arm(args):
+    """The CPU oracle as it stands, on the host cores: each step is one layer of one sequence of the workload."""
+    ws, rank, _ = world()
+    if rank != 0:
+        return
+    name = args.workload
+    w = synth.WORKLOADS[name]
+    n_seq = 1
+    for _ in range(args.warmup):
+        time_oracle(name, n_seq)
+    t = []
+    threads = 1
+    for _ in range(args.steps):
+        sec, threads, toks = time_oracle(name, n_seq)
+        t.append(sec)
+    sec = float(np.mean(t))
+    # one layer of n_seq sequences took `sec`; a decode token needs all layers
+    value = n_seq / (sec * w["layers"])
+    line = {"impl": "reference", "metric": "decode_attn_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": name, "sample": "1 sequence x 1 layer per step, scaled to %d layers" % w["layers"]},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                             "sample": "layer 0 of sequence 0 (%d tokens, %d q heads) per step; tokens/s = 1 / (t * %d layers)" % (toks, w["hq"], w["layers"])},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-bf16", action="store_true", help="skip the BF16-KV comparison run")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--layers", type=int, default=None, help="development only: build fewer layers than the workload has")
+    ap.add_argument("--kernel-only", action="store_true", help="development only: print per-call kernel timing and exit")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    ws, rank, local = world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if ws > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    from paper_2606_29986_b200 import hma
+    hma.lib()
+
+    wl = Workload(args.workload, device, with_bf16=not args.no_bf16, layers=args.layers)
+    peak, peak_kind = measured_peak()
+
+    parity = wl.parity_sample() if rank == 0 else []
+
+    # per-call duration of the dominant kernel (decode attention), CUDA events around each call
+    wl.time_layer_calls("bfp8", 1)
+    call_mean, call_med, call_min = wl.time_layer_calls("bfp8", 3)
+    if args.kernel_only:
+        res = {"workload": args.workload, "layers_built": wl.L, "bfp8_us_per_call": [call_mean * 1e6, call_med * 1e6, call_min * 1e6],
+               "bfp8_gbs": wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9, "parity_sample": parity}
+        if "bf16" in wl.caches:
+            wl.time_layer_calls("bf16", 1)
+            m, md, mn = wl.time_layer_calls("bf16", 2)
+            res.update({"bf16_us_per_call": [m * 1e6, md * 1e6, mn * 1e6], "bf16_gbs": wl.kv_bytes_per_layer("bf16") / m / 1e9})
+        print(json.dumps(res))
+        return
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    sec = wl.time_steps(args.steps, args.warmup)
+    clocks = sampler.stop()
+    n0 = hma.hma_launch_count()
+    wl.step()
+    launches = hma.hma_launch_count() - n0          # kernels of this library per step
+    torch.cuda.synchronize(device)
+
+    sec_decode_only = wl.time_steps(args.steps, args.warmup, ingest=False)
+    sec_e2e = wl.time_steps(max(2, args.steps // 4), 3, host=True)
+    extra = {}
+    if "bf16" in wl.caches:
+        k = max(1, args.steps // 10)
+        sec_bf16 = wl.time_steps(k, 3 if k > 1 else 1, fmt="bf16", ingest=False)
+        extra["bf16_kv"] = {"tokens_per_s": aggregate_value(wl.B, sec_bf16, ws), "ms_per_step": sec_bf16 * 1e3,
+                            "kv_gbs": wl.kv_bytes_per_layer("bf16") * wl.L / sec_bf16 / 1e9, "steps": k,
+                            "bfp8_speedup": sec_bf16 / sec_decode_only}
+
+    kv_step = wl.kv_bytes_per_layer("bfp8") * wl.L
+    value = aggregate_value(wl.B, sec, ws)
+    achieved = wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9
+    q_bytes = wl.L * wl.B * wl.hq * 128 * 2
+    wire_bytes = int(wl.wire_host.numel()) if wl.ingest_tokens else 0
+    line = {
+        "metric": "decode_attn_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": ws, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bfp8 bytes (u8) -> f16 mma operands, f32 accumulate", "data": "synthetic",
+        "config": {"workload": args.workload, "q_heads": wl.hq, "kv_heads": wl.hkv, "batch_per_gpu": wl.B, "layers": wl.L,
+                   "sum_context": wl.sum_t, "page_tokens": 16, "kv_format": "bfp8", "parallelism": "replicas only",
+                   "layers_built": wl.L, "concurrent_ingest_tokens": wl.ingest_tokens, "l2": "inputs_larger_than_l2 (%.0f MB per layer, %d distinct layers)"
+                   % (wl.kv_bytes_per_layer("bfp8") / 1e6, wl.L)},
+        "kv_gbs": kv_step * ws / sec / 1e9,
+        "kv_gbs_frac_of_8000": kv_step / sec / 1e9 / 8000.0,
+        "clocks": clocks,
+        "e2e": {"value": aggregate_value(wl.B, sec_e2e, ws), "unit": "tokens/s", "ms_per_step": sec_e2e * 1e3,
+                "h2d_bytes_per_step": q_bytes + wire_bytes, "d2h_bytes_per_step": q_bytes},
+        "gpu_launches": int(launches * args.steps),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": "of " + peak_kind, "frac_of_8000": achieved / 8000.0,
+                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                     "kernel": "hma_decode_attention (attn_bfp8_kernel + attn_reduce_kernel)",
+                     "bytes_per_launch": wl.kv_bytes_per_layer("bfp8"), "us_per_launch_mean": call_mean * 1e6,
+                     "us_per_launch_median": call_med * 1e6, "us_per_launch_min": call_min * 1e6},
+        "decode_only": {"tokens_per_s": aggregate_value(wl.B, sec_decode_only, ws), "ms_per_step": sec_decode_only * 1e3,
+                        "kv_gbs": kv_step / sec_decode_only / 1e9, "slowdown_from_ingest": sec / sec_decode_only - 1.0},
+        "parity_sample": parity,
+    }
+    line.update(extra)
+    if rank == 0 and ws == 1 and not args.no_cpu:
+        n_seq = wl.B
+        t, threads, toks = time_oracle(args.workload, n_seq)
+        line["cpu_baseline"] = {"value": n_seq / (t * wl.L), "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                                "kv_gbs": toks * wl.hkv * BFP8_ROW / t / 1e9, "seconds": t,
+                                "sample": "layer 0 of all %d sequences (%d tokens x %d q heads); tokens/s = %d / (t x %d layers)"
+                                % (n_seq, toks, wl.hq, n_seq, wl.L)}
+    if rank == 0:
+        print(json.dumps(line))
+    if ws > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

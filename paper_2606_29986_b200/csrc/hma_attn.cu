@@ -233,40 +233,24 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------ producer warp
+        // Every lane owns one record of a chunk of up to 32 consecutive pages of a segment: it waits for
+        // its ring slot, then issues its own bulk copy, so 32 copies are set up in parallel.  The block
+        // table entries of the next chunk are fetched before the current chunk waits.
         uint64_t policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-        const int rb = kBfp8Record;
+        constexpr int rb = kBfp8Record;
         int b = b_cur, g = g_cur;
         int np = cum[b + 1] - cum[b];
         int p = (int)(w0 - ((int64_t)Hkv * cum[b] + (int64_t)g * np));
-        int64_t r = 0;
-        const int64_t R = w1 - w0;
+        const int R = (int)(w1 - w0);
+        int r = 0;
+        int chunk = min(min(32, np - p), R - r);
+        int32_t pid = lane < chunk ? a.block_table[(int64_t)b * a.max_pages + p + lane] : 0;
         bool alive = true;
-        while (r < R && alive) {
-            // up to 32 consecutive pages of the current segment: one coalesced block-table read
-            const int chunk = (int)min((int64_t)min(32, np - p), R - r);
-            int32_t pid = 0;
-            if (lane < chunk) pid = a.block_table[(int64_t)b * a.max_pages + p + lane];
-            for (int k = 0; k < chunk && alive; ++k) {
-                const int32_t id = __shfl_sync(0xFFFFFFFFu, pid, k);
-                const int64_t rr = r + k;
-                const int s = (int)(rr % kStages);
-                if (lane == 0) {
-                    if (rr >= kStages) alive = mbar_wait(empty0 + 8 * s, (uint32_t)((rr / kStages) - 1) & 1u, abort_word, a.cv.flags);
-                    if (alive) {
-                        if (id >= 0 && id < a.cv.num_pages) {
-                            stage_ok[s] = 1;
-                            mbar_arrive_expect_tx(full0 + 8 * s, rb);
-                            bulk_load(smem_u32(ring + s * rb), a.cv.layer + ((int64_t)id * Hkv + g) * rb, rb, full0 + 8 * s, policy);
-                        } else {
-                            stage_ok[s] = 0;
-                            atomicOr(a.cv.flags, HMA_FLAG_BAD_PAGE_ATTENTION);
-                            mbar_arrive(full0 + 8 * s);
-                        }
-                    }
-                }
-                alive = __shfl_sync(0xFFFFFFFFu, (int)alive, 0) != 0;
-            }
+        while (r < R) {
+            const int c_chunk = chunk, c_g = g, c_r = r;
+            const int32_t c_pid = pid;
+            // advance to the next chunk and prefetch its page ids
             r += chunk;
             p += chunk;
             if (p == np) {
@@ -277,14 +261,36 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                     if (b < B) np = cum[b + 1] - cum[b];
                 }
             }
-        }
-        if (!alive && lane == 0) {
-            // give the copies already issued a bounded chance to land before the CTA exits
-            for (int s = 0; s < kStages; ++s) {
-                int64_t last = -1;
-                for (int64_t q = s; q < r; q += kStages) last = q;
-                if (last < 0) continue;
-                for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(full0 + 8 * s, (uint32_t)(last / kStages) & 1u); ++it) {}
+            if (r < R) {
+                chunk = min(min(32, np - p), R - r);
+                pid = lane < chunk ? a.block_table[(int64_t)b * a.max_pages + p + lane] : 0;
+            }
+            if (lane < c_chunk) {
+                const int rr = c_r + lane;
+                const int s = rr % kStages;
+                if (rr >= kStages) alive = mbar_wait(empty0 + 8 * s, (uint32_t)((rr / kStages) - 1) & 1u, abort_word, a.cv.flags);
+                if (alive) {
+                    if (c_pid >= 0 && c_pid < a.cv.num_pages) {
+                        stage_ok[s] = 1;
+                        mbar_arrive_expect_tx(full0 + 8 * s, rb);
+                        bulk_load(smem_u32(ring + s * rb), a.cv.layer + ((int64_t)c_pid * Hkv + c_g) * rb, rb, full0 + 8 * s, policy);
+                    } else {
+                        stage_ok[s] = 0;
+                        atomicOr(a.cv.flags, HMA_FLAG_BAD_PAGE_ATTENTION);
+                        mbar_arrive(full0 + 8 * s);
+                    }
+                }
+            }
+            if (!__all_sync(0xFFFFFFFFu, alive)) {
+                // a wait ran out: give the copies already issued a bounded chance to land, then leave
+                const int issued = c_r;   // records below c_r were all issued
+                for (int s = lane; s < kStages; s += 32) {
+                    int last = -1;
+                    for (int q = s; q < issued; q += kStages) last = q;
+                    if (last < 0) continue;
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(full0 + 8 * s, (uint32_t)(last / kStages) & 1u); ++it) {}
+                }
+                return;
             }
         }
         return;

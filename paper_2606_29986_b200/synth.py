@@ -84,8 +84,11 @@ def outlier_channels(hkv, seed):
     return np.stack([flat // HEAD_DIM, flat % HEAD_DIM], axis=1)
 
 
-def make_kv_fp32(hkv, tokens, seed, device="cpu", outlier_scale=20.0):
-    """One tensor (K or V) of one sequence: FP32 [Hkv][tokens][128], N(0,1) with outlier channels."""
+def make_kv_fp32(hkv, tokens, seed, device="cpu", outlier_scale=20.0, channel_seed=None):
+    """One tensor (K or V) of one sequence: FP32 [Hkv][tokens][128], N(0,1) with outlier channels.
+
+    `channel_seed` picks the outlier channels; sequences of one layer share it (outlier channels
+    are a property of the layer, not of the sequence).  It defaults to `seed`."""
     if torch.device(device).type == "cpu":
         x = torch.from_numpy(np.random.default_rng(seed).standard_normal(
             (hkv, tokens, HEAD_DIM)).astype(np.float32))
@@ -93,7 +96,7 @@ def make_kv_fp32(hkv, tokens, seed, device="cpu", outlier_scale=20.0):
         g = torch.Generator(device=device)
         g.manual_seed(seed)
         x = torch.randn((hkv, tokens, HEAD_DIM), generator=g, device=device, dtype=torch.float32)
-    for h, c in outlier_channels(hkv, seed):
+    for h, c in outlier_channels(hkv, seed if channel_seed is None else channel_seed):
         x[int(h), :, int(c)] *= outlier_scale
     return x
 
@@ -126,9 +129,9 @@ def bfp8_encode(x):
     return out.reshape(*lead, ROW_BYTES)
 
 
-def make_kv_wire(hkv, tokens, seed, device="cpu"):
+def make_kv_wire(hkv, tokens, seed, device="cpu", channel_seed=None):
     """ROWMAJOR wire bytes [Hkv][tokens][136] of one tensor of one sequence."""
-    return bfp8_encode(make_kv_fp32(hkv, tokens, seed, device))
+    return bfp8_encode(make_kv_fp32(hkv, tokens, seed, device, channel_seed=channel_seed))
 
 
 def rowmajor_to_tile32(wire):
@@ -147,6 +150,11 @@ def rowmajor_to_tile32(wire):
     out[..., :64] = ex.permute(0, 1, 4, 2, 5, 3).reshape(H, tr, 4, 64)
     out[..., 64:] = mt.permute(0, 1, 4, 2, 5, 3, 6).reshape(H, tr, 4, 1024)
     return out
+
+
+def channel_seed(base_seed, layer, which):
+    """Seed of the outlier-channel choice of tensor `which` (0 = K, 1 = V) in a layer."""
+    return (base_seed * 1000003 + layer) * 2 + which + 900001
 
 
 def sequence_seed(base_seed, layer, b, which):

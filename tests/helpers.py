@@ -32,8 +32,8 @@ class Scenario:
         for l in range(layers):
             for b, T in enumerate(self.lens):
                 T = int(T)
-                kw = synth.make_kv_wire(hkv, T, synth.sequence_seed(seed, l, b, 0))
-                vw = synth.make_kv_wire(hkv, T, synth.sequence_seed(seed, l, b, 1))
+                kw = synth.make_kv_wire(hkv, T, synth.sequence_seed(seed, l, b, 0), channel_seed=synth.channel_seed(seed, l, 0))
+                vw = synth.make_kv_wire(hkv, T, synth.sequence_seed(seed, l, b, 1), channel_seed=synth.channel_seed(seed, l, 1))
                 self.k_wires[l][b], self.v_wires[l][b] = kw.numpy(), vw.numpy()
                 if T == 0:
                     continue
