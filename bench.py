@@ -187,7 +187,7 @@ class Workload:
         barrier()
         return max_over_ranks(e0.elapsed_time(e1) / 1e3) / steps      # seconds per step
 
-    def time_layer_calls(self, fmt, reps):
+    def time_layer_calls(self, fmt, reps, probe=False):
         """Average duration of one hma_decode_attention call, CUDA events around every call on its stream."""
         cache = self.caches[fmt]
         evs = []
@@ -195,7 +195,12 @@ class Workload:
             for l in range(self.L):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record()
-                self.hma.hma_decode_attention(cache, l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, self.workspace)
+                if probe == "alu":
+                    self.hma.hma_attention_alu_probe(cache, l, self.table, self.ctx, self.workspace)
+                elif probe:
+                    self.hma.hma_kv_read_probe(cache, l, self.table, self.ctx, self.workspace)
+                else:
+                    self.hma.hma_decode_attention(cache, l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, self.workspace)
                 b.record()
                 evs.append((a, b))
         torch.cuda.synchronize(self.device)
@@ -326,9 +331,14 @@ def main():
     # per-call duration of the dominant kernel (decode attention), CUDA events around each call
     wl.time_layer_calls("bfp8", 1)
     call_mean, call_med, call_min = wl.time_layer_calls("bfp8", 3)
+    wl.time_layer_calls("bfp8", 1, probe=True)
+    probe_mean, probe_med, probe_min = wl.time_layer_calls("bfp8", 3, probe=True)
     if args.kernel_only:
-        res = {"workload": args.workload, "layers_built": wl.L, "bfp8_us_per_call": [call_mean * 1e6, call_med * 1e6, call_min * 1e6],
-               "bfp8_gbs": wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9, "parity_sample": parity}
+        wl.time_layer_calls("bfp8", 1, probe="alu")
+        alu_mean = wl.time_layer_calls("bfp8", 3, probe="alu")[0]
+        res = {"alu_probe_us_per_call": alu_mean * 1e6, "workload": args.workload, "layers_built": wl.L, "bfp8_us_per_call": [call_mean * 1e6, call_med * 1e6, call_min * 1e6],
+               "bfp8_gbs": wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9, "probe_us_per_call": probe_mean * 1e6,
+               "probe_gbs": wl.kv_bytes_per_layer("bfp8") / probe_mean / 1e9, "parity_sample": parity}
         if "bf16" in wl.caches:
             wl.time_layer_calls("bf16", 1)
             m, md, mn = wl.time_layer_calls("bf16", 2)
@@ -377,6 +387,8 @@ def main():
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": "of " + peak_kind, "frac_of_8000": achieved / 8000.0,
                      "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                     "probe_gbs": wl.kv_bytes_per_layer("bfp8") / probe_mean / 1e9,
+                     "frac_of_probe": probe_mean / call_mean,
                      "kernel": "hma_decode_attention (attn_bfp8_kernel + attn_reduce_kernel)",
                      "bytes_per_launch": wl.kv_bytes_per_layer("bfp8"), "us_per_launch_mean": call_mean * 1e6,
                      "us_per_launch_median": call_med * 1e6, "us_per_launch_min": call_min * 1e6},

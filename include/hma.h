@@ -154,6 +154,21 @@ hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer
                                          const int32_t *context_lens, int32_t batch, float sm_scale,
                                          void *stream);
 
+/* Bandwidth probe: streams exactly the page records hma_decode_attention would read (same block
+ * tables, same work split, same bulk-copy ring) and does no arithmetic and no output.  Its time is
+ * the ceiling the attention kernel's memory pipeline can reach (section 2.2: decode is memory-bound).
+ * BFP8 caches only.  Workspace as for hma_decode_attention. */
+hma_status_t hma_kv_read_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
+                               int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/* Diagnostic twin of the probe: the arithmetic of every record on whatever shared memory holds, with no
+ * loads and no output; its time is the attention kernel's instruction-issue floor.  The paper has no
+ * counterpart; it exists so that the benchmark can say which of the two floors binds. */
+hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
+                                     int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
+                                     void *workspace, size_t workspace_bytes, void *stream);
+
 /*
  * One-shot reconstruction (section 3.3): tokens [token_begin, token_begin+n_tokens) of a request,
  * tensor `which` (0 = K, 1 = V), all kv heads -> row-major BF16 [n_tokens][num_kv_heads][128].
@@ -173,6 +188,9 @@ hma_status_t hma_bfp8_dequant_blocks_bf16(const uint8_t *exps, const uint8_t *ma
 hma_status_t hma_error_flags(const hma_cache_t *cache, uint32_t *host_out, void *stream);
 
 const char *hma_status_string(int32_t status);
+
+/* Text of the CUDA runtime error behind the calling thread's most recent HMA_ERR_CUDA. */
+const char *hma_last_cuda_error(void);
 
 /* Number of kernels this library has launched in the calling process (for launch accounting). */
 int64_t hma_launch_count(void);

@@ -22,13 +22,20 @@
 
 namespace hma {
 
-constexpr int kConsumerWarps = 8;
+// 15 consumer warps + 1 producer warp = 16 warps, four per SM sub-partition: each sub-partition has 16384
+// registers, so a 17th warp would cap every thread at 96 registers instead of 128.
+constexpr int kConsumerWarps = 15;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kStages = 32;                       // ring depth; multiple of kConsumerWarps
+constexpr int kStages = 45;                       // ring depth
+// A ring slot must be used by the same consumer warp every time round (within a segment): a warp that ran two
+// laps ahead of the slot's previous owner would see the slot's older completed phase and read stale bytes.
+static_assert(kStages % kConsumerWarps == 0, "ring depth must be a multiple of one round of the consumer warps");
 constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile: o[8][128], m[8], l[8]
-constexpr int kCombStride = 132;                  // per (warp, head): o[128], m, l (+pad)
+constexpr int kSlots = 4;                         // states held in shared memory during the merge
+constexpr int kSlotFloats = 1024 + 16;            // one warp's state: 32 accumulators per lane, then m, l per head pair
+static_assert(kSlots * kSlotFloats * 4 >= kConsumerWarps * 768, "per-warp scratch tables live inside the merge slots");
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int kMaxBatch = 8192;
+constexpr int kMaxBatch = 768;
 constexpr int kMaxCtas = 1024;
 
 struct AttnArgs {
@@ -43,6 +50,7 @@ struct AttnArgs {
     float sm_scale;
     int32_t *cum;        // workspace: pages before each sequence, batch+1 entries
     float *tiles;        // workspace: partial tiles
+    int probe;           // 1: stream the records through the ring and do no arithmetic (bandwidth probe)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -103,6 +111,14 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
     return v;
 }
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t x, uint32_t y)
+{
+    asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
     uint32_t d;
@@ -171,8 +187,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
 {
     // shared memory carve-up
     uint8_t *ring = smem_raw;                                                   // kStages x 4352
-    float *comb = reinterpret_cast<float *>(ring + kStages * kBfp8Record);       // [warps][8][kCombStride]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(comb + kConsumerWarps * 8 * kCombStride);   // full[kStages], empty[kStages]
+    float *comb = reinterpret_cast<float *>(ring + kStages * kBfp8Record);       // merge slots / per-warp scratch
+    uint64_t *bars = reinterpret_cast<uint64_t *>(comb + kSlots * kSlotFloats);   // full[kStages], empty[kStages]
     int *stage_ok = reinterpret_cast<int *>(bars + 2 * kStages);                 // [kStages]
     int *misc = stage_ok + kStages;                                              // [0] abort word, [1..] scan scratch
     int *cum = misc + 16 + kThreads;                                             // [batch + 1]
@@ -247,6 +263,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         int chunk = min(min(32, np - p), R - r);
         int32_t pid = lane < chunk ? a.block_table[(int64_t)b * a.max_pages + p + lane] : 0;
         bool alive = true;
+        if (a.probe >= 2) return;            // arithmetic-only diagnostic: nothing is loaded
         while (r < R) {
             const int c_chunk = chunk, c_g = g, c_r = r;
             const int32_t c_pid = pid;
@@ -297,16 +314,25 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
     }
 
     // ---------------------------------------------------------------- consumer warps
+    // One record (16 tokens of one kv head) per warp iteration; a ring slot belongs to the same warp on every lap.
     const int gq = lane >> 2, t4 = lane & 3;
     const float kLog2e = 1.4426950408889634f;
+    // per-warp scratch inside the merge area (idle until the segment ends):
+    // fp32 Q.K^T scales 2^(E-127) of every (token, block) and FP16 P.V scales of every (token pair, block)
+    const uint32_t scrK = smem_u32(comb) + warp * 768;     // 512 B
+    const uint32_t scrV = scrK + 512;                      // 256 B
     int64_t w = w0;
     int b = b_cur, g = g_cur;
     bool alive = true;
-    while (w < w1) {
+    while (w < w1 && alive) {
         const int np = cum[b + 1] - cum[b];
         const int64_t seg0 = (int64_t)Hkv * cum[b] + (int64_t)g * np, seg1 = seg0 + np;
         const int64_t lo = max(seg0, w0), hi = min(seg1, w1);
         const int T = min(a.ctx[b], a.max_pages * kPageTokens);
+        const int rbase = (int)(lo - w0);            // CTA-local index of the segment's first record here
+        const int rend = (int)(hi - w0);
+        const int page0 = (int)(lo - seg0);          // page of the sequence that record rbase holds
+        const int tail = T - (np - 1) * kPageTokens; // valid tokens of the sequence's last page, 1..16
 
         // ---- Q fragments of this (sequence, kv head): FP16, one power-of-two scale per head ----
         uint32_t qf[8][2];
@@ -314,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         {
             float f[8][4];
             float amax = 0.f;
-            const bool hv = gq < G;
+            const bool hv = gq < G && !a.probe;      // the probes have no Q: nothing is read through a.q
             const uint16_t *qp = a.q + ((int64_t)b * a.cv.num_q_heads + (int64_t)g * G + (hv ? gq : 0)) * kHeadDim + 4 * t4;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -348,29 +374,80 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         float o[8][4];
 #pragma unroll
         for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
-        int Rall[8];                                    // reference exponent of each V channel block
-        uint32_t Kpk[8];                                // (30 - R) in both 16-bit lanes
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { Rall[j] = 0; Kpk[j] = 30u * 0x00010001u; }
-        int Rmine = 0;                                  // R of block (lane & 7)
+        int Rmine = 0;                                  // reference exponent of V channel block (lane & 7)
 
-        // first record of this segment owned by this warp: CTA-local index r with r % warps == warp
-        int64_t r = lo - w0;
-        r += (warp - (int)(r % kConsumerWarps) + kConsumerWarps) % kConsumerWarps;
-        for (; alive && r < hi - w0; r += kConsumerWarps) {
-            const int s = (int)(r % kStages);
-            alive = mbar_wait(full0 + 8 * s, (uint32_t)(r / kStages) & 1u, abort_word, a.cv.flags);
-            if (!alive) break;
-            const int page = (int)(w0 + r - seg0);
-            const uint32_t sp = smem_u32(ring + s * kBfp8Record);
-            if (stage_ok[s]) {
-                const int nvalid = min(kPageTokens, T - page * kPageTokens);
-                // ================= Q.K^T =================
-                const uint4 ke = lds128(sp + gq * 16);    // exponents: token gq blocks 0-3 | 4-7, token gq+8 blocks 0-3 | 4-7
-                uint4 km[4];
+        int r = rbase + warp;
+        int stage = r % kStages;
+        uint32_t par = (uint32_t)(r / kStages) & 1u;
+        for (; r < rend; r += kConsumerWarps) {
+            if (a.probe < 2) {
+                alive = mbar_wait(full0 + 8 * stage, par, abort_word, a.cv.flags);
+                if (!alive) break;
+            }
+            const uint32_t sp = smem_u32(ring) + stage * kBfp8Record;
+            const uint32_t my_empty = empty0 + 8 * stage;
+            const bool ok = a.probe >= 2 || stage_ok[stage] != 0;
+            stage += kConsumerWarps;
+            if (stage >= kStages) { stage -= kStages; par ^= 1u; }
+            if (a.probe == 1 || !ok) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(my_empty);
+                continue;
+            }
+            const int page = page0 + (r - rbase);
+            const int nvalid = page == np - 1 ? tail : kPageTokens;
+
+            // ---- exponents: fp32 scales for Q.K^T, reference-exponent check and FP16 scales for P.V ----
+            {
+                const uint32_t kw = lds32(sp + lane * 4);
+                uint32_t vw = lds32(sp + kBfp8Half + lane * 4);
+                if (nvalid < kPageTokens) {
+                    // exponent bytes of masked tokens count as 0: they neither raise the reference exponent
+                    // nor produce non-finite weights
+                    uint32_t keep = 0;
+                    const int tt = lane >> 3;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) km[c] = lds128(sp + 128 + c * 512 + lane * 16);
-                float sc[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int k = 0; k < 4; ++k)
+                        if (2 * tt + (k & 1) + 8 * (k >> 1) < nvalid) keep |= 0xFFu << (8 * k);
+                    vw &= keep;
+                }
+                sts128(scrK + lane * 16, (kw << 23) & 0x7F800000u, (kw << 15) & 0x7F800000u, (kw << 7) & 0x7F800000u,
+                       (kw >> 1) & 0x7F800000u);
+                const uint32_t mx2 = __vmaxu2((vw >> 8) & 0x00FF00FFu, vw & 0x00FF00FFu);
+                int emax = (int)max(mx2 & 0xFFFFu, mx2 >> 16);
+                if (__any_sync(0xFFFFFFFFu, emax > Rmine)) {
+                    // a V block exponent above the reference: raise it and rescale that block's accumulators
+                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
+                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
+                    const int Rnew = max(Rmine, emax);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
+                        const float fr = dlt < -126 ? 0.f : pow2_field(127 + dlt);
+                        o[j][0] *= fr; o[j][1] *= fr; o[j][2] *= fr; o[j][3] *= fr;
+                    }
+                    Rmine = Rnew;
+                }
+                // FP16 scale 2^(E - R + 15) of every (token pair, block): exponent field max(E - R + 30, 0)
+                const uint32_t kmine = ((uint32_t)(30 - Rmine) & 0xFFFFu) * 0x00010001u;
+                sts64(scrV + lane * 8, __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4140u), kmine, 0u) << 10,
+                      __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4342u), kmine, 0u) << 10);
+            }
+            uint4 km[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) km[c] = lds128(sp + 128 + c * 512 + lane * 16);
+            __syncwarp();
+
+            // ================= Q.K^T =================
+            float sc[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                float ks[16];      // 2^(E-127): token gq blocks 0..7, token gq+8 blocks 0..7
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 v = lds128(scrK + gq * 64 + c * 16);
+                    ks[4 * c] = __uint_as_float(v.x); ks[4 * c + 1] = __uint_as_float(v.y);
+                    ks[4 * c + 2] = __uint_as_float(v.z); ks[4 * c + 3] = __uint_as_float(v.w);
+                }
                 const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -384,32 +461,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                     af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
                     float d[4];
                     mma_f16(d, af, qf[j][0], qf[j][1], zero4);
-                    const uint32_t el = j < 4 ? ke.x : ke.y, eh = j < 4 ? ke.z : ke.w;
-                    const int sh = 23 - 8 * (j & 3);
-                    const float fl = __uint_as_float((sh >= 0 ? el << sh : el >> -sh) & 0x7F800000u);   // 2^(E-127)
-                    const float fh = __uint_as_float((sh >= 0 ? eh << sh : eh >> -sh) & 0x7F800000u);
-                    sc[0] = fmaf(d[0], fl, sc[0]);
-                    sc[1] = fmaf(d[1], fl, sc[1]);
-                    sc[2] = fmaf(d[2], fh, sc[2]);
-                    sc[3] = fmaf(d[3], fh, sc[3]);
+                    sc[0] = fmaf(d[0], ks[j], sc[0]);
+                    sc[1] = fmaf(d[1], ks[j], sc[1]);
+                    sc[2] = fmaf(d[2], ks[8 + j], sc[2]);
+                    sc[3] = fmaf(d[3], ks[8 + j], sc[3]);
                 }
-                float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
-                if (nvalid < kPageTokens) {
-                    if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
-                    if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
-                    // zero the exponent bytes of masked tokens in the V part so they neither raise the
-                    // reference exponent nor produce non-finite weights
-                    const uint32_t wa = sp + kBfp8Half + lane * 4;
-                    uint32_t wv = lds32(wa), keep = 0;
-                    const int tt = lane >> 3;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (2 * tt + (k & 1) + 8 * (k >> 1) < nvalid) keep |= 0xFFu << (8 * k);
-                    sts32(wa, wv & keep);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // a later bulk copy overwrites these bytes
-                    __syncwarp();
-                }
-                // ================= online softmax (log2 domain) =================
+            }
+            float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
+            if (nvalid < kPageTokens) {
+                if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
+                if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
+            }
+            // ================= online softmax (log2 domain) =================
+            // The warp-wide maximum is only formed when some score exceeds the running maximum.
+            if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
                 float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
 #pragma unroll
                 for (int d = 4; d <= 16; d <<= 1) {
@@ -417,39 +482,25 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                     mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
                 }
                 const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-                // V exponents of this lane's (token quad, block): does any exceed the block's reference?
-                const uint32_t vw = lds32(sp + kBfp8Half + lane * 4);
-                const uint32_t mx2 = __vmaxu2((vw >> 8) & 0x00FF00FFu, vw & 0x00FF00FFu);
-                int emax = (int)max(mx2 & 0xFFFFu, mx2 >> 16);
-                if (__any_sync(0xFFFFFFFFu, mn0 != m0 || mn1 != m1 || emax > Rmine)) {
-                    const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
-                    m0 = mn0;
-                    m1 = mn1;
-                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
-                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
-                    Rmine = max(Rmine, emax);
-                    lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
+                const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
+                m0 = mn0;
+                m1 = mn1;
+                lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int rn = __shfl_sync(0xFFFFFFFFu, Rmine, j);
-                        const int dlt = Rall[j] - rn;                       // <= 0
-                        const float fr = dlt < -126 ? 0.f : pow2_field(127 + dlt);
-                        Rall[j] = rn;
-                        Kpk[j] = ((uint32_t)(30 - rn) & 0xFFFFu) * 0x00010001u;
-                        const float f0 = a0 * fr, f1 = a1 * fr;
-                        o[j][0] *= f0; o[j][1] *= f1; o[j][2] *= f0; o[j][3] *= f1;
-                    }
-                }
-                const float p0 = ex2f(s0 - m0), p1 = ex2f(s1 - m1), p2 = ex2f(s2 - m0), p3 = ex2f(s3 - m1);
-                // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
-                const uint32_t pb0 = movmatrix_trans(pack_half2(p0, p1));      // tokens 2*t4, 2*t4+1 of head gq
-                const uint32_t pb1 = movmatrix_trans(pack_half2(p2, p3));      // tokens 2*t4+8, 2*t4+9
-                {
-                    const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
-                    mma_f16_acc(lacc, ones, pb0, pb1);
-                }
-                // ================= P.V =================
-                const uint4 ve0 = lds128(sp + kBfp8Half + t4 * 32), ve1 = lds128(sp + kBfp8Half + t4 * 32 + 16);
+                for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
+            }
+            // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
+            const uint32_t pb0 = movmatrix_trans(pack_half2(ex2f(s0 - m0), ex2f(s1 - m1)));   // tokens 2*t4, 2*t4+1 of head gq
+            const uint32_t pb1 = movmatrix_trans(pack_half2(ex2f(s2 - m0), ex2f(s3 - m1)));   // tokens 2*t4+8, 2*t4+9
+            {
+                const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
+                mma_f16_acc(lacc, ones, pb0, pb1);
+            }
+            // ================= P.V =================
+            {
+                uint4 vs[4];           // (f01, f89) of blocks 2c, 2c+1
+#pragma unroll
+                for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + t4 * 64 + c * 16);
                 uint4 vm[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) vm[c] = lds128(sp + kBfp8Half + 128 + c * 512 + lane * 16);
@@ -462,74 +513,101 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                     af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
                     af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
                     af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
-                    const uint4 &ee = j < 4 ? ve0 : ve1;
-                    const uint32_t ew = (j & 3) == 0 ? ee.x : (j & 3) == 1 ? ee.y : (j & 3) == 2 ? ee.z : ee.w;
-                    // FP16 scale 2^(E - R + 15) per token: exponent field max(E - R + 30, 0)
-                    const uint32_t f01 = __viaddmax_s16x2_relu(prmt(ew, 0u, 0x4140u), Kpk[j], 0u) << 10;
-                    const uint32_t f89 = __viaddmax_s16x2_relu(prmt(ew, 0u, 0x4342u), Kpk[j], 0u) << 10;
+                    const uint32_t f01 = (j & 1) ? vs[j >> 1].z : vs[j >> 1].x, f89 = (j & 1) ? vs[j >> 1].w : vs[j >> 1].y;
                     mma_f16_acc(o[j], af, hmul2_u32(pb0, f01), hmul2_u32(pb1, f89));
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8 * s);
+            __syncwarp();      // every lane is done with the ring slot and with the scratch tables
+            if (lane == 0 && a.probe < 2) mbar_arrive(my_empty);
         }
 
-        // ---- merge the warps' partial states of this segment ----
-        {
-            float *mine = comb + warp * 8 * kCombStride;
+        // ---- merge the warps' states of this segment: pairwise tree, at most kSlots states in shared memory ----
+        consumer_bar_sync();                           // the scratch tables (same memory as the slots) are idle now
+        if (!a.probe && alive) {
+            // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                // accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
-                const float vs = pow2_field(min(Rall[j] + 3, 254));
-                mine[(2 * t4) * kCombStride + 16 * j + gq] = o[j][0] * vs;
-                mine[(2 * t4 + 1) * kCombStride + 16 * j + gq] = o[j][1] * vs;
-                mine[(2 * t4) * kCombStride + 16 * j + gq + 8] = o[j][2] * vs;
-                mine[(2 * t4 + 1) * kCombStride + 16 * j + gq + 8] = o[j][3] * vs;
-            }
-            if (gq == 0) {
-                mine[(2 * t4) * kCombStride + 128] = m0;
-                mine[(2 * t4) * kCombStride + 129] = lacc[0];
-                mine[(2 * t4 + 1) * kCombStride + 128] = m1;
-                mine[(2 * t4 + 1) * kCombStride + 129] = lacc[1];
+                const float vsc = pow2_field(min(__shfl_sync(0xFFFFFFFFu, Rmine, j) + 3, 254));
+                o[j][0] *= vsc; o[j][1] *= vsc; o[j][2] *= vsc; o[j][3] *= vsc;
             }
         }
-        consumer_bar_sync();
-        {
+        float l0 = lacc[0], l1 = lacc[1];
+#pragma unroll 1
+        for (int n = kConsumerWarps; n > 1; n = (n + 1) / 2) {
+            const int half = (n + 1) / 2;              // warps [half, n) hand their state to warps [0, n - half)
+#pragma unroll 1
+            for (int base = 0; base < n - half; base += kSlots) {
+                const int wr = warp - half - base;     // slot this warp writes in this round, if in [0, kSlots)
+                if (!a.probe && warp >= half && warp < n && wr >= 0 && wr < kSlots) {
+                    float *slot = comb + wr * kSlotFloats;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) slot[(j * 4 + k) * 32 + lane] = o[j][k];
+                    if (gq == 0) {
+                        slot[1024 + t4 * 4 + 0] = m0; slot[1024 + t4 * 4 + 1] = m1;
+                        slot[1024 + t4 * 4 + 2] = l0; slot[1024 + t4 * 4 + 3] = l1;
+                    }
+                }
+                consumer_bar_sync();
+                const int rd = warp - base;            // slot this warp reads in this round, if in [0, kSlots)
+                if (!a.probe && warp < n - half && rd >= 0 && rd < kSlots) {
+                    const float *slot = comb + rd * kSlotFloats;
+                    const float pm0 = slot[1024 + t4 * 4 + 0], pm1 = slot[1024 + t4 * 4 + 1];
+                    const float pl0 = slot[1024 + t4 * 4 + 2], pl1 = slot[1024 + t4 * 4 + 3];
+                    const float M0 = fmaxf(m0, pm0), M1 = fmaxf(m1, pm1);
+                    const float a0 = m0 == -INFINITY ? 0.f : ex2f(m0 - M0), a1 = m1 == -INFINITY ? 0.f : ex2f(m1 - M1);
+                    const float c0 = pm0 == -INFINITY ? 0.f : ex2f(pm0 - M0), c1 = pm1 == -INFINITY ? 0.f : ex2f(pm1 - M1);
+                    l0 = l0 * a0 + pl0 * c0;
+                    l1 = l1 * a1 + pl1 * c1;
+                    m0 = M0;
+                    m1 = M1;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        o[j][0] = o[j][0] * a0 + slot[(j * 4 + 0) * 32 + lane] * c0;
+                        o[j][1] = o[j][1] * a1 + slot[(j * 4 + 1) * 32 + lane] * c1;
+                        o[j][2] = o[j][2] * a0 + slot[(j * 4 + 2) * 32 + lane] * c0;
+                        o[j][3] = o[j][3] * a1 + slot[(j * 4 + 3) * 32 + lane] * c1;
+                    }
+                }
+                consumer_bar_sync();
+            }
+        }
+        if (warp == 0 && !a.probe && alive) {
             const bool whole = lo == seg0 && hi == seg1;
-            const int64_t tile = (int64_t)blockIdx.x + ((int64_t)b * Hkv + g);
-            float *tp = a.tiles + tile * kTileFloats;
-            for (int idx = tid; idx < G * kHeadDim; idx += kConsumerWarps * 32) {
-                const int h = idx >> 7, c = idx & 127;
-                float M = -INFINITY;
+            const int h0 = 2 * t4, h1 = 2 * t4 + 1;
+            if (whole) {
+                const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+                const int64_t ob = ((int64_t)b * a.cv.num_q_heads + (int64_t)g * G) * kHeadDim;
 #pragma unroll
-                for (int ww = 0; ww < kConsumerWarps; ++ww) M = fmaxf(M, comb[(ww * 8 + h) * kCombStride + 128]);
-                float num = 0.f, den = 0.f;
+                for (int j = 0; j < 8; ++j)
 #pragma unroll
-                for (int ww = 0; ww < kConsumerWarps; ++ww) {
-                    const float mw = comb[(ww * 8 + h) * kCombStride + 128];
-                    const float wgt = mw == -INFINITY ? 0.f : ex2f(mw - M);
-                    num = fmaf(wgt, comb[(ww * 8 + h) * kCombStride + c], num);
-                    den = fmaf(wgt, comb[(ww * 8 + h) * kCombStride + 129], den);
-                }
-                if (whole) {
-                    const float res = den > 0.f ? num / den : 0.f;
-                    const int64_t oi = ((int64_t)b * a.cv.num_q_heads + (int64_t)g * G + h) * kHeadDim + c;
-                    if (a.out_dtype == HMA_OUT_F32) reinterpret_cast<float *>(a.out)[oi] = res;
-                    else reinterpret_cast<uint16_t *>(a.out)[oi] = f32_to_bf16_rne(res);
-                } else {
-                    tp[h * kHeadDim + c] = num;
-                    if (c == 0) { tp[8 * kHeadDim + h] = M; tp[8 * kHeadDim + 8 + h] = den; }
+                    for (int k = 0; k < 4; ++k) {
+                        const int h = (k & 1) ? h1 : h0, c = 16 * j + gq + 8 * (k >> 1);
+                        if (h < G) {
+                            const float res = o[j][k] * ((k & 1) ? i1 : i0);
+                            if (a.out_dtype == HMA_OUT_F32) reinterpret_cast<float *>(a.out)[ob + h * kHeadDim + c] = res;
+                            else reinterpret_cast<uint16_t *>(a.out)[ob + h * kHeadDim + c] = f32_to_bf16_rne(res);
+                        }
+                    }
+            } else {
+                float *tp = a.tiles + ((int64_t)blockIdx.x + ((int64_t)b * Hkv + g)) * kTileFloats;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) tp[((k & 1) ? h1 : h0) * kHeadDim + 16 * j + gq + 8 * (k >> 1)] = o[j][k];
+                if (gq == 0) {
+                    tp[8 * kHeadDim + h0] = m0; tp[8 * kHeadDim + h1] = m1;
+                    tp[8 * kHeadDim + 8 + h0] = l0; tp[8 * kHeadDim + 8 + h1] = l1;
                 }
             }
         }
-        consumer_bar_sync();
 
         w = hi;
         if (++g == Hkv) {
             g = 0;
             do { ++b; } while (b < B && cum[b + 1] == cum[b]);
         }
-        if (!alive) break;
     }
 }
 
@@ -576,7 +654,7 @@ __global__ void __launch_bounds__(128) attn_reduce_kernel(const AttnArgs a, int 
 
 static size_t attn_smem_bytes(int batch)
 {
-    return (size_t)kStages * kBfp8Record + (size_t)kConsumerWarps * 8 * kCombStride * 4 + 2 * kStages * 8 + kStages * 4 +
+    return (size_t)kStages * kBfp8Record + (size_t)kSlots * kSlotFloats * 4 + 2 * kStages * 8 + kStages * 4 +
            (16 + kThreads) * 4 + ((size_t)batch + 1) * 4;
 }
 
@@ -590,18 +668,19 @@ extern "C" size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *d
     return hma::cum_bytes(batch) + ((size_t)hma::kMaxCtas + (size_t)batch * desc->num_kv_heads) * hma::kTileFloats * 4;
 }
 
-extern "C" hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer, const void *q, void *out,
-                                             int32_t out_dtype, const int32_t *block_table, int32_t max_pages_per_seq,
-                                             const int32_t *context_lens, int32_t batch, float sm_scale, void *workspace,
-                                             size_t workspace_bytes, void *stream)
+static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, const void *q, void *out, int32_t out_dtype,
+                                     const int32_t *block_table, int32_t max_pages_per_seq, const int32_t *context_lens,
+                                     int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes, void *stream,
+                                     int probe)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || batch < 0 || max_pages_per_seq < 0) return HMA_ERR_INVALID_ARG;
     if (out_dtype != HMA_OUT_BF16 && out_dtype != HMA_OUT_F32) return HMA_ERR_INVALID_ARG;
     if (batch == 0) return HMA_OK;
-    if (!q || !out || !block_table || !context_lens || !workspace) return HMA_ERR_INVALID_ARG;
+    if (!block_table || !context_lens || !workspace || (!probe && (!q || !out))) return HMA_ERR_INVALID_ARG;
     if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)workspace & 255u)) return HMA_ERR_ALIGNMENT;
     if (batch > hma::kMaxBatch || max_pages_per_seq > (1 << 26)) return HMA_ERR_UNSUPPORTED_SHAPE;
     if (workspace_bytes < hma_decode_attention_workspace_bytes(&cache->desc, batch)) return HMA_ERR_WORKSPACE_TOO_SMALL;
+    if (cache->desc.format != HMA_KV_BFP8 && probe) return HMA_ERR_UNSUPPORTED_SHAPE;
     if (cache->desc.format != HMA_KV_BFP8) {
         // BF16 caches are served by the plain kernel until the tensor-core BF16 variant lands
         return hma_decode_attention_simple(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens,
@@ -633,13 +712,42 @@ extern "C" hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t l
     a.sm_scale = sm_scale;
     a.cum = (int32_t *)workspace;
     a.tiles = (float *)((uint8_t *)workspace + hma::cum_bytes(batch));
+    a.probe = probe;
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
     hma::attn_bfp8_kernel<<<n_ctas, hma::kThreads, smem, s>>>(a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
+    if (probe) return HMA_OK;
     hma::attn_reduce_kernel<<<batch * cache->desc.num_kv_heads, 128, 0, s>>>(a, n_ctas);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;
+}
+
+extern "C" hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer, const void *q, void *out,
+                                             int32_t out_dtype, const int32_t *block_table, int32_t max_pages_per_seq,
+                                             const int32_t *context_lens, int32_t batch, float sm_scale, void *workspace,
+                                             size_t workspace_bytes, void *stream)
+{
+    return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
+                            workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" hma_status_t hma_kv_read_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
+                                          int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
+                                          void *workspace, size_t workspace_bytes, void *stream)
+{
+    return launch_attention(cache, layer, nullptr, nullptr, HMA_OUT_BF16, block_table, max_pages_per_seq, context_lens, batch,
+                            1.0f, workspace, workspace_bytes, stream, 1);
+}
+
+// Diagnostic twin of the probe: the consumer warps run the full arithmetic of every record on whatever
+// the ring holds; nothing is loaded and nothing is written.  Its time is the kernel's instruction-issue floor.
+extern "C" hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
+                                                int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
+                                                void *workspace, size_t workspace_bytes, void *stream)
+{
+    return launch_attention(cache, layer, nullptr, nullptr, HMA_OUT_BF16, block_table, max_pages_per_seq, context_lens, batch,
+                            1.0f, workspace, workspace_bytes, stream, 2);
 }

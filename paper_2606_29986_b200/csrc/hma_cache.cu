@@ -8,6 +8,8 @@
 namespace hma {
 static std::atomic<long long> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+static thread_local cudaError_t g_last_error = cudaSuccess;
+void note_cuda_error(cudaError_t e) { g_last_error = e; }
 }  // namespace hma
 
 static bool desc_ok(const hma_cache_desc_t *d)
@@ -85,5 +87,7 @@ extern "C" const char *hma_status_string(int32_t status)
         default: return "unknown status";
     }
 }
+
+extern "C" const char *hma_last_cuda_error(void) { return cudaGetErrorString(hma::g_last_error); }
 
 extern "C" int64_t hma_launch_count(void) { return (int64_t)hma::g_launches.load(std::memory_order_relaxed); }

@@ -89,9 +89,13 @@ struct hma_cache {
     int device;
 };
 
+namespace hma { void note_cuda_error(cudaError_t e); }
+
 #define HMA_CUDA_OK(expr)                          \
     do {                                           \
-        if ((expr) != cudaSuccess) {               \
+        cudaError_t hma_e_ = (expr);               \
+        if (hma_e_ != cudaSuccess) {               \
+            hma::note_cuda_error(hma_e_);          \
             (void)cudaGetLastError();              \
             return HMA_ERR_CUDA;                   \
         }                                          \

@@ -30,7 +30,10 @@ class CacheDesc(ctypes.Structure):
 class HmaError(RuntimeError):
     def __init__(self, status, where):
         self.status = status
-        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+        detail = ""
+        if status == HMA_ERR_CUDA:
+            detail = ": " + hma_last_cuda_error()
+        super().__init__("%s: %s (status %d)%s" % (where, status_string(status), status, detail))
 
 
 _lib = None
@@ -56,6 +59,10 @@ def lib():
         L.hma_decode_attention_workspace_bytes.argtypes = [ctypes.POINTER(CacheDesc), i32]
         L.hma_decode_attention.restype = i32
         L.hma_decode_attention.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp, sz, vp]
+        L.hma_kv_read_probe.restype = i32
+        L.hma_kv_read_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
+        L.hma_attention_alu_probe.restype = i32
+        L.hma_attention_alu_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
         L.hma_decode_attention_simple.restype = i32
         L.hma_decode_attention_simple.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
         L.hma_bfp8_dequant_bf16.restype = i32
@@ -66,6 +73,8 @@ def lib():
         L.hma_error_flags.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
         L.hma_status_string.restype = ctypes.c_char_p
         L.hma_status_string.argtypes = [i32]
+        L.hma_last_cuda_error.restype = ctypes.c_char_p
+        L.hma_last_cuda_error.argtypes = []
         L.hma_launch_count.restype = i64
         L.hma_launch_count.argtypes = []
         _lib = L
@@ -149,6 +158,18 @@ def hma_decode_attention(cache, layer, q, out, block_table, context_lens, sm_sca
            "hma_decode_attention")
 
 
+def hma_kv_read_probe(cache, layer, block_table, context_lens, workspace, stream=None):
+    _check(lib().hma_kv_read_probe(cache.handle, layer, _ptr(block_table), block_table.shape[1], _ptr(context_lens),
+                                   context_lens.shape[0], _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                   _stream(stream)), "hma_kv_read_probe")
+
+
+def hma_attention_alu_probe(cache, layer, block_table, context_lens, workspace, stream=None):
+    _check(lib().hma_attention_alu_probe(cache.handle, layer, _ptr(block_table), block_table.shape[1], _ptr(context_lens),
+                                         context_lens.shape[0], _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                         _stream(stream)), "hma_attention_alu_probe")
+
+
 def hma_decode_attention_simple(cache, layer, q, out, block_table, context_lens, sm_scale, stream=None):
     out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
     _check(lib().hma_decode_attention_simple(cache.handle, layer, _ptr(q), _ptr(out), out_dtype, _ptr(block_table),
@@ -170,6 +191,10 @@ def hma_error_flags(cache, stream=None):
     v = ctypes.c_uint32(0)
     _check(lib().hma_error_flags(cache.handle, ctypes.byref(v), _stream(stream)), "hma_error_flags")
     return int(v.value)
+
+
+def hma_last_cuda_error():
+    return lib().hma_last_cuda_error().decode()
 
 
 def hma_launch_count():
