@@ -50,7 +50,6 @@ struct AttnArgs {
     float sm_scale;
     int32_t *cum;        // workspace: pages before each sequence, batch+1 entries
     float *tiles;        // workspace: partial tiles
-    int probe;           // 1: stream the records through the ring and do no arithmetic (bandwidth probe)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -183,6 +182,9 @@ __device__ __forceinline__ int pages_of(const AttnArgs &a, int b)
 // ---------------------------------------------------------------- main kernel
 extern __shared__ __align__(128) uint8_t smem_raw[];
 
+// kMode 0: attention.  1: stream the records through the ring, no arithmetic (bandwidth probe).
+// 2: the arithmetic of every record on whatever the ring holds, nothing loaded or written (issue-rate probe).
+template <int kMode>
 __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a)
 {
     // shared memory carve-up
@@ -263,7 +265,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         int chunk = min(min(32, np - p), R - r);
         int32_t pid = lane < chunk ? a.block_table[(int64_t)b * a.max_pages + p + lane] : 0;
         bool alive = true;
-        if (a.probe >= 2) return;            // arithmetic-only diagnostic: nothing is loaded
+        if (kMode == 2) return;              // arithmetic-only diagnostic: nothing is loaded
         while (r < R) {
             const int c_chunk = chunk, c_g = g, c_r = r;
             const int32_t c_pid = pid;
@@ -340,7 +342,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         {
             float f[8][4];
             float amax = 0.f;
-            const bool hv = gq < G && !a.probe;      // the probes have no Q: nothing is read through a.q
+            const bool hv = gq < G && kMode == 0;      // the probes have no Q: nothing is read through a.q
             const uint16_t *qp = a.q + ((int64_t)b * a.cv.num_q_heads + (int64_t)g * G + (hv ? gq : 0)) * kHeadDim + 4 * t4;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -379,22 +381,22 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         int r = rbase + warp;
         int stage = r % kStages;
         uint32_t par = (uint32_t)(r / kStages) & 1u;
-        for (; r < rend; r += kConsumerWarps) {
-            if (a.probe < 2) {
+        int page = page0 + warp;
+        for (; r < rend; r += kConsumerWarps, page += kConsumerWarps) {
+            if (kMode < 2) {
                 alive = mbar_wait(full0 + 8 * stage, par, abort_word, a.cv.flags);
                 if (!alive) break;
             }
             const uint32_t sp = smem_u32(ring) + stage * kBfp8Record;
             const uint32_t my_empty = empty0 + 8 * stage;
-            const bool ok = a.probe >= 2 || stage_ok[stage] != 0;
+            const bool ok = kMode == 2 || stage_ok[stage] != 0;
             stage += kConsumerWarps;
             if (stage >= kStages) { stage -= kStages; par ^= 1u; }
-            if (a.probe == 1 || !ok) {
+            if (kMode == 1 || !ok) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(my_empty);
                 continue;
             }
-            const int page = page0 + (r - rbase);
             const int nvalid = page == np - 1 ? tail : kPageTokens;
 
             // ---- exponents: fp32 scales for Q.K^T, reference-exponent check and FP16 scales for P.V ----
@@ -467,6 +469,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                     sc[3] = fmaf(d[3], ks[8 + j], sc[3]);
                 }
             }
+            // the V element words go to registers now, so that the ring slot can be refilled during softmax and P.V
+            uint4 vm[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) vm[c] = lds128(sp + kBfp8Half + 128 + c * 512 + lane * 16);
+            __syncwarp();
+            if (lane == 0 && kMode < 2) mbar_arrive(my_empty);
             float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
             if (nvalid < kPageTokens) {
                 if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
@@ -501,9 +509,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                 uint4 vs[4];           // (f01, f89) of blocks 2c, 2c+1
 #pragma unroll
                 for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + t4 * 64 + c * 16);
-                uint4 vm[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) vm[c] = lds128(sp + kBfp8Half + 128 + c * 512 + lane * 16);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const uint4 &vv = vm[j >> 1];
@@ -517,13 +522,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                     mma_f16_acc(o[j], af, hmul2_u32(pb0, f01), hmul2_u32(pb1, f89));
                 }
             }
-            __syncwarp();      // every lane is done with the ring slot and with the scratch tables
-            if (lane == 0 && a.probe < 2) mbar_arrive(my_empty);
+            __syncwarp();      // every lane is done with the scratch tables
         }
 
         // ---- merge the warps' states of this segment: pairwise tree, at most kSlots states in shared memory ----
         consumer_bar_sync();                           // the scratch tables (same memory as the slots) are idle now
-        if (!a.probe && alive) {
+        if (kMode != 1 && alive) {
             // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -538,7 +542,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
 #pragma unroll 1
             for (int base = 0; base < n - half; base += kSlots) {
                 const int wr = warp - half - base;     // slot this warp writes in this round, if in [0, kSlots)
-                if (!a.probe && warp >= half && warp < n && wr >= 0 && wr < kSlots) {
+                if (kMode != 1 && warp >= half && warp < n && wr >= 0 && wr < kSlots) {
                     float *slot = comb + wr * kSlotFloats;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
@@ -551,7 +555,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                 }
                 consumer_bar_sync();
                 const int rd = warp - base;            // slot this warp reads in this round, if in [0, kSlots)
-                if (!a.probe && warp < n - half && rd >= 0 && rd < kSlots) {
+                if (kMode != 1 && warp < n - half && rd >= 0 && rd < kSlots) {
                     const float *slot = comb + rd * kSlotFloats;
                     const float pm0 = slot[1024 + t4 * 4 + 0], pm1 = slot[1024 + t4 * 4 + 1];
                     const float pl0 = slot[1024 + t4 * 4 + 2], pl1 = slot[1024 + t4 * 4 + 3];
@@ -573,7 +577,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
                 consumer_bar_sync();
             }
         }
-        if (warp == 0 && !a.probe && alive) {
+        if (warp == 0 && (kMode == 0 || (kMode == 2 && a.batch < 0)) && alive) {   // the issue-rate probe never stores, but keeps its arithmetic live
             const bool whole = lo == seg0 && hi == seg1;
             const int h0 = 2 * t4, h1 = 2 * t4 + 1;
             if (whole) {
@@ -694,8 +698,10 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
         HMA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     }
     const size_t smem = hma::attn_smem_bytes(batch);
-    if (!attr_set || true) {
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_bfp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    if (!attr_set) {
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_bfp8_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_bfp8_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_bfp8_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     if (smem > 227 * 1024) return HMA_ERR_UNSUPPORTED_SHAPE;
@@ -712,10 +718,11 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.sm_scale = sm_scale;
     a.cum = (int32_t *)workspace;
     a.tiles = (float *)((uint8_t *)workspace + hma::cum_bytes(batch));
-    a.probe = probe;
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
-    hma::attn_bfp8_kernel<<<n_ctas, hma::kThreads, smem, s>>>(a);
+    if (probe == 0) hma::attn_bfp8_kernel<0><<<n_ctas, hma::kThreads, smem, s>>>(a);
+    else if (probe == 1) hma::attn_bfp8_kernel<1><<<n_ctas, hma::kThreads, smem, s>>>(a);
+    else hma::attn_bfp8_kernel<2><<<n_ctas, hma::kThreads, smem, s>>>(a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     if (probe) return HMA_OK;
