@@ -2,13 +2,16 @@
 // rebuilt inside the attention kernel).
 //
 // Shape of the kernel
-//   * persistent grid, one CTA per SM.  All (sequence, kv head, page) records of the batch form one
-//     linear work list that is cut into equal contiguous ranges, one per CTA (no tail effect, any
-//     mix of context lengths).  A CTA that holds only part of a (sequence, kv head) segment emits a
-//     partial (max, sum, 128-vector) per q head; a second small kernel merges partials in fixed order.
-//   * one producer warp streams 4352-byte page records HBM -> shared memory with 1-D bulk async
-//     copies (cp.async.bulk + mbarrier transaction counts) through a deep ring; eight consumer warps
-//     each own whole records.
+//   * persistent grid, one CTA of 16 warps per SM (four warps per SM sub-partition, 128 registers each).
+//     All (sequence, kv head, page) records of the batch form one linear work list that is cut into
+//     equal contiguous ranges, one per *warp* (no tail effect, any mix of context lengths, no barrier
+//     between warps).  A warp that holds only part of a (sequence, kv head) segment writes a partial
+//     (max, sum, 128-vector) per q head; a small second kernel, launched with programmatic dependent
+//     launch so that its launch latency hides behind the main kernel, merges the partials in worker
+//     order (fixed order, so results are bitwise repeatable).
+//   * every warp feeds itself: it keeps three 4352-byte page records in flight with 1-D bulk async
+//     copies (cp.async.bulk + mbarrier transaction counts) and re-arms a ring slot as soon as its
+//     Q.K^T phase has pulled the record's words into registers.
 //   * unpack is two integer instructions per pair of elements (byte permute + mask): the element
 //     byte s<<7|m becomes the FP16 bit pattern s<<15|m, which *is* the number +-m * 2^-24 (an FP16
 //     subnormal), so mantissas enter mma.sync.m16n8k16 exactly.  The shared block exponent never
@@ -22,21 +25,16 @@
 
 namespace hma {
 
-// 15 consumer warps + 1 producer warp = 16 warps, four per SM sub-partition: each sub-partition has 16384
-// registers, so a 17th warp would cap every thread at 96 registers instead of 128.
-constexpr int kConsumerWarps = 15;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kStages = 45;                       // ring depth
-// A ring slot must be used by the same consumer warp every time round (within a segment): a warp that ran two
-// laps ahead of the slot's previous owner would see the slot's older completed phase and read stale bytes.
-static_assert(kStages % kConsumerWarps == 0, "ring depth must be a multiple of one round of the consumer warps");
+constexpr int kWarps = 16;
+constexpr int kThreads = kWarps * 32;
+constexpr int kDepth = 3;                         // ring slots per warp
+constexpr int kStages = kWarps * kDepth;
+constexpr int kScratch = 768;                     // per warp: 512 B of fp32 K scales + 256 B of FP16 V scales
 constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile: o[8][128], m[8], l[8]
-constexpr int kSlots = 4;                         // states held in shared memory during the merge
-constexpr int kSlotFloats = 1024 + 16;            // one warp's state: 32 accumulators per lane, then m, l per head pair
-static_assert(kSlots * kSlotFloats * 4 >= kConsumerWarps * 768, "per-warp scratch tables live inside the merge slots");
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int kMaxBatch = 768;
-constexpr int kMaxCtas = 1024;
+constexpr int kMaxBatch = 2048;
+constexpr int kMaxCtas = 256;
+constexpr int kMinRecords = 8;                    // fewest records a worker takes
 
 struct AttnArgs {
     CacheView cv;
@@ -48,8 +46,8 @@ struct AttnArgs {
     const int32_t *ctx;
     int batch;
     float sm_scale;
-    int32_t *cum;        // workspace: pages before each sequence, batch+1 entries
-    float *tiles;        // workspace: partial tiles
+    int32_t *cum;                   // workspace: pages before each sequence, batch + 1 entries (for the merge kernel)
+    float *tiles;                   // workspace: partial tiles
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -150,7 +148,6 @@ __device__ __forceinline__ float ex2f(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
 {
     __half2 h = __floats2half2_rn(lo, hi);
@@ -179,32 +176,33 @@ __device__ __forceinline__ int pages_of(const AttnArgs &a, int b)
     return (T + kPageTokens - 1) / kPageTokens;
 }
 
-// ---------------------------------------------------------------- main kernel
-extern __shared__ __align__(128) uint8_t smem_raw[];
+__device__ __forceinline__ void store_out(const AttnArgs &a, int64_t idx, float v)
+{
+    if (a.out_dtype == HMA_OUT_F32) reinterpret_cast<float *>(a.out)[idx] = v;
+    else reinterpret_cast<uint16_t *>(a.out)[idx] = f32_to_bf16_rne(v);
+}
 
+// ---------------------------------------------------------------- the kernel
 // kMode 0: attention.  1: stream the records through the ring, no arithmetic (bandwidth probe).
 // 2: the arithmetic of every record on whatever the ring holds, nothing loaded or written (issue-rate probe).
+extern __shared__ __align__(128) uint8_t smem_raw[];
+
 template <int kMode>
 __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a)
 {
-    // shared memory carve-up
-    uint8_t *ring = smem_raw;                                                   // kStages x 4352
-    float *comb = reinterpret_cast<float *>(ring + kStages * kBfp8Record);       // merge slots / per-warp scratch
-    uint64_t *bars = reinterpret_cast<uint64_t *>(comb + kSlots * kSlotFloats);   // full[kStages], empty[kStages]
-    int *stage_ok = reinterpret_cast<int *>(bars + 2 * kStages);                 // [kStages]
-    int *misc = stage_ok + kStages;                                              // [0] abort word, [1..] scan scratch
-    int *cum = misc + 16 + kThreads;                                             // [batch + 1]
+    uint8_t *ring = smem_raw;                                                     // kStages x 4352
+    uint8_t *scratch = ring + kStages * kBfp8Record;                              // kWarps x kScratch
+    uint64_t *bars = reinterpret_cast<uint64_t *>(scratch + kWarps * kScratch);   // full[kStages]
+    int *stage_ok = reinterpret_cast<int *>(bars + kStages);                      // [kStages]
+    int *misc = stage_ok + kStages;                                               // [0] abort word, [16..] scan scratch
+    int *cum = misc + 16 + kThreads;                                              // [batch + 1]
     volatile int *abort_word = misc;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int Hkv = a.cv.num_kv_heads, G = a.cv.num_q_heads / Hkv, B = a.batch;
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages);
+    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv, B = a.batch;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, 1);
-        }
+        for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(bars + s), 1);
         misc[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -227,439 +225,418 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         for (int b = b0; b < b1; ++b) { cum[b] = run; run += pages_of(a, b); }
         __syncthreads();
     }
-    if (blockIdx.x == 0)
+    // let the merge kernel be scheduled already; it blocks in griddepcontrol.wait until this grid has finished
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (blockIdx.x == 0 && kMode == 0)
         for (int b = tid; b <= B; b += kThreads) a.cum[b] = cum[b];
-
+    // from here on the warps never synchronise with one another
     const int64_t W = (int64_t)Hkv * cum[B];
-    const int64_t N = gridDim.x;
-    const int64_t w0 = (int64_t)blockIdx.x * W / N, w1 = (int64_t)(blockIdx.x + 1) * W / N;
-    if (w0 >= w1) return;
+    // Workers are numbered across SMs first.  Small batches use fewer workers, at least kMinRecords records
+    // each, so that a segment is never cut into more partials than it is worth.
+    const int64_t NWK = max((int64_t)1, min((int64_t)gridDim.x * kWarps, W / kMinRecords));
+    const int64_t u = (int64_t)warp * gridDim.x + blockIdx.x;      // this warp's worker index
 
-    // locate the segment (b, g) that holds w0
-    int b_cur, g_cur;
+    if (kMode == 0)                                               // empty sequences get rows of zeros
+        for (int64_t b = u; b < B; b += NWK)
+            if (cum[b + 1] == cum[b])
+                for (int i = lane; i < Hq * kHeadDim; i += 32) store_out(a, b * Hq * kHeadDim + i, 0.f);
+
+    if (u >= NWK) return;
+    const int64_t wlo = u * W / NWK, whi = (u + 1) * W / NWK;
+    if (wlo >= whi) return;
+    const int Rw = (int)(whi - wlo);
+
+    // the segment (b, g) and page that hold record wlo
+    int b, g, page, np;
     {
         int lo = 0, hi = B - 1;
-        while (lo < hi) {   // largest b with Hkv*cum[b] <= w0
+        while (lo < hi) {   // largest b with Hkv*cum[b] <= wlo
             int mid = (lo + hi + 1) >> 1;
-            if ((int64_t)Hkv * cum[mid] <= w0) lo = mid; else hi = mid - 1;
+            if ((int64_t)Hkv * cum[mid] <= wlo) lo = mid; else hi = mid - 1;
         }
-        while (cum[lo + 1] == cum[lo]) ++lo;   // cannot run off: w0 < W
-        b_cur = lo;
-        const int np = cum[lo + 1] - cum[lo];
-        g_cur = (int)((w0 - (int64_t)Hkv * cum[lo]) / np);
+        while (cum[lo + 1] == cum[lo]) ++lo;   // cannot run off: wlo < W
+        b = lo;
+        np = cum[lo + 1] - cum[lo];
+        const int64_t off = wlo - (int64_t)Hkv * cum[lo];
+        g = (int)(off / np);
+        page = (int)(off - (int64_t)g * np);
     }
 
-    if (warp == kConsumerWarps) {
-        // ------------------------------------------------------------ producer warp
-        // Every lane owns one record of a chunk of up to 32 consecutive pages of a segment: it waits for
-        // its ring slot, then issues its own bulk copy, so 32 copies are set up in parallel.  The block
-        // table entries of the next chunk are fetched before the current chunk waits.
-        uint64_t policy;
-        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-        constexpr int rb = kBfp8Record;
-        int b = b_cur, g = g_cur;
-        int np = cum[b + 1] - cum[b];
-        int p = (int)(w0 - ((int64_t)Hkv * cum[b] + (int64_t)g * np));
-        const int R = (int)(w1 - w0);
-        int r = 0;
-        int chunk = min(min(32, np - p), R - r);
-        int32_t pid = lane < chunk ? a.block_table[(int64_t)b * a.max_pages + p + lane] : 0;
-        bool alive = true;
-        if (kMode == 2) return;              // arithmetic-only diagnostic: nothing is loaded
-        while (r < R) {
-            const int c_chunk = chunk, c_g = g, c_r = r;
-            const int32_t c_pid = pid;
-            // advance to the next chunk and prefetch its page ids
-            r += chunk;
-            p += chunk;
-            if (p == np) {
-                p = 0;
+    // ---- the warp's own feed: issue cursor, window of block-table entries, three ring slots ----
+    const uint32_t full0 = smem_u32(bars + warp * kDepth);
+    const uint32_t ring0 = smem_u32(ring + warp * kDepth * kBfp8Record);
+    int ib = b, ig = g, ip = page, inp = np;      // cursor of the next record to request
+    int iwb = -1, iw0 = 0;                        // the window holds pages [iw0, iw0+32) of sequence iwb
+    int32_t ipid = -1;
+    int islot = 0;
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    auto issue = [&]() {
+        if (kMode == 2) return;
+        if (iwb != ib || ip < iw0 || ip >= iw0 + 32) {
+            iwb = ib;
+            iw0 = ip;
+            ipid = ip + lane < inp ? a.block_table[(int64_t)ib * a.max_pages + ip + lane] : -1;
+        }
+        const int32_t pid = __shfl_sync(0xFFFFFFFFu, ipid, ip - iw0);
+        if (lane == 0) {
+            const int s = warp * kDepth + islot;
+            if (pid >= 0 && pid < a.cv.num_pages) {
+                stage_ok[s] = 1;
+                mbar_arrive_expect_tx(full0 + 8 * islot, kBfp8Record);
+                bulk_load(ring0 + islot * kBfp8Record, a.cv.layer + ((int64_t)pid * Hkv + ig) * kBfp8Record, kBfp8Record,
+                          full0 + 8 * islot, policy);
+            } else {
+                stage_ok[s] = 0;
+                atomicOr(a.cv.flags, HMA_FLAG_BAD_PAGE_ATTENTION);
+                mbar_arrive(full0 + 8 * islot);
+            }
+        }
+        if (++islot == kDepth) islot = 0;
+        if (++ip == inp) {
+            ip = 0;
+            if (++ig == Hkv) {
+                ig = 0;
+                do { ++ib; } while (ib < B && cum[ib + 1] == cum[ib]);
+                if (ib < B) inp = cum[ib + 1] - cum[ib];
+            }
+        }
+    };
+    for (int k = 0; k < kDepth && k < Rw; ++k) issue();
+
+    // ---- consumer state ----
+    const int gq = lane >> 2, t4 = lane & 3;
+    const float kLog2e = 1.4426950408889634f;
+    const uint32_t scrK = smem_u32(scratch + warp * kScratch);   // fp32 2^(E-127) of every (token, block) of K
+    const uint32_t scrV = scrK + 512;                            // FP16 scales of every (token pair, block) of V
+    uint32_t qf[8][2];
+    float cs0 = 0.f, cs1 = 0.f;                    // score multipliers of heads 2*t4, 2*t4+1
+    float m0 = -INFINITY, m1 = -INFINITY;          // running maxima (log2 domain) of heads 2*t4, 2*t4+1
+    float lacc[4] = {0.f, 0.f, 0.f, 0.f};          // running sums, via an all-ones MMA
+    float o[8][4];
+    int Rmine = 0;                                 // reference exponent of V channel block (lane & 7)
+    int T = 0, tail = kPageTokens;
+    bool whole = false;                            // this warp holds every record of the current segment
+
+    auto begin_segment = [&](int k) {
+        np = cum[b + 1] - cum[b];
+        T = min(a.ctx[b], a.max_pages * kPageTokens);
+        tail = T - (np - 1) * kPageTokens;
+        whole = page == 0 && Rw - k >= np;
+        // Q fragments of this (sequence, kv head): FP16, one power-of-two scale per head
+        float f[8][4];
+        float amax = 0.f;
+        const bool hv = gq < G && kMode == 0;      // the probes have no Q: nothing is read through a.q
+        const uint16_t *qp = a.q + ((int64_t)b * Hq + (int64_t)g * G + (hv ? gq : 0)) * kHeadDim + 4 * t4;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint2 v = hv ? *reinterpret_cast<const uint2 *>(qp + 16 * j) : make_uint2(0u, 0u);
+            f[j][0] = __uint_as_float(v.x << 16);
+            f[j][1] = __uint_as_float(v.x & 0xFFFF0000u);
+            f[j][2] = __uint_as_float(v.y << 16);
+            f[j][3] = __uint_as_float(v.y & 0xFFFF0000u);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) amax = fmaxf(amax, fabsf(f[j][c]));
+        }
+        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+        int shift = 0;
+        if (amax > 0.f && amax < INFINITY) shift = 14 - ((int)((__float_as_uint(amax) >> 23) & 0xFF) - 127);
+        shift = max(-120, min(120, shift));
+        const float up = pow2_field(127 + shift), down = pow2_field(127 - shift);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            qf[j][0] = pack_half2(f[j][0] * up, f[j][1] * up);
+            qf[j][1] = pack_half2(f[j][2] * up, f[j][3] * up);
+        }
+        // mantissas enter as m * 2^-24 and exponents as 2^(E-127) while values are m * 2^(E-133): 2^18 is owed
+        const float cs = a.sm_scale * kLog2e * down * 262144.f;
+        cs0 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4) * 4);
+        cs1 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4 + 1) * 4);
+        m0 = -INFINITY;
+        m1 = -INFINITY;
+        lacc[0] = lacc[1] = lacc[2] = lacc[3] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+        Rmine = 0;
+    };
+
+    auto finish_segment = [&]() {
+        if (kMode == 1) return;
+        // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float vsc = pow2_field(min(__shfl_sync(0xFFFFFFFFu, Rmine, j) + 3, 254));
+            o[j][0] *= vsc; o[j][1] *= vsc; o[j][2] *= vsc; o[j][3] *= vsc;
+        }
+        const float l0 = lacc[0], l1 = lacc[1];
+        const int h0 = 2 * t4, h1 = 2 * t4 + 1;
+        const int64_t ob = ((int64_t)b * Hq + (int64_t)g * G) * kHeadDim;
+        if (kMode == 2 && a.batch >= 0) return;    // the issue-rate probe never stores, but keeps its arithmetic live
+        if (whole) {
+            const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int h = (c & 1) ? h1 : h0;
+                    if (h < G) store_out(a, ob + h * kHeadDim + 16 * j + gq + 8 * (c >> 1), o[j][c] * ((c & 1) ? i1 : i0));
+                }
+            return;
+        }
+        const int64_t seg = (int64_t)b * Hkv + g;
+        float *tp = a.tiles + (u + seg) * kTileFloats;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tp[((c & 1) ? h1 : h0) * kHeadDim + 16 * j + gq + 8 * (c >> 1)] = o[j][c];
+        if (gq == 0) {
+            tp[8 * kHeadDim + h0] = m0; tp[8 * kHeadDim + h1] = m1;
+            tp[8 * kHeadDim + 8 + h0] = l0; tp[8 * kHeadDim + 8 + h1] = l1;
+        }
+    };
+
+    // ---- the records of this warp ----
+    int slot = 0;
+    uint32_t par = 0;
+    int left = 0;                                  // records of the current segment still to do
+    bool alive = true;
+    for (int k = 0; k < Rw; ++k) {
+        if (left == 0) {
+            if (k > 0) {
+                finish_segment();
+                page = 0;
                 if (++g == Hkv) {
                     g = 0;
                     do { ++b; } while (b < B && cum[b + 1] == cum[b]);
-                    if (b < B) np = cum[b + 1] - cum[b];
                 }
             }
-            if (r < R) {
-                chunk = min(min(32, np - p), R - r);
-                pid = lane < chunk ? a.block_table[(int64_t)b * a.max_pages + p + lane] : 0;
-            }
-            if (lane < c_chunk) {
-                const int rr = c_r + lane;
-                const int s = rr % kStages;
-                if (rr >= kStages) alive = mbar_wait(empty0 + 8 * s, (uint32_t)((rr / kStages) - 1) & 1u, abort_word, a.cv.flags);
-                if (alive) {
-                    if (c_pid >= 0 && c_pid < a.cv.num_pages) {
-                        stage_ok[s] = 1;
-                        mbar_arrive_expect_tx(full0 + 8 * s, rb);
-                        bulk_load(smem_u32(ring + s * rb), a.cv.layer + ((int64_t)c_pid * Hkv + c_g) * rb, rb, full0 + 8 * s, policy);
-                    } else {
-                        stage_ok[s] = 0;
-                        atomicOr(a.cv.flags, HMA_FLAG_BAD_PAGE_ATTENTION);
-                        mbar_arrive(full0 + 8 * s);
-                    }
-                }
-            }
-            if (!__all_sync(0xFFFFFFFFu, alive)) {
-                // a wait ran out: give the copies already issued a bounded chance to land, then leave
-                const int issued = c_r;   // records below c_r were all issued
-                for (int s = lane; s < kStages; s += 32) {
-                    int last = -1;
-                    for (int q = s; q < issued; q += kStages) last = q;
-                    if (last < 0) continue;
-                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(full0 + 8 * s, (uint32_t)(last / kStages) & 1u); ++it) {}
-                }
-                return;
-            }
+            begin_segment(k);
+            left = min(np - page, Rw - k);
         }
-        return;
-    }
+        --left;
+        const uint32_t sp = ring0 + slot * kBfp8Record;
+        const int s_idx = warp * kDepth + slot;
+        if (kMode < 2) {
+            alive = mbar_wait(full0 + 8 * slot, par, abort_word, a.cv.flags);
+            if (!alive) break;
+        }
+        if (++slot == kDepth) { slot = 0; par ^= 1u; }
+        const bool ok = kMode == 2 || stage_ok[s_idx] != 0;
+        const int nvalid = page == np - 1 ? tail : kPageTokens;
+        ++page;
+        if (kMode == 1 || !ok) {
+            __syncwarp();
+            if (k + kDepth < Rw) issue();
+            continue;
+        }
 
-    // ---------------------------------------------------------------- consumer warps
-    // One record (16 tokens of one kv head) per warp iteration; a ring slot belongs to the same warp on every lap.
-    const int gq = lane >> 2, t4 = lane & 3;
-    const float kLog2e = 1.4426950408889634f;
-    // per-warp scratch inside the merge area (idle until the segment ends):
-    // fp32 Q.K^T scales 2^(E-127) of every (token, block) and FP16 P.V scales of every (token pair, block)
-    const uint32_t scrK = smem_u32(comb) + warp * 768;     // 512 B
-    const uint32_t scrV = scrK + 512;                      // 256 B
-    int64_t w = w0;
-    int b = b_cur, g = g_cur;
-    bool alive = true;
-    while (w < w1 && alive) {
-        const int np = cum[b + 1] - cum[b];
-        const int64_t seg0 = (int64_t)Hkv * cum[b] + (int64_t)g * np, seg1 = seg0 + np;
-        const int64_t lo = max(seg0, w0), hi = min(seg1, w1);
-        const int T = min(a.ctx[b], a.max_pages * kPageTokens);
-        const int rbase = (int)(lo - w0);            // CTA-local index of the segment's first record here
-        const int rend = (int)(hi - w0);
-        const int page0 = (int)(lo - seg0);          // page of the sequence that record rbase holds
-        const int tail = T - (np - 1) * kPageTokens; // valid tokens of the sequence's last page, 1..16
-
-        // ---- Q fragments of this (sequence, kv head): FP16, one power-of-two scale per head ----
-        uint32_t qf[8][2];
-        float cs0, cs1;   // score multipliers of heads 2*t4, 2*t4+1
+        // ---- exponents: fp32 scales for Q.K^T, reference-exponent check and FP16 scales for P.V ----
         {
-            float f[8][4];
-            float amax = 0.f;
-            const bool hv = gq < G && kMode == 0;      // the probes have no Q: nothing is read through a.q
-            const uint16_t *qp = a.q + ((int64_t)b * a.cv.num_q_heads + (int64_t)g * G + (hv ? gq : 0)) * kHeadDim + 4 * t4;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint2 v = hv ? *reinterpret_cast<const uint2 *>(qp + 16 * j) : make_uint2(0u, 0u);
-                f[j][0] = __uint_as_float(v.x << 16);
-                f[j][1] = __uint_as_float(v.x & 0xFFFF0000u);
-                f[j][2] = __uint_as_float(v.y << 16);
-                f[j][3] = __uint_as_float(v.y & 0xFFFF0000u);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) amax = fmaxf(amax, fabsf(f[j][k]));
-            }
-            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
-            int shift = 0;
-            if (amax > 0.f && amax < INFINITY) shift = 14 - ((int)((__float_as_uint(amax) >> 23) & 0xFF) - 127);
-            shift = max(-120, min(120, shift));
-            const float up = pow2_field(127 + shift), down = pow2_field(127 - shift);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                qf[j][0] = pack_half2(f[j][0] * up, f[j][1] * up);
-                qf[j][1] = pack_half2(f[j][2] * up, f[j][3] * up);
-            }
-            // mantissas enter as m * 2^-24 and exponents as 2^(E-127) while values are m * 2^(E-133): 2^18 is owed
-            const float cs = a.sm_scale * kLog2e * down * 262144.f;
-            cs0 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4) * 4);
-            cs1 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4 + 1) * 4);
-        }
-
-        float m0 = -INFINITY, m1 = -INFINITY;          // running maxima (log2 domain) of heads 2*t4, 2*t4+1
-        float lacc[4] = {0.f, 0.f, 0.f, 0.f};          // running sums, via an all-ones MMA
-        float o[8][4];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
-        int Rmine = 0;                                  // reference exponent of V channel block (lane & 7)
-
-        int r = rbase + warp;
-        int stage = r % kStages;
-        uint32_t par = (uint32_t)(r / kStages) & 1u;
-        int page = page0 + warp;
-        for (; r < rend; r += kConsumerWarps, page += kConsumerWarps) {
-            if (kMode < 2) {
-                alive = mbar_wait(full0 + 8 * stage, par, abort_word, a.cv.flags);
-                if (!alive) break;
-            }
-            const uint32_t sp = smem_u32(ring) + stage * kBfp8Record;
-            const uint32_t my_empty = empty0 + 8 * stage;
-            const bool ok = kMode == 2 || stage_ok[stage] != 0;
-            stage += kConsumerWarps;
-            if (stage >= kStages) { stage -= kStages; par ^= 1u; }
-            if (kMode == 1 || !ok) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(my_empty);
-                continue;
-            }
-            const int nvalid = page == np - 1 ? tail : kPageTokens;
-
-            // ---- exponents: fp32 scales for Q.K^T, reference-exponent check and FP16 scales for P.V ----
-            {
-                const uint32_t kw = lds32(sp + lane * 4);
-                uint32_t vw = lds32(sp + kBfp8Half + lane * 4);
-                if (nvalid < kPageTokens) {
-                    // exponent bytes of masked tokens count as 0: they neither raise the reference exponent
-                    // nor produce non-finite weights
-                    uint32_t keep = 0;
-                    const int tt = lane >> 3;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (2 * tt + (k & 1) + 8 * (k >> 1) < nvalid) keep |= 0xFFu << (8 * k);
-                    vw &= keep;
-                }
-                sts128(scrK + lane * 16, (kw << 23) & 0x7F800000u, (kw << 15) & 0x7F800000u, (kw << 7) & 0x7F800000u,
-                       (kw >> 1) & 0x7F800000u);
-                const uint32_t mx2 = __vmaxu2((vw >> 8) & 0x00FF00FFu, vw & 0x00FF00FFu);
-                int emax = (int)max(mx2 & 0xFFFFu, mx2 >> 16);
-                if (__any_sync(0xFFFFFFFFu, emax > Rmine)) {
-                    // a V block exponent above the reference: raise it and rescale that block's accumulators
-                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
-                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
-                    const int Rnew = max(Rmine, emax);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
-                        const float fr = dlt < -126 ? 0.f : pow2_field(127 + dlt);
-                        o[j][0] *= fr; o[j][1] *= fr; o[j][2] *= fr; o[j][3] *= fr;
-                    }
-                    Rmine = Rnew;
-                }
-                // FP16 scale 2^(E - R + 15) of every (token pair, block): exponent field max(E - R + 30, 0)
-                const uint32_t kmine = ((uint32_t)(30 - Rmine) & 0xFFFFu) * 0x00010001u;
-                sts64(scrV + lane * 8, __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4140u), kmine, 0u) << 10,
-                      __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4342u), kmine, 0u) << 10);
-            }
-            uint4 km[4];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) km[c] = lds128(sp + 128 + c * 512 + lane * 16);
-            __syncwarp();
-
-            // ================= Q.K^T =================
-            float sc[4] = {0.f, 0.f, 0.f, 0.f};
-            {
-                float ks[16];      // 2^(E-127): token gq blocks 0..7, token gq+8 blocks 0..7
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint4 v = lds128(scrK + gq * 64 + c * 16);
-                    ks[4 * c] = __uint_as_float(v.x); ks[4 * c + 1] = __uint_as_float(v.y);
-                    ks[4 * c + 2] = __uint_as_float(v.z); ks[4 * c + 3] = __uint_as_float(v.w);
-                }
-                const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint4 &klo = km[(j >> 2) * 2], &khi = km[(j >> 2) * 2 + 1];
-                    const uint32_t wl = (j & 3) == 0 ? klo.x : (j & 3) == 1 ? klo.y : (j & 3) == 2 ? klo.z : klo.w;
-                    const uint32_t wh = (j & 3) == 0 ? khi.x : (j & 3) == 1 ? khi.y : (j & 3) == 2 ? khi.z : khi.w;
-                    uint32_t af[4];
-                    af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
-                    af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
-                    af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
-                    af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
-                    float d[4];
-                    mma_f16(d, af, qf[j][0], qf[j][1], zero4);
-                    sc[0] = fmaf(d[0], ks[j], sc[0]);
-                    sc[1] = fmaf(d[1], ks[j], sc[1]);
-                    sc[2] = fmaf(d[2], ks[8 + j], sc[2]);
-                    sc[3] = fmaf(d[3], ks[8 + j], sc[3]);
-                }
-            }
-            // the V element words go to registers now, so that the ring slot can be refilled during softmax and P.V
-            uint4 vm[4];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) vm[c] = lds128(sp + kBfp8Half + 128 + c * 512 + lane * 16);
-            __syncwarp();
-            if (lane == 0 && kMode < 2) mbar_arrive(my_empty);
-            float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
+            const uint32_t kw = lds32(sp + lane * 4);
+            uint32_t vw = lds32(sp + kBfp8Half + lane * 4);
             if (nvalid < kPageTokens) {
-                if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
-                if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
-            }
-            // ================= online softmax (log2 domain) =================
-            // The warp-wide maximum is only formed when some score exceeds the running maximum.
-            if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
-                float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
+                // exponent bytes of masked tokens count as 0: they neither raise the reference exponent
+                // nor produce non-finite weights
+                uint32_t keep = 0;
+                const int tt = lane >> 3;
 #pragma unroll
-                for (int d = 4; d <= 16; d <<= 1) {
-                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
-                }
-                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-                const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
-                m0 = mn0;
-                m1 = mn1;
-                lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
+                for (int c = 0; c < 4; ++c)
+                    if (2 * tt + (c & 1) + 8 * (c >> 1) < nvalid) keep |= 0xFFu << (8 * c);
+                vw &= keep;
             }
-            // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
-            const uint32_t pb0 = movmatrix_trans(pack_half2(ex2f(s0 - m0), ex2f(s1 - m1)));   // tokens 2*t4, 2*t4+1 of head gq
-            const uint32_t pb1 = movmatrix_trans(pack_half2(ex2f(s2 - m0), ex2f(s3 - m1)));   // tokens 2*t4+8, 2*t4+9
-            {
-                const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
-                mma_f16_acc(lacc, ones, pb0, pb1);
-            }
-            // ================= P.V =================
-            {
-                uint4 vs[4];           // (f01, f89) of blocks 2c, 2c+1
-#pragma unroll
-                for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + t4 * 64 + c * 16);
+            sts128(scrK + lane * 16, (kw << 23) & 0x7F800000u, (kw << 15) & 0x7F800000u, (kw << 7) & 0x7F800000u,
+                   (kw >> 1) & 0x7F800000u);
+            const uint32_t mx2 = __vmaxu2((vw >> 8) & 0x00FF00FFu, vw & 0x00FF00FFu);
+            int emax = (int)max(mx2 & 0xFFFFu, mx2 >> 16);
+            if (__any_sync(0xFFFFFFFFu, emax > Rmine)) {
+                // a V block exponent above the reference: raise it and rescale that block's accumulators
+                emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
+                emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
+                const int Rnew = max(Rmine, emax);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const uint4 &vv = vm[j >> 1];
-                    const uint32_t wl = (j & 1) ? vv.z : vv.x, wh = (j & 1) ? vv.w : vv.y;   // channels gq, gq+8 of block j
-                    uint32_t af[4];
-                    af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
-                    af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
-                    af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
-                    af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
-                    const uint32_t f01 = (j & 1) ? vs[j >> 1].z : vs[j >> 1].x, f89 = (j & 1) ? vs[j >> 1].w : vs[j >> 1].y;
-                    mma_f16_acc(o[j], af, hmul2_u32(pb0, f01), hmul2_u32(pb1, f89));
+                    const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
+                    const float fr = dlt < -126 ? 0.f : pow2_field(127 + dlt);
+                    o[j][0] *= fr; o[j][1] *= fr; o[j][2] *= fr; o[j][3] *= fr;
                 }
+                Rmine = Rnew;
             }
-            __syncwarp();      // every lane is done with the scratch tables
+            // FP16 scale 2^(E - R + 15) of every (token pair, block): exponent field max(E - R + 30, 0)
+            const uint32_t kmine = ((uint32_t)(30 - Rmine) & 0xFFFFu) * 0x00010001u;
+            sts64(scrV + lane * 8, __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4140u), kmine, 0u) << 10,
+                  __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4342u), kmine, 0u) << 10);
         }
+        uint4 km[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) km[c] = lds128(sp + 128 + c * 512 + lane * 16);
+        __syncwarp();
 
-        // ---- merge the warps' states of this segment: pairwise tree, at most kSlots states in shared memory ----
-        consumer_bar_sync();                           // the scratch tables (same memory as the slots) are idle now
-        if (kMode != 1 && alive) {
-            // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
+        // ================= Q.K^T =================
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+            float ks[16];      // 2^(E-127): token gq blocks 0..7, token gq+8 blocks 0..7
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint4 v = lds128(scrK + gq * 64 + c * 16);
+                ks[4 * c] = __uint_as_float(v.x); ks[4 * c + 1] = __uint_as_float(v.y);
+                ks[4 * c + 2] = __uint_as_float(v.z); ks[4 * c + 3] = __uint_as_float(v.w);
+            }
+            const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float vsc = pow2_field(min(__shfl_sync(0xFFFFFFFFu, Rmine, j) + 3, 254));
-                o[j][0] *= vsc; o[j][1] *= vsc; o[j][2] *= vsc; o[j][3] *= vsc;
+                const uint4 &klo = km[(j >> 2) * 2], &khi = km[(j >> 2) * 2 + 1];
+                const uint32_t wl = (j & 3) == 0 ? klo.x : (j & 3) == 1 ? klo.y : (j & 3) == 2 ? klo.z : klo.w;
+                const uint32_t wh = (j & 3) == 0 ? khi.x : (j & 3) == 1 ? khi.y : (j & 3) == 2 ? khi.z : khi.w;
+                uint32_t af[4];
+                af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
+                af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
+                af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
+                af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
+                float d[4];
+                mma_f16(d, af, qf[j][0], qf[j][1], zero4);
+                sc[0] = fmaf(d[0], ks[j], sc[0]);
+                sc[1] = fmaf(d[1], ks[j], sc[1]);
+                sc[2] = fmaf(d[2], ks[8 + j], sc[2]);
+                sc[3] = fmaf(d[3], ks[8 + j], sc[3]);
             }
         }
-        float l0 = lacc[0], l1 = lacc[1];
-#pragma unroll 1
-        for (int n = kConsumerWarps; n > 1; n = (n + 1) / 2) {
-            const int half = (n + 1) / 2;              // warps [half, n) hand their state to warps [0, n - half)
-#pragma unroll 1
-            for (int base = 0; base < n - half; base += kSlots) {
-                const int wr = warp - half - base;     // slot this warp writes in this round, if in [0, kSlots)
-                if (kMode != 1 && warp >= half && warp < n && wr >= 0 && wr < kSlots) {
-                    float *slot = comb + wr * kSlotFloats;
+        // the V element words go to registers now, so that the ring slot can be re-armed for the record
+        // three ahead while softmax and P.V run
+        uint4 vm[4];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
+        for (int c = 0; c < 4; ++c) vm[c] = lds128(sp + kBfp8Half + 128 + c * 512 + lane * 16);
+        __syncwarp();
+        if (k + kDepth < Rw) {
+            if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads above, bulk write below
+            issue();
+        }
+        float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
+        if (nvalid < kPageTokens) {
+            if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
+            if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
+        }
+        // ================= online softmax (log2 domain) =================
+        // The warp-wide maximum is only formed when some score exceeds the running maximum.
+        if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
+            float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) slot[(j * 4 + k) * 32 + lane] = o[j][k];
-                    if (gq == 0) {
-                        slot[1024 + t4 * 4 + 0] = m0; slot[1024 + t4 * 4 + 1] = m1;
-                        slot[1024 + t4 * 4 + 2] = l0; slot[1024 + t4 * 4 + 3] = l1;
-                    }
-                }
-                consumer_bar_sync();
-                const int rd = warp - base;            // slot this warp reads in this round, if in [0, kSlots)
-                if (kMode != 1 && warp < n - half && rd >= 0 && rd < kSlots) {
-                    const float *slot = comb + rd * kSlotFloats;
-                    const float pm0 = slot[1024 + t4 * 4 + 0], pm1 = slot[1024 + t4 * 4 + 1];
-                    const float pl0 = slot[1024 + t4 * 4 + 2], pl1 = slot[1024 + t4 * 4 + 3];
-                    const float M0 = fmaxf(m0, pm0), M1 = fmaxf(m1, pm1);
-                    const float a0 = m0 == -INFINITY ? 0.f : ex2f(m0 - M0), a1 = m1 == -INFINITY ? 0.f : ex2f(m1 - M1);
-                    const float c0 = pm0 == -INFINITY ? 0.f : ex2f(pm0 - M0), c1 = pm1 == -INFINITY ? 0.f : ex2f(pm1 - M1);
-                    l0 = l0 * a0 + pl0 * c0;
-                    l1 = l1 * a1 + pl1 * c1;
-                    m0 = M0;
-                    m1 = M1;
+            for (int d = 4; d <= 16; d <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
+            }
+            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+            const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
+            m0 = mn0;
+            m1 = mn1;
+            lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        o[j][0] = o[j][0] * a0 + slot[(j * 4 + 0) * 32 + lane] * c0;
-                        o[j][1] = o[j][1] * a1 + slot[(j * 4 + 1) * 32 + lane] * c1;
-                        o[j][2] = o[j][2] * a0 + slot[(j * 4 + 2) * 32 + lane] * c0;
-                        o[j][3] = o[j][3] * a1 + slot[(j * 4 + 3) * 32 + lane] * c1;
-                    }
-                }
-                consumer_bar_sync();
+            for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
+        }
+        // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
+        const uint32_t pb0 = movmatrix_trans(pack_half2(ex2f(s0 - m0), ex2f(s1 - m1)));   // tokens 2*t4, 2*t4+1 of head gq
+        const uint32_t pb1 = movmatrix_trans(pack_half2(ex2f(s2 - m0), ex2f(s3 - m1)));   // tokens 2*t4+8, 2*t4+9
+        {
+            const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
+            mma_f16_acc(lacc, ones, pb0, pb1);
+        }
+        // ================= P.V =================
+        {
+            uint4 vs[4];           // (f01, f89) of blocks 2c, 2c+1
+#pragma unroll
+            for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + t4 * 64 + c * 16);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint4 &vv = vm[j >> 1];
+                const uint32_t wl = (j & 1) ? vv.z : vv.x, wh = (j & 1) ? vv.w : vv.y;   // channels gq, gq+8 of block j
+                uint32_t af[4];
+                af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
+                af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
+                af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
+                af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
+                const uint32_t f01 = (j & 1) ? vs[j >> 1].z : vs[j >> 1].x, f89 = (j & 1) ? vs[j >> 1].w : vs[j >> 1].y;
+                mma_f16_acc(o[j], af, hmul2_u32(pb0, f01), hmul2_u32(pb1, f89));
             }
         }
-        if (warp == 0 && (kMode == 0 || (kMode == 2 && a.batch < 0)) && alive) {   // the issue-rate probe never stores, but keeps its arithmetic live
-            const bool whole = lo == seg0 && hi == seg1;
-            const int h0 = 2 * t4, h1 = 2 * t4 + 1;
-            if (whole) {
-                const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
-                const int64_t ob = ((int64_t)b * a.cv.num_q_heads + (int64_t)g * G) * kHeadDim;
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int h = (k & 1) ? h1 : h0, c = 16 * j + gq + 8 * (k >> 1);
-                        if (h < G) {
-                            const float res = o[j][k] * ((k & 1) ? i1 : i0);
-                            if (a.out_dtype == HMA_OUT_F32) reinterpret_cast<float *>(a.out)[ob + h * kHeadDim + c] = res;
-                            else reinterpret_cast<uint16_t *>(a.out)[ob + h * kHeadDim + c] = f32_to_bf16_rne(res);
-                        }
-                    }
-            } else {
-                float *tp = a.tiles + ((int64_t)blockIdx.x + ((int64_t)b * Hkv + g)) * kTileFloats;
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) tp[((k & 1) ? h1 : h0) * kHeadDim + 16 * j + gq + 8 * (k >> 1)] = o[j][k];
-                if (gq == 0) {
-                    tp[8 * kHeadDim + h0] = m0; tp[8 * kHeadDim + h1] = m1;
-                    tp[8 * kHeadDim + 8 + h0] = l0; tp[8 * kHeadDim + 8 + h1] = l1;
-                }
-            }
-        }
-
-        w = hi;
-        if (++g == Hkv) {
-            g = 0;
-            do { ++b; } while (b < B && cum[b + 1] == cum[b]);
-        }
+        __syncwarp();      // every lane is done with the scratch tables
+    }
+    if (alive) finish_segment();
+    else if (lane == 0 && kMode < 2) {
+        // a wait ran out: give the copies still in flight a bounded chance to land before the warp leaves
+        for (int s = 0; s < kDepth; ++s)
+            for (uint32_t it = 0; it < (1u << 16) && !mbar_try_wait(full0 + 8 * s, 0) && !mbar_try_wait(full0 + 8 * s, 1); ++it) {}
     }
 }
 
-// ---------------------------------------------------------------- cross-split reduction
-// One CTA per (sequence, kv head).  Segments that one CTA of the main kernel covered entirely were
-// already written there; the rest are merged here from their partial tiles, in CTA order.
-__global__ void __launch_bounds__(128) attn_reduce_kernel(const AttnArgs a, int n_ctas)
+// ---------------------------------------------------------------- cross-split merge
+// One CTA per (sequence, kv head), one warp per q head, four channels per lane.  Segments that a single worker
+// held entirely were written by the main kernel.  Lane i of a chunk holds (m, l) of part i, so the weights of up
+// to 32 parts come from one round of loads; the 128-vectors are then fetched four parts at a time.
+__global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int n_ctas)
 {
-    const int Hkv = a.cv.num_kv_heads, G = a.cv.num_q_heads / Hkv;
-    const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, c = threadIdx.x;
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // the main kernel's tiles are complete and visible
+    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
+    const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, h = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (h >= G) return;
     const int np = a.cum[b + 1] - a.cum[b];
-    const int64_t W = (int64_t)Hkv * a.cum[a.batch], N = n_ctas;
-    const int64_t obase = ((int64_t)b * a.cv.num_q_heads + (int64_t)g * G) * kHeadDim + c;
-    if (np == 0) {
-        for (int h = 0; h < G; ++h) {
-            if (a.out_dtype == HMA_OUT_F32) reinterpret_cast<float *>(a.out)[obase + h * kHeadDim] = 0.f;
-            else reinterpret_cast<uint16_t *>(a.out)[obase + h * kHeadDim] = 0;
-        }
-        return;
-    }
+    if (np == 0) return;                                         // rows of empty sequences were zeroed by the main kernel
+    const int64_t W = (int64_t)Hkv * a.cum[a.batch];
+    const int64_t NWK = max((int64_t)1, min((int64_t)n_ctas * kWarps, W / kMinRecords));
     const int64_t ws = (int64_t)Hkv * a.cum[b] + (int64_t)g * np, we = ws + np;
-    const int64_t i0 = ((ws + 1) * N - 1) / W, i1 = (we * N - 1) / W;     // first and last CTA touching the segment
-    if (i0 == i1) return;
-    for (int h = 0; h < G; ++h) {
-        float M = -INFINITY;
-        for (int64_t i = i0; i <= i1; ++i) {
-            if (i * W / N >= (i + 1) * W / N) continue;   // CTA with an empty range wrote nothing
-            M = fmaxf(M, a.tiles[(i + blockIdx.x) * kTileFloats + 8 * kHeadDim + h]);
+    const int64_t u0 = ((ws + 1) * NWK - 1) / W, u1 = (we * NWK - 1) / W;     // first and last worker of the segment
+    if (u0 == u1) return;
+    const float *t0 = a.tiles + (int64_t)blockIdx.x * kTileFloats;           // part i is at t0 + i * kTileFloats
+    float M = -INFINITY;
+    for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
+        const int64_t i = c0 + lane;
+        float mm = i <= u1 ? __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h) : -INFINITY;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, d));
+        M = fmaxf(M, mm);
+    }
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+    for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
+        const int64_t i = c0 + lane;
+        float wgt = 0.f, dsum = 0.f;
+        if (i <= u1) {
+            const float mm = __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h);
+            wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
+            dsum = wgt * __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + 8 + h);
         }
-        float num = 0.f, den = 0.f;
-        for (int64_t i = i0; i <= i1; ++i) {
-            if (i * W / N >= (i + 1) * W / N) continue;
-            const float *tp = a.tiles + (i + blockIdx.x) * kTileFloats;
-            const float mw = tp[8 * kHeadDim + h];
-            const float wgt = mw == -INFINITY ? 0.f : ex2f(mw - M);
-            num = fmaf(wgt, tp[h * kHeadDim + c], num);
-            den = fmaf(wgt, tp[8 * kHeadDim + 8 + h], den);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) dsum += __shfl_xor_sync(0xFFFFFFFFu, dsum, d);     // fixed butterfly order
+        den += dsum;
+        const int cnt = (int)min((int64_t)32, u1 - c0 + 1);
+        for (int j0 = 0; j0 < cnt; j0 += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+                v[jj] = j0 + jj < cnt ? __ldcg(reinterpret_cast<const float4 *>(t0 + (c0 + j0 + jj) * kTileFloats + h * kHeadDim) + lane)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const float wj = __shfl_sync(0xFFFFFFFFu, wgt, (j0 + jj) & 31);
+                num.x = fmaf(wj, v[jj].x, num.x); num.y = fmaf(wj, v[jj].y, num.y);
+                num.z = fmaf(wj, v[jj].z, num.z); num.w = fmaf(wj, v[jj].w, num.w);
+            }
         }
-        const float res = den > 0.f ? num / den : 0.f;
-        if (a.out_dtype == HMA_OUT_F32) reinterpret_cast<float *>(a.out)[obase + h * kHeadDim] = res;
-        else reinterpret_cast<uint16_t *>(a.out)[obase + h * kHeadDim] = f32_to_bf16_rne(res);
+    }
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    const int64_t oi = ((int64_t)b * Hq + (int64_t)g * G + h) * kHeadDim + 4 * lane;
+    if (a.out_dtype == HMA_OUT_F32) {
+        reinterpret_cast<float4 *>(a.out)[oi >> 2] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+    } else {
+        const uint32_t lo = f32_to_bf16_rne(num.x * inv) | ((uint32_t)f32_to_bf16_rne(num.y * inv) << 16);
+        const uint32_t hi = f32_to_bf16_rne(num.z * inv) | ((uint32_t)f32_to_bf16_rne(num.w * inv) << 16);
+        reinterpret_cast<uint2 *>(a.out)[oi >> 2] = make_uint2(lo, hi);
     }
 }
 
 static size_t attn_smem_bytes(int batch)
 {
-    return (size_t)kStages * kBfp8Record + (size_t)kSlots * kSlotFloats * 4 + 2 * kStages * 8 + kStages * 4 +
-           (16 + kThreads) * 4 + ((size_t)batch + 1) * 4;
+    return (size_t)kStages * kBfp8Record + (size_t)kWarps * kScratch + kStages * 8 + kStages * 4 + (16 + kThreads) * 4 +
+           ((size_t)batch + 1) * 4;
 }
 
 static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 4 + 255) & ~(size_t)255; }
@@ -669,7 +646,8 @@ static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 4 + 255) & ~(
 extern "C" size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *desc, int32_t batch)
 {
     if (!desc || batch < 0 || desc->num_kv_heads <= 0) return 0;
-    return hma::cum_bytes(batch) + ((size_t)hma::kMaxCtas + (size_t)batch * desc->num_kv_heads) * hma::kTileFloats * 4;
+    return hma::cum_bytes(batch) +
+           ((size_t)hma::kMaxCtas * hma::kWarps + (size_t)batch * desc->num_kv_heads) * hma::kTileFloats * 4;
 }
 
 static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, const void *q, void *out, int32_t out_dtype,
@@ -726,9 +704,19 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     if (probe) return HMA_OK;
-    hma::attn_reduce_kernel<<<batch * cache->desc.num_kv_heads, 128, 0, s>>>(a, n_ctas);
+    // the merge kernel may be scheduled while the main kernel still runs; it waits on the grid dependency itself
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(batch * cache->desc.num_kv_heads));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_kernel, a, n_ctas));
     hma::count_launch();
-    HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;
 }
 
