@@ -33,7 +33,7 @@ constexpr int kScratch = 768;                     // per warp: 512 B of fp32 K s
 constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile: o[8][128], m[8], l[8]
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kMaxBatch = 2048;
-constexpr int kMaxCtas = 256;
+constexpr int kMaxCtas = 160;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
 constexpr int kMinRecords = 8;                    // fewest records a worker takes
 
 struct AttnArgs {
