@@ -46,7 +46,8 @@ typedef enum {
     HMA_ERR_ALIGNMENT = 3,
     HMA_ERR_WORKSPACE_TOO_SMALL = 4,
     HMA_ERR_CUDA = 5,
-    HMA_ERR_DEVICE_FLAGGED = 6
+    HMA_ERR_DEVICE_FLAGGED = 6,
+    HMA_ERR_STATIC_LIMIT = 7      /* the request does not fit the library's built-in scratch array */
 } hma_status_t;
 
 typedef enum { HMA_KV_BFP8 = 0, HMA_KV_BF16 = 1 } hma_kv_format_t;
@@ -144,6 +145,31 @@ hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,
                                   const int32_t *block_table, int32_t max_pages_per_seq,
                                   const int32_t *context_lens, int32_t batch, float sm_scale,
                                   void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * hma_decode_attention for callers that cannot allocate.  (The paper has no counterpart: this exists for
+ * the way the library gets embedded, not for the method.)  A decode loop that fixed its memory pool at
+ * start-up, or code running where the host framework forbids allocation, has no workspace to pass; here
+ * the scratch is a 12.2 MiB array that is part of the library image on every GPU that loads it
+ * (hma_decode_attention_static_limit_bytes returns the exact size).  The call allocates and frees nothing.
+ *
+ *   - same arguments and results as hma_decode_attention, without the workspace pair; the outputs of the
+ *     two entry points are identical for identical inputs.
+ *   - limit: hma_decode_attention_workspace_bytes(desc, batch) must not exceed the array, which holds for
+ *     batch * num_kv_heads <= 512 with batch <= 1000; anything larger returns HMA_ERR_STATIC_LIMIT and
+ *     enqueues nothing.
+ *   - the first call on each device looks up the array's device address (with that device current) and sets
+ *     kernel attributes; make that first call outside any stream capture.
+ *   - all calls on a device share the one array.  Nothing in it has to start at zero and a call never reads
+ *     what an earlier call left, but two calls that overlap on the GPU (different streams) race on it:
+ *     keep such calls on one stream or order them with events.
+ */
+size_t hma_decode_attention_static_limit_bytes(void);
+hma_status_t hma_decode_attention_static(const hma_cache_t *cache, int32_t layer,
+                                         const void *q, void *out, int32_t out_dtype,
+                                         const int32_t *block_table, int32_t max_pages_per_seq,
+                                         const int32_t *context_lens, int32_t batch, float sm_scale,
+                                         void *stream);
 
 /* Same contract, computed by a plain one-CTA-per-(sequence, kv head) CUDA-core kernel that decodes
  * every element to BF16 first (the elementwise reconstruction section 3.3 compares against).

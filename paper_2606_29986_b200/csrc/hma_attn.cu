@@ -746,3 +746,39 @@ extern "C" hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_
     return launch_attention(cache, layer, nullptr, nullptr, HMA_OUT_BF16, block_table, max_pages_per_seq, context_lens, batch,
                             1.0f, workspace, workspace_bytes, stream, 2);
 }
+
+// ---------------------------------------------------------------- decode attention without a caller workspace
+// Some callers cannot hand the library a workspace because they cannot allocate device memory at the point of
+// the call: a serving loop whose memory pool was sized and frozen at start-up, a plug-in that runs inside
+// another framework's allocator-free region, a host that has already given every byte to the KV cache.  For
+// them the scratch lives in the library image itself.  Every GPU that loads the library carries the array
+// below until the process exits.
+namespace hma {
+constexpr int kStaticMaxSegments = 512;       // batch * num_kv_heads
+constexpr size_t kStaticWsBytes = 4096 + (size_t)(kMaxCtas * kWarps + kStaticMaxSegments) * kTileFloats * 4;   // 12.2 MiB
+static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
+constexpr int kMaxDevices = 64;
+static void *g_static_ws_ptr[kMaxDevices];    // device address of g_static_ws on each device, resolved on first use
+}  // namespace hma
+
+extern "C" size_t hma_decode_attention_static_limit_bytes(void) { return hma::kStaticWsBytes; }
+
+extern "C" hma_status_t hma_decode_attention_static(const hma_cache_t *cache, int32_t layer, const void *q, void *out,
+                                                    int32_t out_dtype, const int32_t *block_table, int32_t max_pages_per_seq,
+                                                    const int32_t *context_lens, int32_t batch, float sm_scale, void *stream)
+{
+    if (!cache || batch < 0) return HMA_ERR_INVALID_ARG;
+    if (hma_decode_attention_workspace_bytes(&cache->desc, batch) > hma::kStaticWsBytes) return HMA_ERR_STATIC_LIMIT;
+    int dev = 0;
+    HMA_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= hma::kMaxDevices) return HMA_ERR_STATIC_LIMIT;
+    if (!hma::g_static_ws_ptr[dev]) {
+        // In host code the array's name is only a handle: the device address has to be asked for, with the
+        // device that will run the kernels current.
+        void *p = nullptr;
+        HMA_CUDA_OK(cudaGetSymbolAddress(&p, hma::g_static_ws));
+        hma::g_static_ws_ptr[dev] = p;
+    }
+    return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
+                            hma::g_static_ws_ptr[dev], hma::kStaticWsBytes, stream, 0);
+}

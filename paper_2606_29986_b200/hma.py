@@ -15,6 +15,7 @@ _LIB_PATH = os.path.join(_HERE, "libhma.so")
 HMA_OK = 0
 HMA_ERR_INVALID_ARG, HMA_ERR_UNSUPPORTED_SHAPE, HMA_ERR_ALIGNMENT = 1, 2, 3
 HMA_ERR_WORKSPACE_TOO_SMALL, HMA_ERR_CUDA, HMA_ERR_DEVICE_FLAGGED = 4, 5, 6
+HMA_ERR_STATIC_LIMIT = 7
 HMA_KV_BFP8, HMA_KV_BF16 = 0, 1
 HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR = 0, 1
 HMA_OUT_BF16, HMA_OUT_F32 = 0, 1
@@ -59,6 +60,10 @@ def lib():
         L.hma_decode_attention_workspace_bytes.argtypes = [ctypes.POINTER(CacheDesc), i32]
         L.hma_decode_attention.restype = i32
         L.hma_decode_attention.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp, sz, vp]
+        L.hma_decode_attention_static.restype = i32
+        L.hma_decode_attention_static.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
+        L.hma_decode_attention_static_limit_bytes.restype = sz
+        L.hma_decode_attention_static_limit_bytes.argtypes = []
         L.hma_kv_read_probe.restype = i32
         L.hma_kv_read_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
         L.hma_attention_alu_probe.restype = i32
@@ -156,6 +161,22 @@ def hma_decode_attention(cache, layer, q, out, block_table, context_lens, sm_sca
                                       block_table.shape[1], _ptr(context_lens), q.shape[0], float(sm_scale),
                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "hma_decode_attention")
+
+
+def hma_decode_attention_static(cache, layer, q, out, block_table, context_lens, sm_scale, stream=None):
+    """hma_decode_attention without a workspace argument, for callers that cannot allocate device memory.
+
+    The scratch is an array inside the library (hma_decode_attention_static_limit_bytes() bytes on every GPU
+    that loads it).  Raises HmaError(HMA_ERR_STATIC_LIMIT) when batch * kv heads is too large for it.  Calls
+    on one device share the array: keep them on one stream.  Make the first call outside stream capture."""
+    out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
+    _check(lib().hma_decode_attention_static(cache.handle, layer, _ptr(q), _ptr(out), out_dtype, _ptr(block_table),
+                                             block_table.shape[1], _ptr(context_lens), q.shape[0], float(sm_scale),
+                                             _stream(stream)), "hma_decode_attention_static")
+
+
+def hma_decode_attention_static_limit_bytes():
+    return int(lib().hma_decode_attention_static_limit_bytes())
 
 
 def hma_kv_read_probe(cache, layer, block_table, context_lens, workspace, stream=None):
