@@ -586,39 +586,67 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int n
     const int64_t u0 = ((ws + 1) * NWK - 1) / W, u1 = (we * NWK - 1) / W;     // first and last worker of the segment
     if (u0 == u1) return;
     const float *t0 = a.tiles + (int64_t)blockIdx.x * kTileFloats;           // part i is at t0 + i * kTileFloats
-    float M = -INFINITY;
-    for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
-        const int64_t i = c0 + lane;
-        float mm = i <= u1 ? __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h) : -INFINITY;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, d));
-        M = fmaxf(M, mm);
-    }
     float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
     float den = 0.f;
-    for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
-        const int64_t i = c0 + lane;
-        float wgt = 0.f, dsum = 0.f;
-        if (i <= u1) {
-            const float mm = __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h);
-            wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
-            dsum = wgt * __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + 8 + h);
+    const int P = (int)(u1 - u0 + 1);
+    if (P <= 16) {
+        // common case: every load of the merge is issued before any is used (one trip to L2)
+        float4 v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            v[j] = j < P ? __ldcg(reinterpret_cast<const float4 *>(t0 + (u0 + j) * kTileFloats + h * kHeadDim) + lane)
+                         : make_float4(0.f, 0.f, 0.f, 0.f);
+        float mm = -INFINITY, ll = 0.f;
+        if (lane < P) {
+            mm = __ldcg(t0 + (u0 + lane) * kTileFloats + 8 * kHeadDim + h);
+            ll = __ldcg(t0 + (u0 + lane) * kTileFloats + 8 * kHeadDim + 8 + h);
         }
+        float M = mm;
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) dsum += __shfl_xor_sync(0xFFFFFFFFu, dsum, d);     // fixed butterfly order
-        den += dsum;
-        const int cnt = (int)min((int64_t)32, u1 - c0 + 1);
-        for (int j0 = 0; j0 < cnt; j0 += 4) {
-            float4 v[4];
+        for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
+        const float wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
+        den = wgt * ll;
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj)
-                v[jj] = j0 + jj < cnt ? __ldcg(reinterpret_cast<const float4 *>(t0 + (c0 + j0 + jj) * kTileFloats + h * kHeadDim) + lane)
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int d = 16; d > 0; d >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, d);          // fixed butterfly order
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-                const float wj = __shfl_sync(0xFFFFFFFFu, wgt, (j0 + jj) & 31);
-                num.x = fmaf(wj, v[jj].x, num.x); num.y = fmaf(wj, v[jj].y, num.y);
-                num.z = fmaf(wj, v[jj].z, num.z); num.w = fmaf(wj, v[jj].w, num.w);
+        for (int j = 0; j < 16; ++j) {
+            const float wj = __shfl_sync(0xFFFFFFFFu, wgt, j);
+            num.x = fmaf(wj, v[j].x, num.x); num.y = fmaf(wj, v[j].y, num.y);
+            num.z = fmaf(wj, v[j].z, num.z); num.w = fmaf(wj, v[j].w, num.w);
+        }
+    } else {
+        float M = -INFINITY;
+        for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
+            const int64_t i = c0 + lane;
+            float mm = i <= u1 ? __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h) : -INFINITY;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, d));
+            M = fmaxf(M, mm);
+        }
+        for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
+            const int64_t i = c0 + lane;
+            float wgt = 0.f, dsum = 0.f;
+            if (i <= u1) {
+                const float mm = __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h);
+                wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
+                dsum = wgt * __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + 8 + h);
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) dsum += __shfl_xor_sync(0xFFFFFFFFu, dsum, d);     // fixed butterfly order
+            den += dsum;
+            const int cnt = (int)min((int64_t)32, u1 - c0 + 1);
+            for (int j0 = 0; j0 < cnt; j0 += 4) {
+                float4 v[4];
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj)
+                    v[jj] = j0 + jj < cnt ? __ldcg(reinterpret_cast<const float4 *>(t0 + (c0 + j0 + jj) * kTileFloats + h * kHeadDim) + lane)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const float wj = __shfl_sync(0xFFFFFFFFu, wgt, (j0 + jj) & 31);
+                    num.x = fmaf(wj, v[jj].x, num.x); num.y = fmaf(wj, v[jj].y, num.y);
+                    num.z = fmaf(wj, v[jj].z, num.z); num.w = fmaf(wj, v[jj].w, num.w);
+                }
             }
         }
     }

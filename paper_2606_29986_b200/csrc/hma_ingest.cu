@@ -66,59 +66,64 @@ __global__ void __launch_bounds__(256) ingest_kernel(CacheView cv, IngestArgs a)
     }
     __syncthreads();
     uint8_t *rec = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)record_bytes(cv.format);
-    const bool full = lo == 0 && hi == kPageTokens;
-    if (cv.format == HMA_KV_BFP8) {
-        for (int wi = threadIdx.x; wi < kBfp8Record / 4; wi += blockDim.x) {
-            const int t = wi >= kBfp8Half / 4;
-            const int o = wi * 4 - t * kBfp8Half;        // offset inside the K or V part
-            uint32_t val = 0, mask = 0;
+    // byte mask of the tokens of a V-side word (tokens 2*tq, 2*tq+1, 2*tq+8, 2*tq+9) that are in range
+    auto vmask = [&](int tq) {
+        uint32_t m = 0;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                int tok, src;
-                const int ob = o + k;
-                if (ob < 128) {                          // exponent bytes
-                    int j;
-                    if (t == 0) { tok = (ob >> 4) + 8 * ((ob >> 3) & 1); j = ob & 7; }
-                    else { const int kk = ob & 3; tok = 2 * (ob >> 5) + (kk & 1) + 8 * (kk >> 1); j = (ob >> 2) & 7; }
-                    src = j;
-                } else {                                  // element bytes
-                    const int e = ob - 128, c = e >> 9, r = e & 511, lane = r >> 4, w4 = (r >> 2) & 3, kk = r & 3;
-                    const int g = lane >> 2, tq = lane & 3;
-                    int ch;
-                    if (t == 0) { tok = g + 8 * (c & 1); ch = 16 * (4 * (c >> 1) + w4) + 4 * tq + kk; }
-                    else { tok = 2 * tq + (kk & 1) + 8 * (kk >> 1); ch = 16 * (2 * c + (w4 >> 1)) + g + 8 * (w4 & 1); }
-                    src = 16 + ch;
-                }
-                if (tok >= lo && tok < hi) {
-                    val |= (uint32_t)rows[t][tok][src] << (8 * k);
-                    mask |= 0xFFu << (8 * k);
-                }
+        for (int k = 0; k < 4; ++k) {
+            const int tok = 2 * tq + (k & 1) + 8 * (k >> 1);
+            if (tok >= lo && tok < hi) m |= 0xFFu << (8 * k);
+        }
+        return m;
+    };
+    auto put = [&](uint32_t *dst, uint32_t val, uint32_t mask) {
+        if (mask == 0xFFFFFFFFu) *dst = val;
+        else if (mask) *dst = (*dst & ~mask) | (val & mask);
+    };
+    if (cv.format == HMA_KV_BFP8) {
+        uint32_t *rk = reinterpret_cast<uint32_t *>(rec), *rv = reinterpret_cast<uint32_t *>(rec + kBfp8Half);
+        // K exponents: word = blocks 4*(w&1)..+3 of token (w>>2) + 8*((w>>1)&1): four consecutive staged bytes
+        // V exponents: word = block (w&7) of tokens 2*tq.., tq = w>>3
+        if (threadIdx.x < 32) {
+            const int w = threadIdx.x, tok = (w >> 2) + 8 * ((w >> 1) & 1);
+            put(rk + w, *reinterpret_cast<const uint32_t *>(&rows[0][tok][4 * (w & 1)]), tok >= lo && tok < hi ? 0xFFFFFFFFu : 0u);
+        } else if (threadIdx.x < 64) {
+            const int w = threadIdx.x - 32, tq = w >> 3, j = w & 7;
+            const uint32_t val = rows[1][2 * tq][j] | (rows[1][2 * tq + 1][j] << 8) | (rows[1][2 * tq + 8][j] << 16) |
+                                 ((uint32_t)rows[1][2 * tq + 9][j] << 24);
+            put(rv + w, val, vmask(tq));
+        }
+        for (int wi = threadIdx.x; wi < 512; wi += blockDim.x) {
+            const int c = wi >> 7, lane = (wi >> 2) & 31, w4 = wi & 3, g = lane >> 2, tq = lane & 3;
+            {   // K elements: four consecutive channels of one token
+                const int tok = g + 8 * (c & 1), ch = 16 * (4 * (c >> 1) + w4) + 4 * tq;
+                put(rk + 32 + wi, *reinterpret_cast<const uint32_t *>(&rows[0][tok][16 + ch]), tok >= lo && tok < hi ? 0xFFFFFFFFu : 0u);
             }
-            uint32_t *dst = reinterpret_cast<uint32_t *>(rec) + wi;
-            if (mask == 0xFFFFFFFFu) *dst = val;
-            else if (mask) *dst = (*dst & ~mask) | val;
+            {   // V elements: one channel of four tokens
+                const int ch = 16 * (2 * c + (w4 >> 1)) + g + 8 * (w4 & 1);
+                const uint32_t val = rows[1][2 * tq][16 + ch] | (rows[1][2 * tq + 1][16 + ch] << 8) |
+                                     (rows[1][2 * tq + 8][16 + ch] << 16) | ((uint32_t)rows[1][2 * tq + 9][16 + ch] << 24);
+                put(rv + 32 + wi, val, vmask(tq));
+            }
         }
     } else {
-        (void)full;
-        for (int wi = threadIdx.x; wi < kBf16Record / 4; wi += blockDim.x) {
-            const int t = wi >= kBf16Half / 4;
-            const int o = wi * 4 - t * kBf16Half;
-            uint32_t val = 0, mask = 0;
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const int ob = o + 2 * k, c = ob >> 9, r = ob & 511, lane = r >> 4, w4 = (r >> 2) & 3, kk = (r >> 1) & 1;
-                const int g = lane >> 2, tq = lane & 3;
-                int tok, ch;
-                if (t == 0) { tok = g + 8 * (c & 1); ch = 16 * (2 * (c >> 1) + (w4 >> 1)) + 4 * tq + 2 * (w4 & 1) + kk; }
-                else { tok = 2 * tq + kk + 8 * (w4 >> 1); ch = 16 * c + g + 8 * (w4 & 1); }
-                if (tok >= lo && tok < hi) {
-                    val |= bfp8_to_bf16_bits(rows[t][tok][ch >> 4], rows[t][tok][16 + ch]) << (16 * k);
-                    mask |= 0xFFFFu << (16 * k);
-                }
+        // BF16 cache: decode while scattering; a word holds two elements
+        uint32_t *rk = reinterpret_cast<uint32_t *>(rec), *rv = reinterpret_cast<uint32_t *>(rec + kBf16Half);
+        for (int wi = threadIdx.x; wi < kBf16Half / 4; wi += blockDim.x) {
+            const int c = wi >> 7, lane = (wi >> 2) & 31, w4 = wi & 3, g = lane >> 2, tq = lane & 3;
+            {   // K: channels ch, ch+1 of one token
+                const int tok = g + 8 * (c & 1), ch = 16 * (2 * (c >> 1) + (w4 >> 1)) + 4 * tq + 2 * (w4 & 1);
+                const uint32_t E = rows[0][tok][ch >> 4];
+                const uint32_t val = bfp8_to_bf16_bits(E, rows[0][tok][16 + ch]) | (bfp8_to_bf16_bits(E, rows[0][tok][16 + ch + 1]) << 16);
+                put(rk + wi, val, tok >= lo && tok < hi ? 0xFFFFFFFFu : 0u);
             }
-            uint32_t *dst = reinterpret_cast<uint32_t *>(rec) + wi;
-            if (mask == 0xFFFFFFFFu) *dst = val;
-            else if (mask) *dst = (*dst & ~mask) | val;
+            {   // V: one channel of tokens t, t+1
+                const int t = 2 * tq + 8 * (w4 >> 1), ch = 16 * c + g + 8 * (w4 & 1);
+                const uint32_t val = bfp8_to_bf16_bits(rows[1][t][ch >> 4], rows[1][t][16 + ch]) |
+                                     (bfp8_to_bf16_bits(rows[1][t + 1][ch >> 4], rows[1][t + 1][16 + ch]) << 16);
+                const uint32_t mask = (t >= lo && t < hi ? 0xFFFFu : 0u) | (t + 1 >= lo && t + 1 < hi ? 0xFFFF0000u : 0u);
+                put(rv + wi, val, mask);
+            }
         }
     }
 }
