@@ -32,7 +32,7 @@ BFP8_ROW = 272      # bytes per (token, kv head): K 136 + V 136
 BF16_ROW = 512
 # DRAM bytes per launch of attn_bfp8_kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
 # see profiles/.  Keyed by workload; None where no capture exists.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"qwen3-32b-b32-ctx8k": 575_200_000}    # profiles/attn_bfp8_kernel_qwen3-32b-b32-ctx8k_ncu_full.md
 
 
 def measured_peak():

@@ -464,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
             }
             // FP16 scale 2^(E - R + 15) of every (token pair, block): exponent field max(E - R + 30, 0)
             const uint32_t kmine = ((uint32_t)(30 - Rmine) & 0xFFFFu) * 0x00010001u;
-            sts64(scrV + lane * 8, __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4140u), kmine, 0u) << 10,
+            sts64(scrV + ((lane & 6) << 5) + ((lane >> 3) << 4) + ((lane & 1) << 3), __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4140u), kmine, 0u) << 10,
                   __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4342u), kmine, 0u) << 10);
         }
         uint4 km[4];
@@ -544,7 +544,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         {
             uint4 vs[4];           // (f01, f89) of blocks 2c, 2c+1
 #pragma unroll
-            for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + t4 * 64 + c * 16);
+            for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + c * 64 + t4 * 16);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const uint4 &vv = vm[j >> 1];
