@@ -25,11 +25,19 @@
 
 namespace hma {
 
-constexpr int kWarps = 16;
-constexpr int kThreads = kWarps * 32;
+constexpr int kWarps = 16;                        // warps per CTA on a BFP8 cache (and the bound used to size the workspace)
 constexpr int kDepth = 3;                         // ring slots per warp
-constexpr int kStages = kWarps * kDepth;
 constexpr int kScratch = 768;                     // per warp: 512 B of fp32 K scales + 256 B of FP16 V scales
+// Per cache format: a BF16 record is 8192 B, so only 8 warps x 3 slots fit in shared memory; its arithmetic is
+// light enough (no unpack) for 8 warps.
+template <int kFmt>
+struct Geo {
+    static constexpr int warps = kFmt == HMA_KV_BFP8 ? kWarps : 8;
+    static constexpr int threads = warps * 32;
+    static constexpr int stages = warps * kDepth;
+    static constexpr int record = kFmt == HMA_KV_BFP8 ? kBfp8Record : kBf16Record;
+    static constexpr int scratch = kFmt == HMA_KV_BFP8 ? kScratch : 0;
+};
 constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile: o[8][128], m[8], l[8]
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kMaxBatch = 2048;
@@ -136,6 +144,20 @@ __device__ __forceinline__ void mma_f16_acc(float (&d)[4], const uint32_t (&a)[4
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_bf16_acc(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// fp32 pair -> packed BF16 (round to nearest even), first argument in the low half
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
 {
     uint32_t d;
@@ -187,12 +209,15 @@ __device__ __forceinline__ void store_out(const AttnArgs &a, int64_t idx, float 
 // 2: the arithmetic of every record on whatever the ring holds, nothing loaded or written (issue-rate probe).
 extern __shared__ __align__(128) uint8_t smem_raw[];
 
-template <int kMode>
-__global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a)
+template <int kMode, int kFmt>
+__global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnArgs a)
 {
-    uint8_t *ring = smem_raw;                                                     // kStages x 4352
-    uint8_t *scratch = ring + kStages * kBfp8Record;                              // kWarps x kScratch
-    uint64_t *bars = reinterpret_cast<uint64_t *>(scratch + kWarps * kScratch);   // full[kStages]
+    constexpr int kWarps = Geo<kFmt>::warps, kThreads = Geo<kFmt>::threads, kStages = Geo<kFmt>::stages;
+    constexpr int kRecord = Geo<kFmt>::record;
+    constexpr bool kBfp8 = kFmt == HMA_KV_BFP8;
+    uint8_t *ring = smem_raw;                                                     // kStages records
+    uint8_t *scratch = ring + kStages * kRecord;                                  // kWarps x kScratch (BFP8 only)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(scratch + kWarps * Geo<kFmt>::scratch);   // full[kStages]
     int *stage_ok = reinterpret_cast<int *>(bars + kStages);                      // [kStages]
     int *misc = stage_ok + kStages;                                               // [0] abort word, [16..] scan scratch
     int *cum = misc + 16 + kThreads;                                              // [batch + 1]
@@ -264,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
 
     // ---- the warp's own feed: issue cursor, window of block-table entries, three ring slots ----
     const uint32_t full0 = smem_u32(bars + warp * kDepth);
-    const uint32_t ring0 = smem_u32(ring + warp * kDepth * kBfp8Record);
+    const uint32_t ring0 = smem_u32(ring + warp * kDepth * kRecord);
     int ib = b, ig = g, ip = page, inp = np;      // cursor of the next record to request
     int iwb = -1, iw0 = 0;                        // the window holds pages [iw0, iw0+32) of sequence iwb
     int32_t ipid = -1;
@@ -283,8 +308,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
             const int s = warp * kDepth + islot;
             if (pid >= 0 && pid < a.cv.num_pages) {
                 stage_ok[s] = 1;
-                mbar_arrive_expect_tx(full0 + 8 * islot, kBfp8Record);
-                bulk_load(ring0 + islot * kBfp8Record, a.cv.layer + ((int64_t)pid * Hkv + ig) * kBfp8Record, kBfp8Record,
+                mbar_arrive_expect_tx(full0 + 8 * islot, kRecord);
+                bulk_load(ring0 + islot * kRecord, a.cv.layer + ((int64_t)pid * Hkv + ig) * kRecord, kRecord,
                           full0 + 8 * islot, policy);
             } else {
                 stage_ok[s] = 0;
@@ -307,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
     // ---- consumer state ----
     const int gq = lane >> 2, t4 = lane & 3;
     const float kLog2e = 1.4426950408889634f;
-    const uint32_t scrK = smem_u32(scratch + warp * kScratch);   // fp32 2^(E-127) of every (token, block) of K
+    const uint32_t scrK = smem_u32(scratch + warp * Geo<kFmt>::scratch);   // fp32 2^(E-127) of every (token, block) of K
     const uint32_t scrV = scrK + 512;                            // FP16 scales of every (token pair, block) of V
     uint32_t qf[8][2];
     float cs0 = 0.f, cs1 = 0.f;                    // score multipliers of heads 2*t4, 2*t4+1
@@ -340,17 +365,27 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
         }
         amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
         amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
-        int shift = 0;
-        if (amax > 0.f && amax < INFINITY) shift = 14 - ((int)((__float_as_uint(amax) >> 23) & 0xFF) - 127);
-        shift = max(-120, min(120, shift));
-        const float up = pow2_field(127 + shift), down = pow2_field(127 - shift);
+        float cs;
+        if (kBfp8) {
+            int shift = 0;
+            if (amax > 0.f && amax < INFINITY) shift = 14 - ((int)((__float_as_uint(amax) >> 23) & 0xFF) - 127);
+            shift = max(-120, min(120, shift));
+            const float up = pow2_field(127 + shift), down = pow2_field(127 - shift);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            qf[j][0] = pack_half2(f[j][0] * up, f[j][1] * up);
-            qf[j][1] = pack_half2(f[j][2] * up, f[j][3] * up);
+            for (int j = 0; j < 8; ++j) {
+                qf[j][0] = pack_half2(f[j][0] * up, f[j][1] * up);
+                qf[j][1] = pack_half2(f[j][2] * up, f[j][3] * up);
+            }
+            // mantissas enter as m * 2^-24 and exponents as 2^(E-127) while values are m * 2^(E-133): 2^18 is owed
+            cs = a.sm_scale * kLog2e * down * 262144.f;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {       // Q stays BF16: exact repacking of the loaded bits
+                qf[j][0] = (__float_as_uint(f[j][0]) >> 16) | (__float_as_uint(f[j][1]) & 0xFFFF0000u);
+                qf[j][1] = (__float_as_uint(f[j][2]) >> 16) | (__float_as_uint(f[j][3]) & 0xFFFF0000u);
+            }
+            cs = a.sm_scale * kLog2e;
         }
-        // mantissas enter as m * 2^-24 and exponents as 2^(E-127) while values are m * 2^(E-133): 2^18 is owed
-        const float cs = a.sm_scale * kLog2e * down * 262144.f;
         cs0 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4) * 4);
         cs1 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4 + 1) * 4);
         m0 = -INFINITY;
@@ -363,11 +398,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
 
     auto finish_segment = [&]() {
         if (kMode == 1) return;
-        // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
+        if (kBfp8) {
+            // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float vsc = pow2_field(min(__shfl_sync(0xFFFFFFFFu, Rmine, j) + 3, 254));
-            o[j][0] *= vsc; o[j][1] *= vsc; o[j][2] *= vsc; o[j][3] *= vsc;
+            for (int j = 0; j < 8; ++j) {
+                const float vsc = pow2_field(min(__shfl_sync(0xFFFFFFFFu, Rmine, j) + 3, 254));
+                o[j][0] *= vsc; o[j][1] *= vsc; o[j][2] *= vsc; o[j][3] *= vsc;
+            }
         }
         const float l0 = lacc[0], l1 = lacc[1];
         const int h0 = 2 * t4, h1 = 2 * t4 + 1;
@@ -415,7 +452,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
             left = min(np - page, Rw - k);
         }
         --left;
-        const uint32_t sp = ring0 + slot * kBfp8Record;
+        const uint32_t sp = ring0 + slot * kRecord;
         const int s_idx = warp * kDepth + slot;
         if (kMode < 2) {
             alive = mbar_wait(full0 + 8 * slot, par, abort_word, a.cv.flags);
@@ -431,134 +468,203 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
             continue;
         }
 
-        // ---- exponents: fp32 scales for Q.K^T, reference-exponent check and FP16 scales for P.V ----
-        {
-            const uint32_t kw = lds32(sp + lane * 4);
-            uint32_t vw = lds32(sp + kBfp8Half + lane * 4);
-            if (nvalid < kPageTokens) {
-                // exponent bytes of masked tokens count as 0: they neither raise the reference exponent
-                // nor produce non-finite weights
-                uint32_t keep = 0;
-                const int tt = lane >> 3;
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (2 * tt + (c & 1) + 8 * (c >> 1) < nvalid) keep |= 0xFFu << (8 * c);
-                vw &= keep;
-            }
-            sts128(scrK + lane * 16, (kw << 23) & 0x7F800000u, (kw << 15) & 0x7F800000u, (kw << 7) & 0x7F800000u,
-                   (kw >> 1) & 0x7F800000u);
-            const uint32_t mx2 = __vmaxu2((vw >> 8) & 0x00FF00FFu, vw & 0x00FF00FFu);
-            int emax = (int)max(mx2 & 0xFFFFu, mx2 >> 16);
-            if (__any_sync(0xFFFFFFFFu, emax > Rmine)) {
-                // a V block exponent above the reference: raise it and rescale that block's accumulators
-                emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
-                emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
-                const int Rnew = max(Rmine, emax);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
-                    const float fr = dlt < -126 ? 0.f : pow2_field(127 + dlt);
-                    o[j][0] *= fr; o[j][1] *= fr; o[j][2] *= fr; o[j][3] *= fr;
+        if constexpr (kBfp8) {
+            // ---- exponents: fp32 scales for Q.K^T, reference-exponent check and FP16 scales for P.V ----
+            {
+                const uint32_t kw = lds32(sp + lane * 4);
+                uint32_t vw = lds32(sp + kBfp8Half + lane * 4);
+                if (nvalid < kPageTokens) {
+                    // exponent bytes of masked tokens count as 0: they neither raise the reference exponent
+                    // nor produce non-finite weights
+                    uint32_t keep = 0;
+                    const int tt = lane >> 3;
+    #pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if (2 * tt + (c & 1) + 8 * (c >> 1) < nvalid) keep |= 0xFFu << (8 * c);
+                    vw &= keep;
                 }
-                Rmine = Rnew;
+                sts128(scrK + lane * 16, (kw << 23) & 0x7F800000u, (kw << 15) & 0x7F800000u, (kw << 7) & 0x7F800000u,
+                       (kw >> 1) & 0x7F800000u);
+                const uint32_t mx2 = __vmaxu2((vw >> 8) & 0x00FF00FFu, vw & 0x00FF00FFu);
+                int emax = (int)max(mx2 & 0xFFFFu, mx2 >> 16);
+                if (__any_sync(0xFFFFFFFFu, emax > Rmine)) {
+                    // a V block exponent above the reference: raise it and rescale that block's accumulators
+                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
+                    emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
+                    const int Rnew = max(Rmine, emax);
+    #pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
+                        const float fr = dlt < -126 ? 0.f : pow2_field(127 + dlt);
+                        o[j][0] *= fr; o[j][1] *= fr; o[j][2] *= fr; o[j][3] *= fr;
+                    }
+                    Rmine = Rnew;
+                }
+                // FP16 scale 2^(E - R + 15) of every (token pair, block): exponent field max(E - R + 30, 0)
+                const uint32_t kmine = ((uint32_t)(30 - Rmine) & 0xFFFFu) * 0x00010001u;
+                sts64(scrV + ((lane & 6) << 5) + ((lane >> 3) << 4) + ((lane & 1) << 3), __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4140u), kmine, 0u) << 10,
+                      __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4342u), kmine, 0u) << 10);
             }
-            // FP16 scale 2^(E - R + 15) of every (token pair, block): exponent field max(E - R + 30, 0)
-            const uint32_t kmine = ((uint32_t)(30 - Rmine) & 0xFFFFu) * 0x00010001u;
-            sts64(scrV + ((lane & 6) << 5) + ((lane >> 3) << 4) + ((lane & 1) << 3), __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4140u), kmine, 0u) << 10,
-                  __viaddmax_s16x2_relu(prmt(vw, 0u, 0x4342u), kmine, 0u) << 10);
-        }
-        uint4 km[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) km[c] = lds128(sp + 128 + c * 512 + lane * 16);
-        __syncwarp();
+            uint4 km[4];
+    #pragma unroll
+            for (int c = 0; c < 4; ++c) km[c] = lds128(sp + 128 + c * 512 + lane * 16);
+            __syncwarp();
 
-        // ================= Q.K^T =================
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
-        {
-            float ks[16];      // 2^(E-127): token gq blocks 0..7, token gq+8 blocks 0..7
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint4 v = lds128(scrK + gq * 64 + c * 16);
-                ks[4 * c] = __uint_as_float(v.x); ks[4 * c + 1] = __uint_as_float(v.y);
-                ks[4 * c + 2] = __uint_as_float(v.z); ks[4 * c + 3] = __uint_as_float(v.w);
+            // ================= Q.K^T =================
+            float sc[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                float ks[16];      // 2^(E-127): token gq blocks 0..7, token gq+8 blocks 0..7
+    #pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 v = lds128(scrK + gq * 64 + c * 16);
+                    ks[4 * c] = __uint_as_float(v.x); ks[4 * c + 1] = __uint_as_float(v.y);
+                    ks[4 * c + 2] = __uint_as_float(v.z); ks[4 * c + 3] = __uint_as_float(v.w);
+                }
+                const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 &klo = km[(j >> 2) * 2], &khi = km[(j >> 2) * 2 + 1];
+                    const uint32_t wl = (j & 3) == 0 ? klo.x : (j & 3) == 1 ? klo.y : (j & 3) == 2 ? klo.z : klo.w;
+                    const uint32_t wh = (j & 3) == 0 ? khi.x : (j & 3) == 1 ? khi.y : (j & 3) == 2 ? khi.z : khi.w;
+                    uint32_t af[4];
+                    af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
+                    af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
+                    af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
+                    af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
+                    float d[4];
+                    mma_f16(d, af, qf[j][0], qf[j][1], zero4);
+                    sc[0] = fmaf(d[0], ks[j], sc[0]);
+                    sc[1] = fmaf(d[1], ks[j], sc[1]);
+                    sc[2] = fmaf(d[2], ks[8 + j], sc[2]);
+                    sc[3] = fmaf(d[3], ks[8 + j], sc[3]);
+                }
             }
-            const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
+            // the V element words go to registers now, so that the ring slot can be re-armed for the record
+            // three ahead while softmax and P.V run
+            uint4 vm[4];
+    #pragma unroll
+            for (int c = 0; c < 4; ++c) vm[c] = lds128(sp + kBfp8Half + 128 + c * 512 + lane * 16);
+            __syncwarp();
+            if (k + kDepth < Rw) {
+                if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads above, bulk write below
+                issue();
+            }
+            float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
+            if (nvalid < kPageTokens) {
+                if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
+                if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
+            }
+            // ================= online softmax (log2 domain) =================
+            // The warp-wide maximum is only formed when some score exceeds the running maximum.
+            if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
+                float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
+    #pragma unroll
+                for (int d = 4; d <= 16; d <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
+                }
+                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
+                m0 = mn0;
+                m1 = mn1;
+                lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
+            }
+            // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
+            const uint32_t pb0 = movmatrix_trans(pack_half2(ex2f(s0 - m0), ex2f(s1 - m1)));   // tokens 2*t4, 2*t4+1 of head gq
+            const uint32_t pb1 = movmatrix_trans(pack_half2(ex2f(s2 - m0), ex2f(s3 - m1)));   // tokens 2*t4+8, 2*t4+9
+            {
+                const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
+                mma_f16_acc(lacc, ones, pb0, pb1);
+            }
+            // ================= P.V =================
+            {
+                uint4 vs[4];           // (f01, f89) of blocks 2c, 2c+1
+    #pragma unroll
+                for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + c * 64 + t4 * 16);
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 &vv = vm[j >> 1];
+                    const uint32_t wl = (j & 1) ? vv.z : vv.x, wh = (j & 1) ? vv.w : vv.y;   // channels gq, gq+8 of block j
+                    uint32_t af[4];
+                    af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
+                    af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
+                    af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
+                    af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
+                    const uint32_t f01 = (j & 1) ? vs[j >> 1].z : vs[j >> 1].x, f89 = (j & 1) ? vs[j >> 1].w : vs[j >> 1].y;
+                    mma_f16_acc(o[j], af, hmul2_u32(pb0, f01), hmul2_u32(pb1, f89));
+                }
+            }
+            __syncwarp();      // every lane is done with the scratch tables
+        } else {
+            // ================= BF16 cache: the dequant-free baseline of section 3.3 =================
+            // Q.K^T: tokens on M, BF16 operands straight from the record, two accumulators to shorten the chain
+            float sca[4] = {0.f, 0.f, 0.f, 0.f}, scb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int jp = 0; jp < 4; ++jp) {
+                const uint4 klo = lds128(sp + (2 * jp) * 512 + lane * 16);       // token gq: blocks 2jp, 2jp+1
+                const uint4 khi = lds128(sp + (2 * jp + 1) * 512 + lane * 16);   // token gq+8
+                const uint32_t a0[4] = {klo.x, khi.x, klo.y, khi.y}, a1[4] = {klo.z, khi.z, klo.w, khi.w};
+                mma_bf16_acc(sca, a0, qf[2 * jp][0], qf[2 * jp][1]);
+                mma_bf16_acc(scb, a1, qf[2 * jp + 1][0], qf[2 * jp + 1][1]);
+            }
+            // the V words go to registers now, so that the ring slot can be re-armed while softmax and P.V run
+            uint4 vm[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) vm[j] = lds128(sp + kBf16Half + j * 512 + lane * 16);
+            if (nvalid < kPageTokens) {
+                // whatever the tail of the last page holds (NaN patterns included) must not reach the MMA: 0 * NaN = NaN
+                const uint32_t mlo = (2 * t4 < nvalid ? 0xFFFFu : 0u) | (2 * t4 + 1 < nvalid ? 0xFFFF0000u : 0u);
+                const uint32_t mhi = (2 * t4 + 8 < nvalid ? 0xFFFFu : 0u) | (2 * t4 + 9 < nvalid ? 0xFFFF0000u : 0u);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { vm[j].x &= mlo; vm[j].y &= mlo; vm[j].z &= mhi; vm[j].w &= mhi; }
+            }
+            __syncwarp();
+            if (k + kDepth < Rw) {
+                if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads above, bulk write below
+                issue();
+            }
+            float s0 = (sca[0] + scb[0]) * cs0, s1 = (sca[1] + scb[1]) * cs1, s2 = (sca[2] + scb[2]) * cs0, s3 = (sca[3] + scb[3]) * cs1;
+            if (nvalid < kPageTokens) {
+                if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
+                if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
+            }
+            if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
+                float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
+#pragma unroll
+                for (int d = 4; d <= 16; d <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
+                }
+                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
+                m0 = mn0;
+                m1 = mn1;
+                lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
+            }
+            // weights as BF16 hi + lo (16 significant bits): BF16-rounded weights alone would cost 1e-3 of relative error
+            const float p0 = ex2f(s0 - m0), p1 = ex2f(s1 - m1), p2 = ex2f(s2 - m0), p3 = ex2f(s3 - m1);
+            const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);
+            const uint32_t l01 = pack_bf16x2(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xFFFF0000u));
+            const uint32_t l23 = pack_bf16x2(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xFFFF0000u));
+            const uint32_t ph0 = movmatrix_trans(h01), ph1 = movmatrix_trans(h23);
+            const uint32_t pl0 = movmatrix_trans(l01), pl1 = movmatrix_trans(l23);
+            {
+                const uint32_t ones[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};
+                mma_bf16_acc(lacc, ones, ph0, ph1);
+                mma_bf16_acc(lacc, ones, pl0, pl1);
+            }
+            // P.V: channels on M, tokens on K; one 16-byte word per lane is one operand fragment
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const uint4 &klo = km[(j >> 2) * 2], &khi = km[(j >> 2) * 2 + 1];
-                const uint32_t wl = (j & 3) == 0 ? klo.x : (j & 3) == 1 ? klo.y : (j & 3) == 2 ? klo.z : klo.w;
-                const uint32_t wh = (j & 3) == 0 ? khi.x : (j & 3) == 1 ? khi.y : (j & 3) == 2 ? khi.z : khi.w;
-                uint32_t af[4];
-                af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
-                af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
-                af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
-                af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
-                float d[4];
-                mma_f16(d, af, qf[j][0], qf[j][1], zero4);
-                sc[0] = fmaf(d[0], ks[j], sc[0]);
-                sc[1] = fmaf(d[1], ks[j], sc[1]);
-                sc[2] = fmaf(d[2], ks[8 + j], sc[2]);
-                sc[3] = fmaf(d[3], ks[8 + j], sc[3]);
+                const uint32_t af[4] = {vm[j].x, vm[j].y, vm[j].z, vm[j].w};
+                mma_bf16_acc(o[j], af, ph0, ph1);
+                mma_bf16_acc(o[j], af, pl0, pl1);
             }
         }
-        // the V element words go to registers now, so that the ring slot can be re-armed for the record
-        // three ahead while softmax and P.V run
-        uint4 vm[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) vm[c] = lds128(sp + kBfp8Half + 128 + c * 512 + lane * 16);
-        __syncwarp();
-        if (k + kDepth < Rw) {
-            if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads above, bulk write below
-            issue();
-        }
-        float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
-        if (nvalid < kPageTokens) {
-            if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
-            if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
-        }
-        // ================= online softmax (log2 domain) =================
-        // The warp-wide maximum is only formed when some score exceeds the running maximum.
-        if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
-            float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
-#pragma unroll
-            for (int d = 4; d <= 16; d <<= 1) {
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
-            }
-            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-            const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
-            m0 = mn0;
-            m1 = mn1;
-            lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
-        }
-        // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
-        const uint32_t pb0 = movmatrix_trans(pack_half2(ex2f(s0 - m0), ex2f(s1 - m1)));   // tokens 2*t4, 2*t4+1 of head gq
-        const uint32_t pb1 = movmatrix_trans(pack_half2(ex2f(s2 - m0), ex2f(s3 - m1)));   // tokens 2*t4+8, 2*t4+9
-        {
-            const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
-            mma_f16_acc(lacc, ones, pb0, pb1);
-        }
-        // ================= P.V =================
-        {
-            uint4 vs[4];           // (f01, f89) of blocks 2c, 2c+1
-#pragma unroll
-            for (int c = 0; c < 4; ++c) vs[c] = lds128(scrV + c * 64 + t4 * 16);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint4 &vv = vm[j >> 1];
-                const uint32_t wl = (j & 1) ? vv.z : vv.x, wh = (j & 1) ? vv.w : vv.y;   // channels gq, gq+8 of block j
-                uint32_t af[4];
-                af[0] = prmt(wl, 0u, 0x1100u) & 0x807F807Fu;
-                af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
-                af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
-                af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
-                const uint32_t f01 = (j & 1) ? vs[j >> 1].z : vs[j >> 1].x, f89 = (j & 1) ? vs[j >> 1].w : vs[j >> 1].y;
-                mma_f16_acc(o[j], af, hmul2_u32(pb0, f01), hmul2_u32(pb1, f89));
-            }
-        }
-        __syncwarp();      // every lane is done with the scratch tables
     }
     if (alive) finish_segment();
     else if (lane == 0 && kMode < 2) {
@@ -572,7 +678,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bfp8_kernel(const AttnArgs a
 // One CTA per (sequence, kv head), one warp per q head, four channels per lane.  Segments that a single worker
 // held entirely were written by the main kernel.  Lane i of a chunk holds (m, l) of part i, so the weights of up
 // to 32 parts come from one round of loads; the 128-vectors are then fetched four parts at a time.
-__global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int n_ctas)
+__global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int max_workers)
 {
     asm volatile("griddepcontrol.wait;" ::: "memory");           // the main kernel's tiles are complete and visible
     const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
@@ -581,7 +687,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int n
     const int np = a.cum[b + 1] - a.cum[b];
     if (np == 0) return;                                         // rows of empty sequences were zeroed by the main kernel
     const int64_t W = (int64_t)Hkv * a.cum[a.batch];
-    const int64_t NWK = max((int64_t)1, min((int64_t)n_ctas * kWarps, W / kMinRecords));
+    const int64_t NWK = max((int64_t)1, min((int64_t)max_workers, W / kMinRecords));
     const int64_t ws = (int64_t)Hkv * a.cum[b] + (int64_t)g * np, we = ws + np;
     const int64_t u0 = ((ws + 1) * NWK - 1) / W, u1 = (we * NWK - 1) / W;     // first and last worker of the segment
     if (u0 == u1) return;
@@ -661,9 +767,11 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int n
     }
 }
 
+template <int kFmt>
 static size_t attn_smem_bytes(int batch)
 {
-    return (size_t)kStages * kBfp8Record + (size_t)kWarps * kScratch + kStages * 8 + kStages * 4 + (16 + kThreads) * 4 +
+    using G = Geo<kFmt>;
+    return (size_t)G::stages * G::record + (size_t)G::warps * G::scratch + G::stages * 8 + G::stages * 4 + (16 + G::threads) * 4 +
            ((size_t)batch + 1) * 4;
 }
 
@@ -690,12 +798,8 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)workspace & 255u)) return HMA_ERR_ALIGNMENT;
     if (batch > hma::kMaxBatch || max_pages_per_seq > (1 << 26)) return HMA_ERR_UNSUPPORTED_SHAPE;
     if (workspace_bytes < hma_decode_attention_workspace_bytes(&cache->desc, batch)) return HMA_ERR_WORKSPACE_TOO_SMALL;
-    if (cache->desc.format != HMA_KV_BFP8 && probe) return HMA_ERR_UNSUPPORTED_SHAPE;
-    if (cache->desc.format != HMA_KV_BFP8) {
-        // BF16 caches are served by the plain kernel until the tensor-core BF16 variant lands
-        return hma_decode_attention_simple(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens,
-                                           batch, sm_scale, stream);
-    }
+    const bool bf16 = cache->desc.format != HMA_KV_BFP8;
+    if (bf16 && probe == 2) return HMA_ERR_UNSUPPORTED_SHAPE;
     static int n_sm = 0;
     static bool attr_set = false;
     if (!n_sm) {
@@ -703,11 +807,13 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
         HMA_CUDA_OK(cudaGetDevice(&dev));
         HMA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     }
-    const size_t smem = hma::attn_smem_bytes(batch);
+    const size_t smem = bf16 ? hma::attn_smem_bytes<HMA_KV_BF16>(batch) : hma::attn_smem_bytes<HMA_KV_BFP8>(batch);
     if (!attr_set) {
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_bfp8_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_bfp8_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_bfp8_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<2, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     if (smem > 227 * 1024) return HMA_ERR_UNSUPPORTED_SHAPE;
@@ -726,9 +832,12 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.tiles = (float *)((uint8_t *)workspace + hma::cum_bytes(batch));
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
-    if (probe == 0) hma::attn_bfp8_kernel<0><<<n_ctas, hma::kThreads, smem, s>>>(a);
-    else if (probe == 1) hma::attn_bfp8_kernel<1><<<n_ctas, hma::kThreads, smem, s>>>(a);
-    else hma::attn_bfp8_kernel<2><<<n_ctas, hma::kThreads, smem, s>>>(a);
+    constexpr int tb = hma::Geo<HMA_KV_BFP8>::threads, tf = hma::Geo<HMA_KV_BF16>::threads;
+    if (bf16 && probe == 0) hma::attn_kernel<0, HMA_KV_BF16><<<n_ctas, tf, smem, s>>>(a);
+    else if (bf16) hma::attn_kernel<1, HMA_KV_BF16><<<n_ctas, tf, smem, s>>>(a);
+    else if (probe == 0) hma::attn_kernel<0, HMA_KV_BFP8><<<n_ctas, tb, smem, s>>>(a);
+    else if (probe == 1) hma::attn_kernel<1, HMA_KV_BFP8><<<n_ctas, tb, smem, s>>>(a);
+    else hma::attn_kernel<2, HMA_KV_BFP8><<<n_ctas, tb, smem, s>>>(a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     if (probe) return HMA_OK;
@@ -743,7 +852,8 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_kernel, a, n_ctas));
+    HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_kernel, a,
+                                   n_ctas * (bf16 ? hma::Geo<HMA_KV_BF16>::warps : hma::Geo<HMA_KV_BFP8>::warps)));
     hma::count_launch();
     return HMA_OK;
 }

@@ -55,6 +55,21 @@ def test_simple_kernel_and_bf16_cache_agree_with_oracle():
             check_attention(sc.attention(0, torch.float32).cpu().numpy(), bf16_bits(sc.attention(0, torch.bfloat16)), ref64)
 
 
+@pytest.mark.parametrize("hq,hkv", [(64, 8), (40, 8), (8, 8), (4, 1)])
+def test_bf16_cache_tensor_core_path(hq, hkv):
+    """The same values in a BF16 cache (filled by the decoding ingest) through the BF16 variant of the fused kernel."""
+    lens = [1, 15, 16, 17, 33, 0, 700, 48, 5000]
+    sc = Scenario(lens, hq, hkv, seed=hq + 3 * hkv, permute=True, fmt=hma.HMA_KV_BF16, fill=0xFF)
+    _, ref64, o32, o16 = _run_and_check(sc)
+    assert not o32[5].any()
+    again = bf16_bits(sc.attention(0, torch.bfloat16))
+    assert np.array_equal(again, o16)
+    twin = Scenario(lens, hq, hkv, seed=hq + 3 * hkv, permute=True, fmt=hma.HMA_KV_BFP8)
+    t32 = twin.attention(0, torch.float32).cpu().numpy()
+    assert np.abs(t32 - o32).max() <= 5e-3           # BFP8 path and BF16 path see identical values
+    assert hma.hma_error_flags(sc.cache) == 0
+
+
 def test_long_context_many_splits_and_determinism():
     """One long sequence is cut across every CTA (split-K), short ones sit inside a single CTA."""
     lens = [6000, 40, 2500, 16]
