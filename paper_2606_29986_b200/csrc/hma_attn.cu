@@ -39,7 +39,8 @@ struct Geo {
     static constexpr int scratch = kFmt == HMA_KV_BFP8 ? kScratch : 0;
 };
 constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile: o[8][128], m[8], l[8]
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 20;           // polls of a bounded wait
+constexpr uint32_t kSuspendNs = 2000;              // a failed poll may keep the thread parked this long
 constexpr int kMaxBatch = 2048;
 constexpr int kMaxCtas = 160;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
 constexpr int kMinRecords = 8;                    // fewest records a worker takes
@@ -77,10 +78,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendNs)
         : "memory");
     return ok != 0;
 }
@@ -287,46 +288,52 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         page = (int)(off - (int64_t)g * np);
     }
 
-    // ---- the warp's own feed: issue cursor, window of block-table entries, three ring slots ----
+    // ---- the warp's own feed: three ring slots; record addresses are worked out 32 at a time, one per lane ----
     const uint32_t full0 = smem_u32(bars + warp * kDepth);
     const uint32_t ring0 = smem_u32(ring + warp * kDepth * kRecord);
-    int ib = b, ig = g, ip = page, inp = np;      // cursor of the next record to request
-    int iwb = -1, iw0 = 0;                        // the window holds pages [iw0, iw0+32) of sequence iwb
-    int32_t ipid = -1;
+    constexpr uint32_t kNoRecord = 0xFFFFFFFFu;
+    uint32_t roff = kNoRecord;                    // this lane's record of the current window, in units of 128 bytes
+    int kwin = 0;                                 // the window covers records [kwin, kwin + 32) of this warp
+    int kissue = 0;                               // next record to request
     int islot = 0;
     uint64_t policy;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    auto refill = [&]() {
+        // lane i resolves record kwin + i: sequence by binary search over the page prefix, then head and page
+        roff = kNoRecord;
+        const int kk = kwin + lane;
+        if (kk < Rw) {
+            const int64_t wr = wlo + kk;
+            int lo = 0, hi = B - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if ((int64_t)Hkv * cum[mid] <= wr) lo = mid; else hi = mid - 1;
+            }
+            const int npb = cum[lo + 1] - cum[lo];
+            const int off = (int)(wr - (int64_t)Hkv * cum[lo]);
+            const int gg = off / npb, pp = off - gg * npb;
+            const int32_t pid = a.block_table[(int64_t)lo * a.max_pages + pp];
+            if (pid >= 0 && pid < a.cv.num_pages) roff = (uint32_t)(((int64_t)pid * Hkv + gg) * (kRecord / 128));
+        }
+    };
     auto issue = [&]() {
         if (kMode == 2) return;
-        if (iwb != ib || ip < iw0 || ip >= iw0 + 32) {
-            iwb = ib;
-            iw0 = ip;
-            ipid = ip + lane < inp ? a.block_table[(int64_t)ib * a.max_pages + ip + lane] : -1;
-        }
-        const int32_t pid = __shfl_sync(0xFFFFFFFFu, ipid, ip - iw0);
+        const uint32_t off = __shfl_sync(0xFFFFFFFFu, roff, kissue - kwin);
         if (lane == 0) {
-            const int s = warp * kDepth + islot;
-            if (pid >= 0 && pid < a.cv.num_pages) {
-                stage_ok[s] = 1;
+            if (off != kNoRecord) {
+                stage_ok[warp * kDepth + islot] = 1;
                 mbar_arrive_expect_tx(full0 + 8 * islot, kRecord);
-                bulk_load(ring0 + islot * kRecord, a.cv.layer + ((int64_t)pid * Hkv + ig) * kRecord, kRecord,
-                          full0 + 8 * islot, policy);
+                bulk_load(ring0 + islot * kRecord, a.cv.layer + (uint64_t)off * 128u, kRecord, full0 + 8 * islot, policy);
             } else {
-                stage_ok[s] = 0;
+                stage_ok[warp * kDepth + islot] = 0;
                 atomicOr(a.cv.flags, HMA_FLAG_BAD_PAGE_ATTENTION);
                 mbar_arrive(full0 + 8 * islot);
             }
         }
         if (++islot == kDepth) islot = 0;
-        if (++ip == inp) {
-            ip = 0;
-            if (++ig == Hkv) {
-                ig = 0;
-                do { ++ib; } while (ib < B && cum[ib + 1] == cum[ib]);
-                if (ib < B) inp = cum[ib + 1] - cum[ib];
-            }
-        }
+        if (++kissue == kwin + 32 && kissue < Rw) { kwin = kissue; refill(); }
     };
+    if (kMode != 2) refill();
     for (int k = 0; k < kDepth && k < Rw; ++k) issue();
 
     // ---- consumer state ----
