@@ -124,6 +124,16 @@ hma_status_t hma_kv_ingest_layer(hma_cache_t *cache, int32_t layer,
                                  const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
                                  void *stream);
 
+/* The same for several producer shards in one launch (section 3.3: "merges the per-chip KV shards"; Table 2
+ * runs Qwen3-32B prefill as one TP=4 group, so a layer arrives as four head ranges).  k_wires, v_wires,
+ * head_begins, head_counts are host arrays of n_shards (1..8) entries; shard i carries heads
+ * [head_begins[i], head_begins[i]+head_counts[i]) in the wire layout described above; head ranges must not
+ * overlap.  Everything else as hma_kv_ingest_layer. */
+hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32_t n_shards,
+                                        const void *const *k_wires, const void *const *v_wires, int32_t wire_layout,
+                                        const int32_t *head_begins, const int32_t *head_counts,
+                                        const int32_t *page_ids, int64_t token_begin, int64_t n_tokens, void *stream);
+
 /*
  * Decode attention over block tables (section 3.3; one query token per sequence, section 1).
  * For sequence b, q head h, kv head g = h / (num_q_heads/num_kv_heads), T = context_lens[b]:

@@ -6,11 +6,14 @@
 
 namespace hma {
 
+constexpr int kMaxShards = 8;
 struct IngestArgs {
-    const uint8_t *k_wire, *v_wire;
+    const uint8_t *k_wire[kMaxShards], *v_wire[kMaxShards];   // per producer shard
+    int32_t head_begin[kMaxShards], head_count[kMaxShards];
+    int32_t n_shards;
     const int32_t *page_ids;
     int64_t token_begin, n_tokens;
-    int32_t layout, head_begin, head_count;
+    int32_t layout;
 };
 
 // Address of the 16 element bytes of block j of wire token wt of shard head hs, and of its exponent byte.
@@ -36,8 +39,10 @@ __device__ __forceinline__ int64_t wire_block_off(int layout, int64_t n_tokens, 
 __global__ void __launch_bounds__(256) ingest_kernel(CacheView cv, IngestArgs a)
 {
     __shared__ __align__(16) uint8_t rows[2][kPageTokens][kRowBytes + 8];   // +8 keeps element bytes 16-byte aligned
-    const int hs = blockIdx.y;
-    const int h = a.head_begin + hs;
+    // blockIdx.y runs over the heads of all shards in turn
+    int shard = 0, hs = blockIdx.y;
+    while (shard + 1 < a.n_shards && hs >= a.head_count[shard]) hs -= a.head_count[shard++];
+    const int h = a.head_begin[shard] + hs;
     const int64_t lp = a.token_begin / kPageTokens + blockIdx.x;            // logical page of the request
     const int32_t pid = a.page_ids[blockIdx.x];
     if (pid < 0 || pid >= cv.num_pages) {
@@ -52,7 +57,7 @@ __global__ void __launch_bounds__(256) ingest_kernel(CacheView cv, IngestArgs a)
     for (int item = threadIdx.x; item < 2 * kPageTokens * kBlocksPerRow; item += blockDim.x) {
         const int t = item >> 7 & 1, tok = (item >> 3) & 15, j = item & 7;
         if (tok < lo || tok >= hi) continue;
-        const uint8_t *w = t ? a.v_wire : a.k_wire;
+        const uint8_t *w = t ? a.v_wire[shard] : a.k_wire[shard];
         int64_t eo;
         const int64_t mo = wire_block_off(a.layout, a.n_tokens, hs, lp * kPageTokens + tok - a.token_begin, j, &eo);
         uint8_t *dst = &rows[t][tok][8 + 8 + j * kBlock];                    // elements start at byte 16 of the padded row
@@ -130,28 +135,67 @@ __global__ void __launch_bounds__(256) ingest_kernel(CacheView cv, IngestArgs a)
 
 }  // namespace hma
 
-extern "C" hma_status_t hma_kv_ingest_layer(hma_cache_t *cache, int32_t layer, const void *k_wire, const void *v_wire,
-                                            int32_t wire_layout, int32_t head_begin, int32_t head_count,
-                                            const int32_t *page_ids, int64_t token_begin, int64_t n_tokens, void *stream)
+static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_shards, const void *const *k_wires,
+                                  const void *const *v_wires, int32_t wire_layout, const int32_t *head_begins,
+                                  const int32_t *head_counts, const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
+                                  void *stream)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers) return HMA_ERR_INVALID_ARG;
     if (wire_layout != HMA_WIRE_TILE32 && wire_layout != HMA_WIRE_ROWMAJOR) return HMA_ERR_INVALID_ARG;
-    if (head_begin < 0 || head_count <= 0 || head_begin + head_count > cache->desc.num_kv_heads) return HMA_ERR_INVALID_ARG;
+    if (n_shards < 1 || n_shards > hma::kMaxShards || !k_wires || !v_wires || !head_begins || !head_counts) return HMA_ERR_INVALID_ARG;
     if (token_begin < 0 || n_tokens < 0) return HMA_ERR_INVALID_ARG;
+    hma::IngestArgs a = {};
+    int heads = 0;
+    unsigned seen = 0;
+    for (int s = 0; s < n_shards; ++s) {
+        if (head_begins[s] < 0 || head_counts[s] <= 0 || head_begins[s] + head_counts[s] > cache->desc.num_kv_heads) return HMA_ERR_INVALID_ARG;
+        for (int h = head_begins[s]; h < head_begins[s] + head_counts[s]; ++h) {
+            if (seen & (1u << (h & 31))) return HMA_ERR_INVALID_ARG;     // two shards may not write the same head
+            seen |= 1u << (h & 31);
+        }
+        a.k_wire[s] = (const uint8_t *)k_wires[s];
+        a.v_wire[s] = (const uint8_t *)v_wires[s];
+        a.head_begin[s] = head_begins[s];
+        a.head_count[s] = head_counts[s];
+        heads += head_counts[s];
+    }
     if (n_tokens == 0) return HMA_OK;
-    if (!k_wire || !v_wire || !page_ids) return HMA_ERR_INVALID_ARG;
-    if (((uintptr_t)k_wire & 15u) || ((uintptr_t)v_wire & 15u)) return HMA_ERR_ALIGNMENT;
+    if (!page_ids) return HMA_ERR_INVALID_ARG;
+    for (int s = 0; s < n_shards; ++s) {
+        if (!a.k_wire[s] || !a.v_wire[s]) return HMA_ERR_INVALID_ARG;
+        if (((uintptr_t)a.k_wire[s] & 15u) || ((uintptr_t)a.v_wire[s] & 15u)) return HMA_ERR_ALIGNMENT;
+    }
     const int64_t first = token_begin / hma::kPageTokens;
     const int64_t last = (token_begin + n_tokens - 1) / hma::kPageTokens;
     const int64_t n_pages = last - first + 1;
     if (n_pages > 0x7FFFFFFF) return HMA_ERR_INVALID_ARG;
     hma::CacheView cv{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
                       cache->desc.num_q_heads, cache->desc.format, cache->flags};
-    hma::IngestArgs a{(const uint8_t *)k_wire, (const uint8_t *)v_wire, page_ids, token_begin, n_tokens,
-                      wire_layout, head_begin, head_count};
-    dim3 grid((unsigned)n_pages, (unsigned)head_count);
+    a.n_shards = n_shards;
+    a.page_ids = page_ids;
+    a.token_begin = token_begin;
+    a.n_tokens = n_tokens;
+    a.layout = wire_layout;
+    dim3 grid((unsigned)n_pages, (unsigned)heads);
     hma::ingest_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(cv, a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;
+}
+
+extern "C" hma_status_t hma_kv_ingest_layer(hma_cache_t *cache, int32_t layer, const void *k_wire, const void *v_wire,
+                                            int32_t wire_layout, int32_t head_begin, int32_t head_count,
+                                            const int32_t *page_ids, int64_t token_begin, int64_t n_tokens, void *stream)
+{
+    return launch_ingest(cache, layer, 1, &k_wire, &v_wire, wire_layout, &head_begin, &head_count, page_ids, token_begin,
+                         n_tokens, stream);
+}
+
+extern "C" hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32_t n_shards,
+                                                   const void *const *k_wires, const void *const *v_wires,
+                                                   int32_t wire_layout, const int32_t *head_begins, const int32_t *head_counts,
+                                                   const int32_t *page_ids, int64_t token_begin, int64_t n_tokens, void *stream)
+{
+    return launch_ingest(cache, layer, n_shards, k_wires, v_wires, wire_layout, head_begins, head_counts, page_ids,
+                         token_begin, n_tokens, stream);
 }

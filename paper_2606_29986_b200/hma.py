@@ -56,6 +56,9 @@ def lib():
         L.hma_cache_destroy.argtypes = [vp]
         L.hma_kv_ingest_layer.restype = i32
         L.hma_kv_ingest_layer.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, i64, i64, vp]
+        L.hma_kv_ingest_layer_shards.restype = i32
+        L.hma_kv_ingest_layer_shards.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), i32,
+                                                 ctypes.POINTER(i32), ctypes.POINTER(i32), vp, i64, i64, vp]
         L.hma_decode_attention_workspace_bytes.restype = sz
         L.hma_decode_attention_workspace_bytes.argtypes = [ctypes.POINTER(CacheDesc), i32]
         L.hma_decode_attention.restype = i32
@@ -149,6 +152,18 @@ def hma_kv_ingest_layer(cache, layer, k_wire, v_wire, wire_layout, head_begin, h
     _check(lib().hma_kv_ingest_layer(cache.handle, layer, _ptr(k_wire), _ptr(v_wire), wire_layout, head_begin,
                                      head_count, _ptr(page_ids), token_begin, n_tokens, _stream(stream)),
            "hma_kv_ingest_layer")
+
+
+def hma_kv_ingest_layer_shards(cache, layer, k_wires, v_wires, wire_layout, head_begins, head_counts, page_ids,
+                               token_begin, n_tokens, stream=None):
+    """All producer shards of one layer in one launch; k_wires / v_wires are lists of tensors, one per shard."""
+    n = len(k_wires)
+    kp = (ctypes.c_void_p * n)(*[t.data_ptr() for t in k_wires])
+    vp_ = (ctypes.c_void_p * n)(*[t.data_ptr() for t in v_wires])
+    hb = (ctypes.c_int32 * n)(*head_begins)
+    hc = (ctypes.c_int32 * n)(*head_counts)
+    _check(lib().hma_kv_ingest_layer_shards(cache.handle, layer, n, kp, vp_, wire_layout, hb, hc, _ptr(page_ids),
+                                            token_begin, n_tokens, _stream(stream)), "hma_kv_ingest_layer_shards")
 
 
 def hma_decode_attention_workspace_bytes(desc, batch):

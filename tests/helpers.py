@@ -17,7 +17,7 @@ class Scenario:
     """A batch of sequences with seeded BFP8 wire bytes, ingested into a paged cache on the GPU."""
 
     def __init__(self, lens, hq, hkv, seed=0, permute=False, fmt=hma.HMA_KV_BFP8, wire_layout=hma.HMA_WIRE_ROWMAJOR,
-                 shards=1, layers=1, extra_pages=3, fill=0xA5, device="cuda"):
+                 shards=1, layers=1, extra_pages=3, fill=0xA5, device="cuda", one_launch=False):
         self.lens = np.asarray(lens, np.int32)
         self.B, self.hq, self.hkv, self.layers = len(lens), hq, hkv, layers
         self.seed = seed
@@ -39,11 +39,18 @@ class Scenario:
                     continue
                 pages = self.table[b, :(T + 15) // 16].contiguous()
                 hs = hkv // shards
+                kss, vss = [], []
                 for s in range(shards):
                     ks, vs = kw[s * hs:(s + 1) * hs].contiguous(), vw[s * hs:(s + 1) * hs].contiguous()
                     if wire_layout == hma.HMA_WIRE_TILE32:
                         ks, vs = synth.rowmajor_to_tile32(ks), synth.rowmajor_to_tile32(vs)
-                    hma.hma_kv_ingest_layer(self.cache, l, ks.to(device), vs.to(device), wire_layout, s * hs, hs, pages, 0, T)
+                    kss.append(ks.to(device))
+                    vss.append(vs.to(device))
+                    if not one_launch:
+                        hma.hma_kv_ingest_layer(self.cache, l, kss[-1], vss[-1], wire_layout, s * hs, hs, pages, 0, T)
+                if one_launch:      # every shard of the layer in a single call
+                    hma.hma_kv_ingest_layer_shards(self.cache, l, kss, vss, wire_layout, [s * hs for s in range(shards)],
+                                                   [hs] * shards, pages, 0, T)
         torch.cuda.synchronize()
         ws = hma.hma_decode_attention_workspace_bytes(self.desc, self.B)
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=device)

@@ -89,6 +89,18 @@ def test_partial_range_ingest_keeps_other_bytes(fmt, layout):
     assert np.array_equal(bf16_bits(out).transpose(1, 0, 2), orc.decode_rowmajor_bf16(new_v.numpy()))
 
 
+@pytest.mark.parametrize("layout", [hma.HMA_WIRE_ROWMAJOR, hma.HMA_WIRE_TILE32])
+def test_all_shards_in_one_launch_equal_shard_by_shard(layout):
+    lens = [33, 100, 16, 1]
+    a = Scenario(lens, 32, 8, seed=9, permute=True, wire_layout=layout, shards=4, fill=0x11)
+    b = Scenario(lens, 32, 8, seed=9, permute=True, wire_layout=layout, shards=4, fill=0x11, one_launch=True)
+    assert torch.equal(a.cache.layers[0], b.cache.layers[0])
+    kw = torch.from_numpy(a.k_wires[0][0][:2]).cuda()
+    with pytest.raises(hma.HmaError) as e:       # overlapping head ranges are refused
+        hma.hma_kv_ingest_layer_shards(a.cache, 0, [kw, kw], [kw, kw], hma.HMA_WIRE_ROWMAJOR, [0, 1], [2, 2], a.table[0, :3].contiguous(), 0, 33)
+    assert e.value.status == hma.HMA_ERR_INVALID_ARG
+
+
 def test_bfp8_cache_holds_the_wire_bytes_unchanged():
     """Ingest permutes positions only: the multiset of bytes of a fully written page equals that of its wire rows."""
     sc = Scenario([32], 8, 2, seed=6, layers=1, extra_pages=0)
