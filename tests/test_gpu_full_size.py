@@ -1,0 +1,58 @@
+"""Sampled parity at the full sizes of the benchmark workloads, in the launch configuration bench.py times.
+
+One layer of each workload is built exactly as the benchmark builds it (GPU-generated values, real block tables,
+permuted pages where the workload says so); the outputs of the shortest, longest, first and last sequence are
+compared with the oracle run on the wire bytes copied back from the device."""
+import os
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["qwen3-8b-b64-ctx4k", "qwen3-14b-b128-lognormal", "qwen3-32b-b32-ctx8k", "qwen3-32b-b256-trace"])
+def test_sampled_parity_full_batch(name):
+    import bench
+    from paper_2606_29986_b200 import hma
+    wl = bench.Workload(name, torch.device("cuda", 0), with_bf16=False, with_ingest=False, layers=1)
+    res = wl.parity_sample()
+    assert len(res) >= 2
+    for r in res:
+        assert r["f32_max_abs"] <= 1e-2 and r["f32_rel_l2"] <= 2e-3, (name, r)      # the bar, literally, on the F32 output
+        assert r["bf16_is_rne_of_f32"], (name, r)                                     # BF16 output = exact rounding of it
+        assert r["bf16_max_abs"] <= 1e-2 + 2.0 ** -8 * 25.0, (name, r)
+    assert hma.hma_error_flags(wl.caches["bfp8"]) == 0
+    # the read probe moves the same records without touching the outputs
+    before = wl.out.clone()
+    hma.hma_kv_read_probe(wl.caches["bfp8"], 0, wl.table, wl.ctx, wl.workspace)
+    torch.cuda.synchronize()
+    assert torch.equal(before, wl.out)
+
+
+def test_longest_supported_context_and_limits():
+    from paper_2606_29986_b200 import hma
+    from helpers import Scenario, check_attention, bf16_bits
+    sc = Scenario([32768, 17], 64, 8, seed=77, permute=True)
+    ref64, _ = sc.oracle()
+    check_attention(sc.attention(0, torch.float32).cpu().numpy(), bf16_bits(sc.attention(0, torch.bfloat16)), ref64)
+    # a batch beyond the kernel's limit is refused, not mis-run
+    big = 5000
+    q = torch.zeros((big, 64, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(q)
+    tbl = torch.zeros((big, 1), dtype=torch.int32, device="cuda")
+    ctx = torch.zeros(big, dtype=torch.int32, device="cuda")
+    ws = torch.empty(hma.hma_decode_attention_workspace_bytes(sc.desc, big), dtype=torch.uint8, device="cuda")
+    with pytest.raises(hma.HmaError) as e:
+        hma.hma_decode_attention(sc.cache, 0, q, out, tbl, ctx, 0.1, ws)
+    assert e.value.status == hma.HMA_ERR_UNSUPPORTED_SHAPE
+    # 2048 empty sequences are fine: every row is zero
+    q2, out2 = q[:2048], torch.ones((2048, 64, 128), dtype=torch.bfloat16, device="cuda")
+    hma.hma_decode_attention(sc.cache, 0, q2, out2, tbl[:2048], ctx[:2048], 0.1, ws)
+    torch.cuda.synchronize()
+    assert not out2.any()
