@@ -30,9 +30,9 @@ from paper_2606_29986_b200 import synth  # noqa: E402
 DEFAULT_WORKLOAD = "qwen3-32b-b32-ctx8k"
 BFP8_ROW = 272      # bytes per (token, kv head): K 136 + V 136
 BF16_ROW = 512
-# DRAM bytes per launch of attn_bfp8_kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
+# DRAM bytes per launch of the attention kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
 # see profiles/.  Keyed by workload; None where no capture exists.
-NCU_TRAFFIC_BYTES = {"qwen3-32b-b32-ctx8k": 575_200_000}    # profiles/attn_bfp8_kernel_qwen3-32b-b32-ctx8k_ncu_full.md
+NCU_TRAFFIC_BYTES = {"qwen3-32b-b32-ctx8k": 575_400_000}    # profiles/attn_kernel_bfp8_qwen3-32b-b32-ctx8k_ncu_full.md
 
 
 def measured_peak():
@@ -422,7 +422,7 @@ def main():
                      "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                      "probe_gbs": wl.kv_bytes_per_layer("bfp8") / probe_mean / 1e9,
                      "frac_of_probe": probe_mean / call_mean,
-                     "kernel": "hma_decode_attention (attn_bfp8_kernel + attn_merge_kernel)",
+                     "kernel": "hma_decode_attention (attn_kernel<0,0> + attn_merge_kernel)",
                      "bytes_per_launch": wl.kv_bytes_per_layer("bfp8"), "us_per_launch_mean": call_mean * 1e6,
                      "us_per_launch_median": call_med * 1e6, "us_per_launch_min": call_min * 1e6},
         "decode_only": {"tokens_per_s": aggregate_value(wl.B, sec_decode_only, ws), "ms_per_step": sec_decode_only * 1e3,
