@@ -53,6 +53,12 @@ typedef enum {
 typedef enum { HMA_KV_BFP8 = 0, HMA_KV_BF16 = 1 } hma_kv_format_t;
 typedef enum { HMA_WIRE_TILE32 = 0, HMA_WIRE_ROWMAJOR = 1 } hma_wire_layout_t;
 typedef enum { HMA_OUT_BF16 = 0, HMA_OUT_F32 = 1 } hma_out_dtype_t;
+/* Head-dim order of the cached keys relative to the queries (section 3.3: the prefill accelerator writes post-RoPE
+ * keys with rotary pairs interleaved, (2i, 2i+1); FlashAttention-style decoders use the half-split order, (i, i+64)).
+ * HMA_KEYS_AS_QUERIES: cached keys are in the queries' order.  HMA_KEYS_INTERLEAVED: cached key channel c is the
+ * half-split channel (c >> 1) + 64 * (c & 1); queries (and the output of hma_bfp8_dequant_bf16 for K) are half-split.
+ * Values carry no rotary embedding and are never re-ordered. */
+typedef enum { HMA_KEYS_AS_QUERIES = 0, HMA_KEYS_INTERLEAVED = 1 } hma_key_layout_t;
 
 /* bits of the device flag word (hma_error_flags) */
 #define HMA_FLAG_BAD_PAGE_ATTENTION 1u  /* block table entry outside [0, num_pages): page skipped */
@@ -69,6 +75,7 @@ typedef struct {
     int32_t bfp_block;     /* must be 16  */
     int64_t num_pages;     /* physical pages per layer */
     int32_t format;        /* hma_kv_format_t */
+    int32_t key_layout;    /* hma_key_layout_t */
 } hma_cache_desc_t;
 
 typedef struct hma_cache hma_cache_t;   /* opaque; host-side metadata only */

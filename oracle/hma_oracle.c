@@ -199,9 +199,15 @@ void orc_unpack_tile32(const uint8_t *tiles, int64_t n_tokens, int32_t heads, ui
  *   out_bf16 [B][Hq][128]   the same rounded to BF16 by RNE (may be NULL)
  *   probs    if not NULL: fp64 softmax weights of sequence 0, head 0 (ctx_lens[0] values); for tests
  * T = 0 gives a row of zeros. */
+/* Position, in the half-split head-dim order (rotary pairs (i, i+64)), of channel c of the interleaved order
+ * (rotary pairs (2i, 2i+1)): the key re-layout of section 3.3. */
+int32_t orc_half_split_index(int32_t c) { return (c >> 1) + 64 * (c & 1); }
+
+/* keys_interleaved != 0: the wire keys are in interleaved rotary order while the queries are half-split, so key
+ * channel c meets query channel orc_half_split_index(c). */
 void orc_decode_attention(const uint16_t *q_bf16, const uint8_t *k_wire, const uint8_t *v_wire,
                           const int64_t *wire_off, const int32_t *ctx_lens,
-                          int32_t B, int32_t Hq, int32_t Hkv, double sm_scale,
+                          int32_t B, int32_t Hq, int32_t Hkv, double sm_scale, int32_t keys_interleaved,
                           double *out_f64, uint16_t *out_bf16, double *probs)
 {
     const int G = Hq / Hkv;
@@ -224,7 +230,7 @@ void orc_decode_attention(const uint16_t *q_bf16, const uint8_t *k_wire, const u
                     const uint8_t *row = kr + t * ORC_ROW_BYTES;
                     double acc = 0.0;
                     for (int d = 0; d < ORC_HEAD_DIM; ++d)
-                        acc += q[d] * bfp8_value(row[d / ORC_BLOCK], row[ORC_BLOCKS_PER_ROW + d]);
+                        acc += q[keys_interleaved ? orc_half_split_index(d) : d] * bfp8_value(row[d / ORC_BLOCK], row[ORC_BLOCKS_PER_ROW + d]);
                     s[t] = sm_scale * acc;
                     if (s[t] > smax) smax = s[t];
                 }

@@ -139,7 +139,7 @@ def unpack_tile32(tiles, n_tokens, heads):
     return out
 
 
-def decode_attention(q_bf16, k_wires, v_wires, num_kv_heads, sm_scale=None, want_probs=False):
+def decode_attention(q_bf16, k_wires, v_wires, num_kv_heads, sm_scale=None, want_probs=False, keys_interleaved=False):
     """fp64 decode attention over ROWMAJOR wire bytes.
 
     q_bf16  : uint16 [B][Hq][128] (BF16 bit patterns)
@@ -166,11 +166,26 @@ def decode_attention(q_bf16, k_wires, v_wires, num_kv_heads, sm_scale=None, want
     probs = np.zeros(max(int(lens[0]), 1), np.float64) if want_probs else None
     lib().orc_decode_attention(_p(q_bf16), _p(kcat), _p(vcat), _p(offs), _p(lens),
                                ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(num_kv_heads),
-                               ctypes.c_double(sm_scale), _p(out64), _p(out16),
+                               ctypes.c_double(sm_scale), ctypes.c_int32(1 if keys_interleaved else 0), _p(out64), _p(out16),
                                _p(probs) if want_probs else None)
     if want_probs:
         return out64, out16, probs[:int(lens[0])]
     return out64, out16
+
+
+def half_split_index(c):
+    """Half-split position of interleaved-order channel c (the key re-layout of section 3.3)."""
+    lib().orc_half_split_index.restype = ctypes.c_int32
+    return int(lib().orc_half_split_index(ctypes.c_int32(int(c))))
+
+
+def relayout_keys_to_half_split(x):
+    """x[..., 128] in interleaved rotary order -> the same values in half-split order."""
+    x = np.asarray(x)
+    out = np.empty_like(x)
+    for c in range(HEAD_DIM):
+        out[..., half_split_index(c)] = x[..., c]
+    return out
 
 
 def num_threads():

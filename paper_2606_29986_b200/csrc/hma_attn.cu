@@ -359,10 +359,19 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         float f[8][4];
         float amax = 0.f;
         const bool hv = gq < G && kMode == 0;      // the probes have no Q: nothing is read through a.q
-        const uint16_t *qp = a.q + ((int64_t)b * Hq + (int64_t)g * G + (hv ? gq : 0)) * kHeadDim + 4 * t4;
+        const uint16_t *qrow = a.q + ((int64_t)b * Hq + (int64_t)g * G + (hv ? gq : 0)) * kHeadDim;
+        const bool inter = a.cv.key_layout == HMA_KEYS_INTERLEAVED;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            uint2 v = hv ? *reinterpret_cast<const uint2 *>(qp + 16 * j) : make_uint2(0u, 0u);
+            // this lane's cached key channels 16j + 4*t4 .. +3 meet the query channels of the same rotary pairs
+            uint2 v = make_uint2(0u, 0u);
+            if (hv && !inter) v = *reinterpret_cast<const uint2 *>(qrow + 16 * j + 4 * t4);
+            if (hv && inter) {
+                const uint32_t lo = *reinterpret_cast<const uint32_t *>(qrow + 8 * j + 2 * t4);        // q[a], q[a+1]
+                const uint32_t hi = *reinterpret_cast<const uint32_t *>(qrow + 8 * j + 2 * t4 + 64);   // q[a+64], q[a+65]
+                v.x = (lo & 0xFFFFu) | (hi << 16);            // key channels 4*t4, 4*t4+1  <- q[a], q[a+64]
+                v.y = (lo >> 16) | (hi & 0xFFFF0000u);        // key channels 4*t4+2, +3    <- q[a+1], q[a+65]
+            }
             f[j][0] = __uint_as_float(v.x << 16);
             f[j][1] = __uint_as_float(v.x & 0xFFFF0000u);
             f[j][2] = __uint_as_float(v.y << 16);
@@ -826,7 +835,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     if (smem > 227 * 1024) return HMA_ERR_UNSUPPORTED_SHAPE;
     hma::AttnArgs a;
     a.cv = hma::CacheView{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
-                          cache->desc.num_q_heads, cache->desc.format, cache->flags};
+                          cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
     a.q = (const uint16_t *)q;
     a.out = out;
     a.out_dtype = out_dtype;

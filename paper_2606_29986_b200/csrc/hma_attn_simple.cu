@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kSimpleWarps * 32) attn_simple_kernel(CacheVie
         for (int h = 0; h < G; ++h) {
             float s = 0.f;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) s = fmaf(sq[h][lane * 4 + k], kf[k], s);
+            for (int k = 0; k < 4; ++k) s = fmaf(sq[h][key_channel_of_query(lane * 4 + k, cv.key_layout)], kf[k], s);
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
             s *= sm_scale;
@@ -105,7 +105,7 @@ extern "C" hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, in
     if (!q || !out || !block_table || !context_lens) return HMA_ERR_INVALID_ARG;
     if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u)) return HMA_ERR_ALIGNMENT;
     hma::CacheView cv{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
-                      cache->desc.num_q_heads, cache->desc.format, cache->flags};
+                      cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
     dim3 grid((unsigned)batch, (unsigned)cache->desc.num_kv_heads);
     cudaStream_t s = (cudaStream_t)stream;
     const int G = cache->desc.num_q_heads / cache->desc.num_kv_heads;

@@ -21,6 +21,7 @@ static bool desc_ok(const hma_cache_desc_t *d)
     int g = d->num_q_heads / d->num_kv_heads;
     if (g < 1 || g > hma::kMaxGroup) return false;
     if (d->format != HMA_KV_BFP8 && d->format != HMA_KV_BF16) return false;
+    if (d->key_layout != HMA_KEYS_AS_QUERIES && d->key_layout != HMA_KEYS_INTERLEAVED) return false;
     return true;
 }
 

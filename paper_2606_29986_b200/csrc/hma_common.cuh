@@ -26,6 +26,7 @@ struct CacheView {
     int32_t num_q_heads;
     int32_t format;        // hma_kv_format_t
     uint32_t *flags;       // device flag word
+    int32_t key_layout;    // hma_key_layout_t
 };
 
 __host__ __device__ inline int record_bytes(int format) { return format == HMA_KV_BFP8 ? kBfp8Record : kBf16Record; }
@@ -75,6 +76,9 @@ __device__ __forceinline__ uint32_t bfp8_to_bf16_bits(uint32_t E, uint32_t b)
     else r = m << E;                       // BF16 subnormal: m * 2^E units of 2^-133
     return s | r;
 }
+
+// half-split position of cached key channel c when keys are cached with rotary pairs interleaved
+__host__ __device__ inline int key_channel_of_query(int c, int key_layout) { return key_layout == HMA_KEYS_INTERLEAVED ? (c >> 1) + 64 * (c & 1) : c; }
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
 

@@ -70,8 +70,17 @@ __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int wh
                 }
             }
         }
-        uint16_t *dst = out + ((gt - token_begin) * cv.num_kv_heads + h) * kHeadDim + c0;
-        *reinterpret_cast<uint4 *>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+        uint16_t *row = out + ((gt - token_begin) * cv.num_kv_heads + h) * kHeadDim;
+        if (which == 0 && cv.key_layout == HMA_KEYS_INTERLEAVED) {
+            // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout):
+            // cached channels c0, c0+2, .. go to c0/2 .., cached channels c0+1, c0+3, .. to 64 + c0/2 ..
+            const uint32_t e0 = (o[0] & 0xFFFFu) | (o[1] << 16), e1 = (o[2] & 0xFFFFu) | (o[3] << 16);
+            const uint32_t d0 = (o[0] >> 16) | (o[1] & 0xFFFF0000u), d1 = (o[2] >> 16) | (o[3] & 0xFFFF0000u);
+            *reinterpret_cast<uint2 *>(row + (c0 >> 1)) = make_uint2(e0, e1);
+            *reinterpret_cast<uint2 *>(row + 64 + (c0 >> 1)) = make_uint2(d0, d1);
+        } else {
+            *reinterpret_cast<uint4 *>(row + c0) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
     }
 }
 
@@ -106,7 +115,7 @@ extern "C" hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t 
     const int64_t n_pages = last - first + 1;
     if (n_pages > 0x7FFFFFFF) return HMA_ERR_INVALID_ARG;
     hma::CacheView cv{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
-                      cache->desc.num_q_heads, cache->desc.format, cache->flags};
+                      cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
     dim3 grid((unsigned)n_pages, (unsigned)cache->desc.num_kv_heads);
     hma::dequant_paged_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, which, page_ids, token_begin, n_tokens,
                                                                       (uint16_t *)out_bf16);

@@ -170,7 +170,7 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
     const int64_t n_pages = last - first + 1;
     if (n_pages > 0x7FFFFFFF) return HMA_ERR_INVALID_ARG;
     hma::CacheView cv{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
-                      cache->desc.num_q_heads, cache->desc.format, cache->flags};
+                      cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
     a.n_shards = n_shards;
     a.page_ids = page_ids;
     a.token_begin = token_begin;

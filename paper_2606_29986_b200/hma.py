@@ -19,13 +19,14 @@ HMA_ERR_STATIC_LIMIT = 7
 HMA_KV_BFP8, HMA_KV_BF16 = 0, 1
 HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR = 0, 1
 HMA_OUT_BF16, HMA_OUT_F32 = 0, 1
+HMA_KEYS_AS_QUERIES, HMA_KEYS_INTERLEAVED = 0, 1
 HMA_FLAG_BAD_PAGE_ATTENTION, HMA_FLAG_BAD_PAGE_INGEST, HMA_FLAG_BAD_PAGE_DEQUANT, HMA_FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
 
 
 class CacheDesc(ctypes.Structure):
     _fields_ = [("num_layers", ctypes.c_int32), ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("page_tokens", ctypes.c_int32), ("bfp_block", ctypes.c_int32),
-                ("num_pages", ctypes.c_int64), ("format", ctypes.c_int32)]
+                ("num_pages", ctypes.c_int64), ("format", ctypes.c_int32), ("key_layout", ctypes.c_int32)]
 
 
 class HmaError(RuntimeError):
@@ -108,8 +109,9 @@ def _ptr(t):
     return ctypes.c_void_p(t.data_ptr()) if t is not None else ctypes.c_void_p(0)
 
 
-def make_desc(num_layers, num_q_heads, num_kv_heads, num_pages, fmt=HMA_KV_BFP8, head_dim=128, page_tokens=16, bfp_block=16):
-    return CacheDesc(num_layers, num_q_heads, num_kv_heads, head_dim, page_tokens, bfp_block, num_pages, fmt)
+def make_desc(num_layers, num_q_heads, num_kv_heads, num_pages, fmt=HMA_KV_BFP8, head_dim=128, page_tokens=16, bfp_block=16,
+              key_layout=0):
+    return CacheDesc(num_layers, num_q_heads, num_kv_heads, head_dim, page_tokens, bfp_block, num_pages, fmt, key_layout)
 
 
 def hma_cache_layer_bytes(desc):

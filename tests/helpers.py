@@ -17,12 +17,13 @@ class Scenario:
     """A batch of sequences with seeded BFP8 wire bytes, ingested into a paged cache on the GPU."""
 
     def __init__(self, lens, hq, hkv, seed=0, permute=False, fmt=hma.HMA_KV_BFP8, wire_layout=hma.HMA_WIRE_ROWMAJOR,
-                 shards=1, layers=1, extra_pages=3, fill=0xA5, device="cuda", one_launch=False):
+                 shards=1, layers=1, extra_pages=3, fill=0xA5, device="cuda", one_launch=False, key_layout=0):
         self.lens = np.asarray(lens, np.int32)
         self.B, self.hq, self.hkv, self.layers = len(lens), hq, hkv, layers
         self.seed = seed
         self.table_np, self.num_pages, self.spare = synth.block_table(self.lens, permute, seed, extra_pages)
-        self.desc = hma.make_desc(layers, hq, hkv, self.num_pages, fmt)
+        self.key_layout = key_layout
+        self.desc = hma.make_desc(layers, hq, hkv, self.num_pages, fmt, key_layout=key_layout)
         self.cache = hma.KVCache(self.desc, device, fill=fill)
         self.table = torch.from_numpy(self.table_np).to(device)
         self.ctx = torch.from_numpy(self.lens).to(device)
@@ -69,7 +70,8 @@ class Scenario:
     def oracle(self, layer=0, sm_scale=None, q=None):
         from oracle import oracle as orc
         q = self.q if q is None else q
-        return orc.decode_attention(bf16_bits(q), self.k_wires[layer], self.v_wires[layer], self.hkv, sm_scale)
+        return orc.decode_attention(bf16_bits(q), self.k_wires[layer], self.v_wires[layer], self.hkv, sm_scale,
+                                    keys_interleaved=bool(self.key_layout))
 
 
 def parity_metrics(got, ref64):

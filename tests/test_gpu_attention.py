@@ -70,6 +70,30 @@ def test_bf16_cache_tensor_core_path(hq, hkv):
     assert hma.hma_error_flags(sc.cache) == 0
 
 
+@pytest.mark.parametrize("fmt", [hma.HMA_KV_BFP8, hma.HMA_KV_BF16])
+def test_interleaved_rotary_keys(fmt):
+    """Keys cached in the prefill accelerator's interleaved rotary order, queries in half-split order (key re-layout)."""
+    lens = [33, 700, 16, 0, 2100]
+    sc = Scenario(lens, 40, 8, seed=91, permute=True, fmt=fmt, key_layout=hma.HMA_KEYS_INTERLEAVED)
+    _, ref64, o32, _ = _run_and_check(sc)
+    plain = Scenario(lens, 40, 8, seed=91, permute=True, fmt=fmt)
+    assert np.abs(plain.attention(0, torch.float32).cpu().numpy() - o32).max() > 0.1      # the layout flag matters
+    simple = sc.attention(0, torch.float32, simple=True).cpu().numpy()
+    assert np.abs(simple - o32).max() <= 5e-3
+    # the one-shot rebuild hands the keys over in half-split order; values are untouched
+    from oracle import oracle as orc
+    T = lens[1]
+    pages = sc.table[1, :(T + 15) // 16].contiguous()
+    for which, wires in ((0, sc.k_wires), (1, sc.v_wires)):
+        out = torch.zeros((T, 8, 128), dtype=torch.bfloat16, device="cuda")
+        hma.hma_bfp8_dequant_bf16(sc.cache, 0, which, pages, 0, T, out)
+        torch.cuda.synchronize()
+        want = orc.decode_rowmajor_bf16(wires[0][1])
+        if which == 0:
+            want = orc.relayout_keys_to_half_split(want)
+        assert np.array_equal(bf16_bits(out).transpose(1, 0, 2), want), which
+
+
 def test_long_context_many_splits_and_determinism():
     """One long sequence is cut across every CTA (split-K), short ones sit inside a single CTA."""
     lens = [6000, 40, 2500, 16]

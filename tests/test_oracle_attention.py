@@ -122,3 +122,35 @@ def test_softmax_shift_invariance_and_scale():
     o_b, _ = orc.decode_attention(q, kw, vw, 1, sm_scale=1e3)    # near-argmax
     s = _np_values(kw[0])[0] @ _bf16_to_f64(q[0, 0])
     assert np.allclose(o_b[0, 0], v[0, int(np.argmax(s))], rtol=0, atol=1e-6 * np.abs(v).max()) or np.sort(s)[-1] - np.sort(s)[-2] < 0.02
+
+
+def test_key_relayout_matches_the_two_rotary_conventions():
+    """The interleaved -> half-split map is pinned by RoPE itself: rotating pairs (2i, 2i+1) and then re-laying out
+    equals re-laying out and then rotating pairs (i, i+64) with the same angles."""
+    idx = [orc.half_split_index(c) for c in range(128)]
+    assert sorted(idx) == list(range(128))                                   # a permutation
+    assert idx[:4] == [0, 64, 1, 65] and idx[126:] == [63, 127]
+    rng = np.random.default_rng(10)
+    x = rng.standard_normal((3, 128))
+    theta = rng.uniform(0, 2 * np.pi, 64)
+    c, s = np.cos(theta), np.sin(theta)
+    inter = np.empty_like(x)                                                  # RoPE in interleaved convention
+    inter[:, 0::2] = x[:, 0::2] * c - x[:, 1::2] * s
+    inter[:, 1::2] = x[:, 0::2] * s + x[:, 1::2] * c
+    xs = orc.relayout_keys_to_half_split(x)
+    half = np.empty_like(x)                                                   # RoPE in half-split convention
+    half[:, :64] = xs[:, :64] * c - xs[:, 64:] * s
+    half[:, 64:] = xs[:, :64] * s + xs[:, 64:] * c
+    assert np.allclose(orc.relayout_keys_to_half_split(inter), half, rtol=0, atol=1e-14)
+
+
+def test_attention_with_interleaved_keys_equals_attention_in_one_layout():
+    q, kw, vw = _case(2, 8, 2, [37, 12], 11)
+    o_int, _ = orc.decode_attention(q, kw, vw, 2, keys_interleaved=True)       # q is half-split, keys interleaved
+    q_int = np.empty_like(q)                                                   # the same queries brought to the keys' order
+    for c in range(128):
+        q_int[..., c] = q[..., orc.half_split_index(c)]
+    o_same, _ = orc.decode_attention(q_int, kw, vw, 2)
+    assert np.array_equal(o_int, o_same)
+    o_plain, _ = orc.decode_attention(q, kw, vw, 2)
+    assert not np.allclose(o_int, o_plain)                                     # and the flag does change the result
