@@ -221,6 +221,26 @@ class Workload:
         t = np.array([a.elapsed_time(b) for a, b in evs]) / 1e3
         return float(t.mean()), float(np.median(t)), float(t.min())
 
+    def time_rebuild(self, reps=3):
+        """One-shot BFP8 -> BF16 rebuild of one whole request (sequence 0: every layer, K and V): seconds, bytes moved."""
+        T = int(self.lens[0])
+        pages = self.table[0, :(T + 15) // 16].contiguous()
+        out = torch.empty((self.L, 2, T, self.hkv, 128), dtype=torch.bfloat16, device=self.device)
+        cache = self.caches["bfp8"]
+
+        def run():
+            self.hma.hma_bfp8_rebuild_request(cache, pages, 0, T, out)
+        run()
+        torch.cuda.synchronize(self.device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record()
+        torch.cuda.synchronize(self.device)
+        elems = 2 * self.L * T * self.hkv * 128
+        return e0.elapsed_time(e1) / 1e3 / reps, elems * (17 / 16 + 2), elems
+
     def parity_sample(self):
         """Outputs of sampled sequences against the oracle on the same wire bytes, in the full-size launch configuration.
 
@@ -396,6 +416,10 @@ def main():
                             "kv_gbs": wl.kv_bytes_per_layer("bf16") * wl.L / sec_bf16 / 1e9, "steps": k,
                             "bfp8_speedup": sec_bf16 / sec_decode_only}
 
+    t_rb, rb_bytes, rb_elems = wl.time_rebuild()
+    extra["rebuild_request"] = {"ms": t_rb * 1e3, "tokens": int(wl.lens[0]), "layers": wl.L, "gbs": rb_bytes / t_rb / 1e9,
+                                "frac_of_peak": rb_bytes / t_rb / 1e9 / peak, "calls": 1,
+                                "what": "hma_bfp8_rebuild_request: one request, K and V, all layers, one launch (1.0625 B in + 2 B out per element)"}
     kv_step = wl.kv_bytes_per_layer("bfp8") * wl.L
     value = aggregate_value(wl.B, sec, ws)
     achieved = wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9

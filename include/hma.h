@@ -21,7 +21,8 @@
  *     device, "host" = ordinary host memory, "pinned" = page-locked host memory mapped into the
  *     device address space.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *   - ownership: the caller owns every buffer (cache layers, wire, Q, output, tables, workspace);
- *     the library allocates one 4-byte device flag word per cache handle and nothing else.
+ *     the library makes one small device allocation per cache handle (a flag word and a copy of the
+ *     layer pointers) and nothing else.
  *   - asynchrony: a call validates its arguments on the host, enqueues work on `stream`, and
  *     returns; no call synchronises the device except hma_error_flags.
  *   - errors: invalid arguments return a status and enqueue nothing.  Device-side anomalies never
@@ -222,6 +223,12 @@ hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_t layer, co
 hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t layer, int32_t which,
                                    const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
                                    void *out_bf16, void *stream);
+
+/* The whole request in one launch (section 3.3: "a fused kernel rebuilds a whole request's KV"): every layer, K and V,
+ * -> out_bf16 [num_layers][2 (K, V)][n_tokens][num_kv_heads][128] (device, 16-byte aligned), with the same decode,
+ * key re-layout and page_ids convention as hma_bfp8_dequant_bf16. */
+hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const int32_t *page_ids, int64_t token_begin,
+                                      int64_t n_tokens, void *out_bf16, void *stream);
 
 /* Flat variant: n_blocks blocks, exps[i] with mants[16*i .. 16*i+15] -> out_bf16[16*i ..] (device pointers). */
 hma_status_t hma_bfp8_dequant_blocks_bf16(const uint8_t *exps, const uint8_t *mants, int64_t n_blocks,

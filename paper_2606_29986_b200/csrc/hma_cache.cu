@@ -46,13 +46,18 @@ extern "C" hma_status_t hma_cache_create(const hma_cache_desc_t *desc, void *con
     c->desc = *desc;
     c->layers = (void **)std::malloc(sizeof(void *) * (size_t)desc->num_layers);
     std::memcpy(c->layers, layer_ptrs, sizeof(void *) * (size_t)desc->num_layers);
-    if (cudaGetDevice(&c->device) != cudaSuccess || cudaMalloc((void **)&c->flags, sizeof(uint32_t)) != cudaSuccess ||
-        cudaMemset(c->flags, 0, sizeof(uint32_t)) != cudaSuccess) {
+    // one small device allocation: the flag word (16 bytes reserved), then the table of layer pointers
+    const size_t table = sizeof(void *) * (size_t)desc->num_layers;
+    if (cudaGetDevice(&c->device) != cudaSuccess || cudaMalloc((void **)&c->flags, 16 + table) != cudaSuccess ||
+        cudaMemset(c->flags, 0, 16) != cudaSuccess ||
+        cudaMemcpy((uint8_t *)c->flags + 16, layer_ptrs, table, cudaMemcpyHostToDevice) != cudaSuccess) {
+        if (c->flags) (void)cudaFree(c->flags);
         (void)cudaGetLastError();
         std::free(c->layers);
         std::free(c);
         return HMA_ERR_CUDA;
     }
+    c->d_layers = (void **)((uint8_t *)c->flags + 16);
     *out = c;
     return HMA_OK;
 }

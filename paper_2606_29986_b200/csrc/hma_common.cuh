@@ -89,7 +89,8 @@ void count_launch();
 struct hma_cache {
     hma_cache_desc_t desc;
     void **layers;       // host copy of the device pointers
-    uint32_t *flags;     // device flag word
+    uint32_t *flags;     // device flag word (first word of the handle's one device allocation)
+    void **d_layers;     // device copy of the layer pointers (same allocation, after the flag word)
     int device;
 };
 

@@ -1,7 +1,31 @@
 // Stand-alone BFP8 -> BF16 reconstruction (section 3.3: block-float decode to BF16, bit-exact).
+#include <cuda_fp16.h>
+
 #include "hma_common.cuh"
 
 namespace hma {
+
+// Four elements of one block -> four BF16 bit patterns, bit-exact for every (E, byte) pair.
+// The byte s<<7|m is first spread to the FP16 pattern s<<15|m, the FP16 subnormal +-m * 2^-24 (two integer
+// instructions per pair: section 3.3's "shifts, masks, ORs and a bitcast"); widening to fp32 and multiplying by
+// 2^(E-109), split in two exact power-of-two factors so that every E in 0..255 stays in range, gives
+// m * 2^(E-133) exactly (fp32 subnormals and overflow to Inf included); its upper 16 bits are the BF16 value.
+// The sign rides along, so m = 0 keeps its sign.
+__device__ __forceinline__ uint2 dequant4(uint32_t w, uint32_t E)
+{
+    const float s1 = __uint_as_float(((E >> 1) + 73u) << 23);           // 2^(floor(E/2) - 54)
+    const float s2 = __uint_as_float(((E - (E >> 1)) + 72u) << 23);     // 2^(ceil(E/2) - 55)
+    uint32_t h01, h23;
+    asm("prmt.b32 %0, %1, 0, 0x1100;" : "=r"(h01) : "r"(w));
+    asm("prmt.b32 %0, %1, 0, 0x3322;" : "=r"(h23) : "r"(w));
+    h01 &= 0x807F807Fu;
+    h23 &= 0x807F807Fu;
+    const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&h01));
+    const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&h23));
+    const uint32_t b0 = __float_as_uint((f01.x * s1) * s2), b1 = __float_as_uint((f01.y * s1) * s2);
+    const uint32_t b2 = __float_as_uint((f23.x * s1) * s2), b3 = __float_as_uint((f23.y * s1) * s2);
+    return make_uint2(__byte_perm(b0, b1, 0x7632), __byte_perm(b2, b3, 0x7632));
+}
 
 // Flat blocks: two threads per block, 8 elements each; 8-byte loads, 16-byte stores, both coalesced.
 __global__ void __launch_bounds__(256) dequant_blocks_kernel(const uint8_t *__restrict__ exps,
@@ -11,75 +35,87 @@ __global__ void __launch_bounds__(256) dequant_blocks_kernel(const uint8_t *__re
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // index of an 8-element half block
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (; i < 2 * n_blocks; i += stride) {
-        uint32_t E = exps[i >> 1];
-        uint2 m = *reinterpret_cast<const uint2 *>(mants + i * 8);
-        uint32_t w[2] = {m.x, m.y};
-        uint32_t o[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            uint32_t lo = bfp8_to_bf16_bits(E, (w[k >> 1] >> ((k & 1) * 16)) & 0xFFu);
-            uint32_t hi = bfp8_to_bf16_bits(E, (w[k >> 1] >> ((k & 1) * 16 + 8)) & 0xFFu);
-            o[k] = lo | (hi << 16);
-        }
-        *reinterpret_cast<uint4 *>(out + i * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+        const uint32_t E = exps[i >> 1];
+        const uint2 m = *reinterpret_cast<const uint2 *>(mants + i * 8);
+        const uint2 lo = dequant4(m.x, E), hi = dequant4(m.y, E);
+        *reinterpret_cast<uint4 *>(out + i * 8) = make_uint4(lo.x, lo.y, hi.x, hi.y);
     }
 }
 
-// One CTA per (logical page of the request, kv head): stage the K or V part of the record in shared
-// memory, then each thread rebuilds 8 consecutive channels of one token and stores 16 bytes.
+// One CTA per (logical page of the request, kv head): the K or V half record is staged in shared memory, then each
+// thread rebuilds 4 consecutive channels of one token at a time and stores 8 bytes.  (One CTA per page covering all
+// heads was measured slower: too few threads in flight for a copy-like kernel.)
+constexpr int kDequantHeads = 1;
+// With `layers` set, blockIdx.z = 2 * layer + which selects the layer and the tensor, and the output is
+// [num_layers][2][n_tokens][Hkv][128]: the whole request in one launch.
 __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int which, const int32_t *__restrict__ page_ids,
                                                             int64_t token_begin, int64_t n_tokens,
-                                                            uint16_t *__restrict__ out)
+                                                            uint16_t *__restrict__ out, void *const *__restrict__ layers)
 {
-    __shared__ __align__(16) uint8_t rec[kBf16Half];
-    const int h = blockIdx.y;
+    if (layers) {
+        cv.layer = (uint8_t *)layers[blockIdx.z >> 1];
+        which = blockIdx.z & 1;
+        out += (int64_t)blockIdx.z * n_tokens * cv.num_kv_heads * kHeadDim;
+    }
+    __shared__ __align__(16) uint8_t recs[kDequantHeads][kBf16Half];
     const int64_t first_page = token_begin / kPageTokens;
     const int64_t lp = first_page + blockIdx.x;
     const int32_t pid = page_ids[blockIdx.x];
     const bool bad = pid < 0 || pid >= cv.num_pages;
     const int half = cv.format == HMA_KV_BFP8 ? kBfp8Half : kBf16Half;
-    if (!bad) {
-        const uint8_t *src = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)(2 * half) + (int64_t)which * half;
-        for (int o = threadIdx.x * 16; o < half; o += blockDim.x * 16)
-            *reinterpret_cast<uint4 *>(rec + o) = *reinterpret_cast<const uint4 *>(src + o);
-    } else if (threadIdx.x == 0) {
-        atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_DEQUANT);
-    }
-    __syncthreads();
-    for (int item = threadIdx.x; item < kPageTokens * 16; item += blockDim.x) {
-        const int tok = item >> 4, c0 = (item & 15) * 8;
-        const int64_t gt = lp * kPageTokens + tok;
-        if (gt < token_begin || gt >= token_begin + n_tokens) continue;
-        uint32_t o[4] = {0, 0, 0, 0};
+    const bool relayout = which == 0 && cv.key_layout == HMA_KEYS_INTERLEAVED;
+    if (bad && threadIdx.x == 0) atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_DEQUANT);
+    {
+        const int h0 = blockIdx.y;
+        constexpr int nh = 1;
         if (!bad) {
-            if (cv.format == HMA_KV_BFP8) {
-                // `rec` holds one half record: offsets are relative to the start of that half
-                const uint32_t E = which == 0 ? rec[bfp8_k_exp_off(tok, c0 >> 4)] : rec[bfp8_v_exp_off(tok, c0 >> 4) - kBfp8Half];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int ch = c0 + k;
-                    const uint32_t b = which == 0 ? rec[bfp8_k_el_off(tok, ch)] : rec[bfp8_v_el_off(tok, ch) - kBfp8Half];
-                    o[k >> 1] |= bfp8_to_bf16_bits(E, b) << ((k & 1) * 16);
-                }
-            } else {
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int ch = c0 + k;
-                    const int off = which == 0 ? bf16_k_el_off(tok, ch) : bf16_v_el_off(tok, ch) - kBf16Half;
-                    o[k >> 1] |= (uint32_t)(*reinterpret_cast<const uint16_t *>(rec + off)) << ((k & 1) * 16);
-                }
+            const int per = half / 16;                                  // 16-byte pieces per head
+            for (int i = threadIdx.x; i < nh * per; i += blockDim.x) {
+                const int hh = i / per, o = (i - hh * per) * 16;
+                const uint8_t *src = cv.layer + ((int64_t)pid * cv.num_kv_heads + h0 + hh) * (int64_t)(2 * half) + (int64_t)which * half;
+                *reinterpret_cast<uint4 *>(&recs[hh][o]) = *reinterpret_cast<const uint4 *>(src + o);
             }
         }
-        uint16_t *row = out + ((gt - token_begin) * cv.num_kv_heads + h) * kHeadDim;
-        if (which == 0 && cv.key_layout == HMA_KEYS_INTERLEAVED) {
-            // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout):
-            // cached channels c0, c0+2, .. go to c0/2 .., cached channels c0+1, c0+3, .. to 64 + c0/2 ..
-            const uint32_t e0 = (o[0] & 0xFFFFu) | (o[1] << 16), e1 = (o[2] & 0xFFFFu) | (o[3] << 16);
-            const uint32_t d0 = (o[0] >> 16) | (o[1] & 0xFFFF0000u), d1 = (o[2] >> 16) | (o[3] & 0xFFFF0000u);
-            *reinterpret_cast<uint2 *>(row + (c0 >> 1)) = make_uint2(e0, e1);
-            *reinterpret_cast<uint2 *>(row + 64 + (c0 >> 1)) = make_uint2(d0, d1);
-        } else {
-            *reinterpret_cast<uint4 *>(row + c0) = make_uint4(o[0], o[1], o[2], o[3]);
+        __syncthreads();
+        for (int item = threadIdx.x; item < kPageTokens * nh * 32; item += blockDim.x) {
+            const int c0 = (item & 31) * 4;                             // channels c0 .. c0+3
+            const int hh = (item >> 5) % nh, tok = (item >> 5) / nh;    // items ordered like the output: token, head, channel
+            const int64_t gt = lp * kPageTokens + tok;
+            if (gt < token_begin || gt >= token_begin + n_tokens) continue;
+            const uint8_t *rec = recs[hh];
+            uint2 o = make_uint2(0u, 0u);
+            if (!bad) {
+                // `rec` holds one half record: offsets below are relative to the start of that half
+                if (cv.format == HMA_KV_BFP8) {
+                    uint32_t w, E;
+                    if (which == 0) {
+                        E = rec[bfp8_k_exp_off(tok, c0 >> 4)];
+                        w = *reinterpret_cast<const uint32_t *>(rec + bfp8_k_el_off(tok, c0));   // four channels are one word
+                    } else {
+                        E = rec[bfp8_v_exp_off(tok, c0 >> 4) - kBfp8Half];
+                        w = rec[bfp8_v_el_off(tok, c0) - kBfp8Half] | (rec[bfp8_v_el_off(tok, c0 + 1) - kBfp8Half] << 8) |
+                            (rec[bfp8_v_el_off(tok, c0 + 2) - kBfp8Half] << 16) |
+                            ((uint32_t)rec[bfp8_v_el_off(tok, c0 + 3) - kBfp8Half] << 24);
+                    }
+                    o = dequant4(w, E);
+                } else if (which == 0) {
+                    o = *reinterpret_cast<const uint2 *>(rec + bf16_k_el_off(tok, c0));            // four channels are 8 bytes
+                } else {
+                    uint32_t e[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) e[k] = *reinterpret_cast<const uint16_t *>(rec + bf16_v_el_off(tok, c0 + k) - kBf16Half);
+                    o = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
+                }
+            }
+            uint16_t *row = out + ((gt - token_begin) * cv.num_kv_heads + h0 + hh) * kHeadDim;
+            if (relayout) {
+                // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout):
+                // cached channels c0, c0+2 go to c0/2, c0/2+1; cached channels c0+1, c0+3 to 64 + c0/2, 64 + c0/2 + 1
+                *reinterpret_cast<uint32_t *>(row + (c0 >> 1)) = (o.x & 0xFFFFu) | (o.y << 16);
+                *reinterpret_cast<uint32_t *>(row + 64 + (c0 >> 1)) = (o.x >> 16) | (o.y & 0xFFFF0000u);
+            } else {
+                *reinterpret_cast<uint2 *>(row + c0) = o;
+            }
         }
     }
 }
@@ -118,7 +154,28 @@ extern "C" hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t 
                       cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
     dim3 grid((unsigned)n_pages, (unsigned)cache->desc.num_kv_heads);
     hma::dequant_paged_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, which, page_ids, token_begin, n_tokens,
-                                                                      (uint16_t *)out_bf16);
+                                                                      (uint16_t *)out_bf16, nullptr);
+    hma::count_launch();
+    HMA_CUDA_OK(cudaGetLastError());
+    return HMA_OK;
+}
+
+extern "C" hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const int32_t *page_ids, int64_t token_begin,
+                                                 int64_t n_tokens, void *out_bf16, void *stream)
+{
+    if (!cache || token_begin < 0 || n_tokens < 0) return HMA_ERR_INVALID_ARG;
+    if (n_tokens == 0) return HMA_OK;
+    if (!page_ids || !out_bf16) return HMA_ERR_INVALID_ARG;
+    if ((uintptr_t)out_bf16 & 15u) return HMA_ERR_ALIGNMENT;
+    const int64_t first = token_begin / hma::kPageTokens;
+    const int64_t last = (token_begin + n_tokens - 1) / hma::kPageTokens;
+    const int64_t n_pages = last - first + 1;
+    if (n_pages > 0x7FFFFFFF || cache->desc.num_layers > 32767) return HMA_ERR_INVALID_ARG;
+    hma::CacheView cv{(uint8_t *)cache->layers[0], cache->desc.num_pages, cache->desc.num_kv_heads,
+                      cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
+    dim3 grid((unsigned)n_pages, (unsigned)cache->desc.num_kv_heads, (unsigned)(2 * cache->desc.num_layers));
+    hma::dequant_paged_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, 0, page_ids, token_begin, n_tokens,
+                                                                      (uint16_t *)out_bf16, cache->d_layers);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;

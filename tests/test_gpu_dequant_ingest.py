@@ -101,6 +101,43 @@ def test_all_shards_in_one_launch_equal_shard_by_shard(layout):
     assert e.value.status == hma.HMA_ERR_INVALID_ARG
 
 
+def test_paged_dequant_of_arbitrary_bytes_every_exponent():
+    """Random wire bytes (every exponent 0..255, every element byte) through ingest and the paged rebuild."""
+    rng = np.random.default_rng(12)
+    T, H = 64, 2
+    desc = hma.make_desc(1, 2, H, 6)
+    cache = hma.KVCache(desc, "cuda", fill=0)
+    pages = torch.tensor([4, 1, 5, 2], dtype=torch.int32, device="cuda")
+    for trial in range(3):
+        kw = rng.integers(0, 256, (H, T, 136)).astype(np.uint8)
+        vw = rng.integers(0, 256, (H, T, 136)).astype(np.uint8)
+        kw[0, :32, :8] = np.arange(256, dtype=np.uint8).reshape(32, 8)           # each exponent at least once
+        vw[1, 32:, :8] = np.arange(256, dtype=np.uint8).reshape(32, 8)[::-1]
+        hma.hma_kv_ingest_layer(cache, 0, torch.from_numpy(kw).cuda(), torch.from_numpy(vw).cuda(), hma.HMA_WIRE_ROWMAJOR, 0, H, pages, 0, T)
+        for which, wire in ((0, kw), (1, vw)):
+            out = torch.zeros((T, H, 128), dtype=torch.bfloat16, device="cuda")
+            hma.hma_bfp8_dequant_bf16(cache, 0, which, pages, 0, T, out)
+            torch.cuda.synchronize()
+            assert np.array_equal(bf16_bits(out).transpose(1, 0, 2), orc.decode_rowmajor_bf16(wire))
+    assert hma.hma_error_flags(cache) == 0
+
+
+@pytest.mark.parametrize("fmt", [hma.HMA_KV_BFP8, hma.HMA_KV_BF16])
+def test_whole_request_rebuild_in_one_launch(fmt):
+    sc = Scenario([75, 16, 200], 16, 4, seed=14, permute=True, fmt=fmt, layers=3, key_layout=hma.HMA_KEYS_INTERLEAVED)
+    for b, t0, n in ((0, 0, 75), (2, 37, 101)):
+        first, last = t0 // 16, (t0 + n - 1) // 16
+        pages = sc.table[b, first:last + 1].contiguous()
+        out = torch.zeros((3, 2, n, 4, 128), dtype=torch.bfloat16, device="cuda")
+        hma.hma_bfp8_rebuild_request(sc.cache, pages, t0, n, out)
+        torch.cuda.synchronize()
+        got = bf16_bits(out)
+        for l in range(3):
+            wk = orc.relayout_keys_to_half_split(orc.decode_rowmajor_bf16(sc.k_wires[l][b][:, t0:t0 + n]))
+            wv = orc.decode_rowmajor_bf16(sc.v_wires[l][b][:, t0:t0 + n])
+            assert np.array_equal(got[l, 0].transpose(1, 0, 2), wk) and np.array_equal(got[l, 1].transpose(1, 0, 2), wv)
+
+
 def test_bfp8_cache_holds_the_wire_bytes_unchanged():
     """Ingest permutes positions only: the multiset of bytes of a fully written page equals that of its wire rows."""
     sc = Scenario([32], 8, 2, seed=6, layers=1, extra_pages=0)
