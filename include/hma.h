@@ -66,6 +66,7 @@ typedef enum { HMA_KEYS_AS_QUERIES = 0, HMA_KEYS_INTERLEAVED = 1 } hma_key_layou
 #define HMA_FLAG_BAD_PAGE_INGEST    2u  /* page id outside [0, num_pages): page not written      */
 #define HMA_FLAG_BAD_PAGE_DEQUANT   4u  /* page id outside [0, num_pages): output rows zeroed    */
 #define HMA_FLAG_WAIT_TIMEOUT       8u  /* a bounded wait inside a kernel ran out                */
+#define HMA_FLAG_BAD_VALUE_ENCODE  16u  /* hma_bfp8_encode_rows met NaN/Inf: encoded as zero      */
 
 typedef struct {
     int32_t num_layers;
@@ -155,6 +156,7 @@ hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32
  *   context_lens device int32 [batch]; every entry <= max_pages_per_seq*16
  *   workspace    device, 256-byte aligned, >= hma_decode_attention_workspace_bytes(...) bytes;
  *                contents need no initialisation and are clobbered
+ *   batch        at most 2048 (HMA_ERR_UNSUPPORTED_SHAPE beyond)
  * Accuracy: fp32 accumulation; element exponents above 250 are outside the supported range.
  */
 size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *desc, int32_t batch);
@@ -233,6 +235,18 @@ hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const int32_t *p
 /* Flat variant: n_blocks blocks, exps[i] with mants[16*i .. 16*i+15] -> out_bf16[16*i ..] (device pointers). */
 hma_status_t hma_bfp8_dequant_blocks_bf16(const uint8_t *exps, const uint8_t *mants, int64_t n_blocks,
                                           void *out_bf16, void *stream);
+
+/*
+ * BFP8 encode on the GPU: n_rows rows of 128 channels (FP32, or BF16 when x_is_bf16 = 1; device, 16-byte aligned)
+ * -> HMA_WIRE_ROWMAJOR rows of 136 bytes (device, 8-byte aligned), ready for hma_kv_ingest_layer.  This is the
+ * format the prefill accelerator produces (sections 3.1, 3.3); the paper does not say how KV made on the decode GPU
+ * (freshly generated tokens) joins a BFP8 cache, and this call is this library's answer: encode the token's K and V
+ * rows here, then ingest them at token_begin = current length.  Shared exponent = largest FP32 exponent field of the
+ * block; significands rounded to nearest-even onto 7 bits, a carry saturates at 127; FP32 subnormals encode as zero;
+ * the sign is always copied.  NaN/Inf encode as zero and raise HMA_FLAG_BAD_VALUE_ENCODE in the cache's flag word
+ * (`cache` is used for nothing else). */
+hma_status_t hma_bfp8_encode_rows(const hma_cache_t *cache, const void *x, int32_t x_is_bf16, int64_t n_rows,
+                                  void *wire_rowmajor, void *stream);
 
 /* Copies the cache's device flag word to *host_out and clears it.  Synchronises `stream`. */
 hma_status_t hma_error_flags(const hma_cache_t *cache, uint32_t *host_out, void *stream);

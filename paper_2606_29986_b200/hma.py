@@ -21,6 +21,7 @@ HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR = 0, 1
 HMA_OUT_BF16, HMA_OUT_F32 = 0, 1
 HMA_KEYS_AS_QUERIES, HMA_KEYS_INTERLEAVED = 0, 1
 HMA_FLAG_BAD_PAGE_ATTENTION, HMA_FLAG_BAD_PAGE_INGEST, HMA_FLAG_BAD_PAGE_DEQUANT, HMA_FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
+HMA_FLAG_BAD_VALUE_ENCODE = 16
 
 
 class CacheDesc(ctypes.Structure):
@@ -78,6 +79,8 @@ def lib():
         L.hma_bfp8_dequant_bf16.argtypes = [vp, i32, i32, vp, i64, i64, vp, vp]
         L.hma_bfp8_rebuild_request.restype = i32
         L.hma_bfp8_rebuild_request.argtypes = [vp, vp, i64, i64, vp, vp]
+        L.hma_bfp8_encode_rows.restype = i32
+        L.hma_bfp8_encode_rows.argtypes = [vp, vp, i32, i64, vp, vp]
         L.hma_bfp8_dequant_blocks_bf16.restype = i32
         L.hma_bfp8_dequant_blocks_bf16.argtypes = [vp, vp, i64, vp, vp]
         L.hma_error_flags.restype = i32
@@ -226,6 +229,13 @@ def hma_bfp8_rebuild_request(cache, page_ids, token_begin, n_tokens, out_bf16, s
     """Every layer, K and V, of one request in a single launch -> out_bf16 [layers][2][n_tokens][Hkv][128]."""
     _check(lib().hma_bfp8_rebuild_request(cache.handle, _ptr(page_ids), token_begin, n_tokens, _ptr(out_bf16), _stream(stream)),
            "hma_bfp8_rebuild_request")
+
+
+def hma_bfp8_encode_rows(cache, x, wire_rowmajor, stream=None):
+    """x: float32 or bfloat16 tensor [..., 128] -> ROWMAJOR BFP8 rows in wire_rowmajor (uint8 [..., 136])."""
+    n_rows = x.numel() // 128
+    _check(lib().hma_bfp8_encode_rows(cache.handle, _ptr(x), 1 if x.dtype == torch.bfloat16 else 0, n_rows,
+                                      _ptr(wire_rowmajor), _stream(stream)), "hma_bfp8_encode_rows")
 
 
 def hma_bfp8_dequant_blocks_bf16(exps, mants, n_blocks, out_bf16, stream=None):

@@ -138,6 +138,43 @@ def test_whole_request_rebuild_in_one_launch(fmt):
             assert np.array_equal(got[l, 0].transpose(1, 0, 2), wk) and np.array_equal(got[l, 1].transpose(1, 0, 2), wv)
 
 
+def test_gpu_encoder_is_bit_identical_to_the_oracle_encoder():
+    rng = np.random.default_rng(15)
+    x = (rng.standard_normal((3, 37, 128)) * 4.0 ** rng.integers(-6, 7, (3, 37, 1))).astype(np.float32)
+    x[rng.random(x.shape) < 0.02] *= 20
+    x[rng.random(x.shape) < 0.02] = 0.0
+    x[0, 0, :16] = [1.0, 0.5, -0.25, 0.0, 127 / 64, 1 / 64, 1 / 128, 3 / 128, 255 / 128, -1 / 3, 0.1, -0.0, 0.75, 1e-3, -1.5, 0.3]
+    x[0, 1, :] = 1e-41                       # FP32 subnormals
+    x[0, 2, :] = 0
+    x[0, 3, :16] = 2.0 ** -140
+    x[0, 3, 0] = 3e38
+    x[1, 0, :16] = 2.0 ** np.arange(-20, -4, dtype=np.float32)      # shifts beyond 24 bits
+    sc = Scenario([16], 9, 3, seed=15)
+    wire = torch.zeros((3, 37, 136), dtype=torch.uint8, device="cuda")
+    hma.hma_bfp8_encode_rows(sc.cache, torch.from_numpy(x).cuda(), wire)
+    torch.cuda.synchronize()
+    assert np.array_equal(wire.cpu().numpy(), orc.encode_rowmajor(x))
+    xb = torch.from_numpy(x).to(torch.bfloat16)
+    hma.hma_bfp8_encode_rows(sc.cache, xb.cuda(), wire)
+    torch.cuda.synchronize()
+    assert np.array_equal(wire.cpu().numpy(), orc.encode_rowmajor(xb.float().numpy()))
+    assert hma.hma_error_flags(sc.cache) == 0
+    # a token made on the GPU joins the cache: encode its K, V rows and ingest them at the end of the sequence
+    knew, vnew = torch.from_numpy(x[:, :1]).cuda().contiguous(), torch.from_numpy(x[:, 1:2]).cuda().contiguous()
+    kw, vw = torch.zeros((3, 1, 136), dtype=torch.uint8, device="cuda"), torch.zeros((3, 1, 136), dtype=torch.uint8, device="cuda")
+    hma.hma_bfp8_encode_rows(sc.cache, knew, kw)
+    hma.hma_bfp8_encode_rows(sc.cache, vnew, vw)
+    page = sc.spare[:1].copy()
+    hma.hma_kv_ingest_layer(sc.cache, 0, kw, vw, hma.HMA_WIRE_ROWMAJOR, 0, 3, torch.from_numpy(page).cuda(), 16, 1)
+    out = torch.zeros((1, 3, 128), dtype=torch.bfloat16, device="cuda")
+    hma.hma_bfp8_dequant_bf16(sc.cache, 0, 0, torch.from_numpy(page).cuda(), 16, 1, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_bits(out).transpose(1, 0, 2), orc.decode_rowmajor_bf16(orc.encode_rowmajor(x[:, :1])))
+    bad = torch.full((1, 128), float("inf"), device="cuda")
+    hma.hma_bfp8_encode_rows(sc.cache, bad, kw[:1])
+    assert hma.hma_error_flags(sc.cache) == hma.HMA_FLAG_BAD_VALUE_ENCODE
+
+
 def test_bfp8_cache_holds_the_wire_bytes_unchanged():
     """Ingest permutes positions only: the multiset of bytes of a fully written page equals that of its wire rows."""
     sc = Scenario([32], 8, 2, seed=6, layers=1, extra_pages=0)
