@@ -233,21 +233,33 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    // exclusive prefix of pages per sequence
+    // exclusive prefix of pages per sequence: each thread owns `per` consecutive sequences, warps scan with
+    // shuffles, one warp scans the warp totals
     {
         const int per = (B + kThreads - 1) / kThreads;
         const int b0 = min(B, tid * per), b1 = min(B, b0 + per);
-        int sum = 0;
-        for (int b = b0; b < b1; ++b) sum += pages_of(a, b);
-        misc[16 + tid] = sum;
+        int mine = 0;
+        for (int b = b0; b < b1; ++b) mine += pages_of(a, b);
+        int incl = mine;                                   // inclusive scan inside the warp
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= d) incl += v;
+        }
+        if (lane == 31) misc[16 + warp] = incl;
         __syncthreads();
-        if (tid == 0) {
-            int run = 0;
-            for (int i = 0; i < kThreads; ++i) { int v = misc[16 + i]; misc[16 + i] = run; run += v; }
-            cum[B] = run;
+        if (warp == 0) {
+            int tot = lane < kWarps ? misc[16 + lane] : 0, run = tot;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int v = __shfl_up_sync(0xFFFFFFFFu, run, d);
+                if (lane >= d) run += v;
+            }
+            if (lane < kWarps) misc[16 + lane] = run - tot;              // pages before each warp's sequences
+            if (lane == kWarps - 1) cum[B] = run;
         }
         __syncthreads();
-        int run = misc[16 + tid];
+        int run = misc[16 + warp] + incl - mine;
         for (int b = b0; b < b1; ++b) { cum[b] = run; run += pages_of(a, b); }
         __syncthreads();
     }
