@@ -233,6 +233,9 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // The kernel is launched with programmatic stream serialisation: its CTAs may be placed while the previous
+    // kernel of the stream drains.  Nothing that a predecessor could have written is read before this wait.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // exclusive prefix of pages per sequence: each thread owns `per` consecutive sequences, warps scan with
     // shuffles, one warp scans the warp totals
     {
@@ -708,7 +711,8 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
 // to 32 parts come from one round of loads; the 128-vectors are then fetched four parts at a time.
 __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int max_workers)
 {
-    asm volatile("griddepcontrol.wait;" ::: "memory");           // the main kernel's tiles are complete and visible
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may be placed; it waits by itself
+    asm volatile("griddepcontrol.wait;" ::: "memory");               // the main kernel's tiles are complete and visible
     const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
     const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, h = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (h >= G) return;
@@ -861,25 +865,28 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
     constexpr int tb = hma::Geo<HMA_KV_BFP8>::threads, tf = hma::Geo<HMA_KV_BF16>::threads;
-    if (bf16 && probe == 0) hma::attn_kernel<0, HMA_KV_BF16><<<n_ctas, tf, smem, s>>>(a);
-    else if (bf16) hma::attn_kernel<1, HMA_KV_BF16><<<n_ctas, tf, smem, s>>>(a);
-    else if (probe == 0) hma::attn_kernel<0, HMA_KV_BFP8><<<n_ctas, tb, smem, s>>>(a);
-    else if (probe == 1) hma::attn_kernel<1, HMA_KV_BFP8><<<n_ctas, tb, smem, s>>>(a);
-    else hma::attn_kernel<2, HMA_KV_BFP8><<<n_ctas, tb, smem, s>>>(a);
-    hma::count_launch();
-    HMA_CUDA_OK(cudaGetLastError());
-    if (probe) return HMA_OK;
-    // the merge kernel may be scheduled while the main kernel still runs; it waits on the grid dependency itself
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(batch * cache->desc.num_kv_heads));
-    cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = s;
+    // Both kernels are launched with programmatic stream serialisation: each may be placed on the SMs while its
+    // predecessor drains, and each waits on the grid dependency itself before it reads anything.
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_ctas);
+    cfg.blockDim = dim3((unsigned)(bf16 ? tf : tb));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (bf16 && probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BF16>, a));
+    else if (bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BF16>, a));
+    else if (probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BFP8>, a));
+    else if (probe == 1) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BFP8>, a));
+    else HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<2, HMA_KV_BFP8>, a));
+    hma::count_launch();
+    if (probe) return HMA_OK;
+    cfg.gridDim = dim3((unsigned)(batch * cache->desc.num_kv_heads));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
     HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_kernel, a,
                                    n_ctas * (bf16 ? hma::Geo<HMA_KV_BF16>::warps : hma::Geo<HMA_KV_BFP8>::warps)));
     hma::count_launch();
