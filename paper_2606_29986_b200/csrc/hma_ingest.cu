@@ -36,7 +36,7 @@ __device__ __forceinline__ int64_t wire_block_off(int layout, int64_t n_tokens, 
 // memory in row-major form (16-byte or 8-byte coalesced reads).  Phase 2 walks the destination
 // record word by word, gathers its bytes from the staged rows, and writes whole words; a word that
 // mixes tokens inside and outside the range is merged with the bytes already in the cache.
-__global__ void __launch_bounds__(256) ingest_kernel(CacheView cv, IngestArgs a)
+__global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
 {
     __shared__ __align__(16) uint8_t rows[2][kPageTokens][kRowBytes + 8];   // +8 keeps element bytes 16-byte aligned
     // blockIdx.y runs over the heads of all shards in turn
@@ -177,7 +177,7 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
     a.n_tokens = n_tokens;
     a.layout = wire_layout;
     dim3 grid((unsigned)n_pages, (unsigned)heads);
-    hma::ingest_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(cv, a);
+    hma::ingest_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;
