@@ -158,6 +158,10 @@ hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32
  *                contents need no initialisation and are clobbered
  *   batch        at most 2048 (HMA_ERR_UNSUPPORTED_SHAPE beyond)
  * Accuracy: fp32 accumulation; element exponents above 250 are outside the supported range.
+ * Launches: two kernels per call (attention, then a small merge of the per-worker partials), both with
+ * programmatic stream serialisation; each waits on the grid dependency before it reads any input, so the
+ * usual stream order holds whatever kernel precedes the call.  The first call on a device sets the kernels'
+ * shared-memory attributes.
  */
 size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *desc, int32_t batch);
 hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,

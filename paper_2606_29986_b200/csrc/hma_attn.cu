@@ -20,6 +20,7 @@
 //     to a running per-block reference exponent that is handled like the running softmax maximum.
 //   * the softmax weights go to the second MMA as FP16 (11 significant bits), not BF16.
 #include <cuda_fp16.h>
+#include <mutex>
 
 #include "hma_common.cuh"
 
@@ -44,6 +45,7 @@ constexpr uint32_t kSuspendNs = 2000;              // a failed poll may keep the
 constexpr int kMaxBatch = 2048;
 constexpr int kMaxCtas = 160;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
 constexpr int kMinRecords = 8;                    // fewest records a worker takes
+constexpr int kMaxDevices = 64;
 
 struct AttnArgs {
     CacheView cv;
@@ -832,22 +834,27 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     if (workspace_bytes < hma_decode_attention_workspace_bytes(&cache->desc, batch)) return HMA_ERR_WORKSPACE_TOO_SMALL;
     const bool bf16 = cache->desc.format != HMA_KV_BFP8;
     if (bf16 && probe == 2) return HMA_ERR_UNSUPPORTED_SHAPE;
-    static int n_sm = 0;
-    static bool attr_set = false;
-    if (!n_sm) {
-        int dev = 0;
-        HMA_CUDA_OK(cudaGetDevice(&dev));
-        HMA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    // per-device set-up, done by the first call on each device: SM count and the kernels' shared-memory opt-in
+    static std::mutex setup_lock;
+    static int sm_count[hma::kMaxDevices] = {};
+    int dev = 0;
+    HMA_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= hma::kMaxDevices) return HMA_ERR_UNSUPPORTED_SHAPE;
+    {
+        std::lock_guard<std::mutex> guard(setup_lock);
+        if (!sm_count[dev]) {
+            int n = 0;
+            HMA_CUDA_OK(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<2, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            sm_count[dev] = n;
+        }
     }
+    const int n_sm = sm_count[dev];
     const size_t smem = bf16 ? hma::attn_smem_bytes<HMA_KV_BF16>(batch) : hma::attn_smem_bytes<HMA_KV_BFP8>(batch);
-    if (!attr_set) {
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<2, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set = true;
-    }
     if (smem > 227 * 1024) return HMA_ERR_UNSUPPORTED_SHAPE;
     hma::AttnArgs a;
     a.cv = hma::CacheView{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
@@ -930,7 +937,6 @@ namespace hma {
 constexpr int kStaticMaxSegments = 512;       // batch * num_kv_heads
 constexpr size_t kStaticWsBytes = 4096 + (size_t)(kMaxCtas * kWarps + kStaticMaxSegments) * kTileFloats * 4;   // 12.2 MiB
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
-constexpr int kMaxDevices = 64;
 static void *g_static_ws_ptr[kMaxDevices];    // device address of g_static_ws on each device, resolved on first use
 }  // namespace hma
 
