@@ -44,7 +44,7 @@ constexpr uint32_t kSpinLimit = 1u << 20;           // polls of a bounded wait
 constexpr uint32_t kSuspendNs = 2000;              // a failed poll may keep the thread parked this long
 constexpr int kMaxBatch = 2048;
 constexpr int kMaxCtas = 160;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
-constexpr int kMinRecords = 8;                    // fewest records a worker takes
+constexpr int kMinRecords = 4;                    // fewest records a worker takes
 constexpr int kMaxDevices = 64;
 
 struct AttnArgs {
