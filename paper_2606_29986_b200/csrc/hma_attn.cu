@@ -351,7 +351,9 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         if (++kissue == kwin + 32 && kissue < Rw) { kwin = kissue; refill(); }
     };
     if (kMode != 2) refill();
-    for (int k = 0; k < kDepth && k < Rw; ++k) issue();
+    // Only the first record is requested now; the other slots are armed after the first segment's Q loads have been
+    // issued, so that across the GPU every warp's first record is ahead of anybody's second in the memory queues.
+    issue();
 
     // ---- consumer state ----
     const int gq = lane >> 2, t4 = lane & 3;
@@ -482,6 +484,8 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                 }
             }
             begin_segment(k);
+            if (k == 0)
+                for (int kk = 1; kk < kDepth && kk < Rw; ++kk) issue();
             left = min(np - page, Rw - k);
         }
         --left;
