@@ -151,12 +151,17 @@ class Workload:
     def kv_bytes_per_layer(self, fmt):
         return self.sum_t * self.hkv * (BFP8_ROW if fmt == "bfp8" else BF16_ROW)
 
-    def _ingest_all(self, wire, stream, staged=False):
+    def _ingest_all(self, wire, stream, staged=False, layers=None):
         """Ingest every layer of the arriving request on `stream`.  With `staged`, each layer's pinned host bytes are
         first copied to a device staging buffer by the copy engine (same stream), then scattered from there."""
         hma = self.hma
         hs = self.hkv // 4
-        for l in range(self.L):
+        if layers is None:
+            todo = range(self.L)
+        else:       # `layers` layers per step, continuing where the previous step stopped (a request arriving over many steps)
+            todo = [(self._ingest_next + i) % self.L for i in range(layers)]
+            self._ingest_next = (self._ingest_next + layers) % self.L
+        for l in todo:
             src = wire[l]
             if staged:
                 with torch.cuda.stream(stream):
@@ -166,14 +171,16 @@ class Workload:
                                            hma.HMA_WIRE_TILE32, [s * hs for s in range(4)], [hs] * 4, self.spare, 0,
                                            self.ingest_tokens, stream)
 
-    def step(self, fmt="bfp8", ingest=True, host=False, staged=True):
+    _ingest_next = 0
+
+    def step(self, fmt="bfp8", ingest=True, host=False, staged=True, ingest_layers=None):
         """One decode pass over all layers (+ the concurrent ingest).  Everything is enqueued; nothing syncs."""
         hma = self.hma
         main = torch.cuda.current_stream(self.device)
         do_ingest = ingest and self.ingest_tokens and fmt == "bfp8"
         if do_ingest:
             self.side.wait_stream(main)
-            self._ingest_all(self.wire_host if host else self.wire_dev, self.side, staged=host and staged)
+            self._ingest_all(self.wire_host if host else self.wire_dev, self.side, staged=host and staged, layers=ingest_layers)
         cache = self.caches[fmt]
         for l in range(self.L):
             q = self.q[l]
@@ -406,6 +413,14 @@ def main():
     torch.cuda.synchronize(device)
 
     sec_decode_only = wl.time_steps(args.steps, args.warmup, ingest=False)
+    # the same request arriving at the rate of the paper's 100 Gb link (92.3 Gb/s measured, section 3.2): layers per step
+    paced = {}
+    if wl.ingest_tokens:
+        layer_bytes = 2 * 4 * wl.shard_bytes
+        per_step = max(1, int(round(92.3e9 / 8 * sec_decode_only / layer_bytes)))
+        sec_paced = wl.time_steps(args.steps, args.warmup, ingest_layers=per_step)
+        paced = {"layers_per_step": per_step, "link_gbit_s": 92.3, "ms_per_step": sec_paced * 1e3,
+                 "tokens_per_s": aggregate_value(wl.B, sec_paced, ws), "slowdown_vs_decode_only": sec_paced / sec_decode_only - 1.0}
     sec_e2e = wl.time_steps(max(2, args.steps // 4), 3, host=True)
     sec_e2e_mapped = wl.time_steps(max(2, args.steps // 4), 3, host=True, staged=False) if wl.ingest_tokens else sec_e2e
     extra = {}
@@ -451,6 +466,7 @@ def main():
                      "us_per_launch_median": call_med * 1e6, "us_per_launch_min": call_min * 1e6},
         "decode_only": {"tokens_per_s": aggregate_value(wl.B, sec_decode_only, ws), "ms_per_step": sec_decode_only * 1e3,
                         "kv_gbs": kv_step / sec_decode_only / 1e9, "slowdown_from_ingest": sec / sec_decode_only - 1.0},
+        "ingest_paced_at_link_rate": paced,
         "parity_sample": parity,
     }
     line.update(extra)
