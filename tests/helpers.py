@@ -96,3 +96,29 @@ def check_attention(out_f32, out_bf16, ref64):
     mb, rb = parity_metrics(got, ref64)
     assert (err <= 1e-2 + 2.0 ** -8 * np.abs(ref64)).all(), ("bf16 output bound", (err - 2.0 ** -8 * np.abs(ref64)).max())
     return ma, rl, mb, rb
+
+
+def parity_sample(wl):
+    """Outputs of the sequences a bench.Workload kept wire bytes of, against the oracle on those bytes, in the
+    full-size launch configuration.  The bar (max-abs 1e-2, rel-L2 2e-3) is taken on the F32 output; the BF16 output
+    must be exactly its rounding; the BF16 numbers and the oracle's own BF16 rounding floor are returned beside it."""
+    from oracle import oracle as orc
+    res = []
+    out32 = torch.empty((wl.B, wl.hq, 128), dtype=torch.float32, device=wl.device)
+    for (l, b), (kw, vw) in sorted(wl.sample_wires.items()):
+        c = wl.caches["bfp8"]
+        hma.hma_decode_attention(c, l, wl.q[l], out32, wl.table, wl.ctx, wl.sm_scale, wl.workspace)
+        hma.hma_decode_attention(c, l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wl.workspace)
+        torch.cuda.synchronize(wl.device)
+        qb = bf16_bits(wl.q[l][b:b + 1])
+        ref64, ref16 = orc.decode_attention(qb, [kw], [vw], wl.hkv, wl.sm_scale)
+        ref = ref64[0]
+        rel = lambda x: float(np.sqrt(((x - ref) ** 2).sum() / (ref ** 2).sum()))
+        g32 = out32[b].cpu().numpy().astype(np.float64)
+        g16 = wl.out[l][b].float().cpu().numpy().astype(np.float64)
+        res.append({"layer": l, "seq": b, "context": int(wl.lens[b]),
+                    "f32_max_abs": float(np.abs(g32 - ref).max()), "f32_rel_l2": rel(g32),
+                    "bf16_max_abs": float(np.abs(g16 - ref).max()), "bf16_rel_l2": rel(g16),
+                    "bf16_is_rne_of_f32": bool(torch.equal(out32[b].to(torch.bfloat16), wl.out[l][b])),
+                    "bf16_floor_rel_l2": rel(bf16_bits_to_f64(ref16[0]))})
+    return res
