@@ -156,7 +156,7 @@ hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32
  *   context_lens device int32 [batch]; every entry <= max_pages_per_seq*16
  *   workspace    device, 256-byte aligned, >= hma_decode_attention_workspace_bytes(...) bytes;
  *                contents need no initialisation and are clobbered
- *   batch        at most 2048 (HMA_ERR_UNSUPPORTED_SHAPE beyond)
+ *   batch        at most 1024 (HMA_ERR_UNSUPPORTED_SHAPE beyond)
  * Accuracy: fp32 accumulation; element exponents above 250 are outside the supported range.
  * Launches: two kernels per call (attention, then a small merge of the per-worker partials), both with
  * programmatic stream serialisation; each waits on the grid dependency before it reads any input, so the

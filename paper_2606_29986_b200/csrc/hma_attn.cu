@@ -42,7 +42,8 @@ struct Geo {
 constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile: o[8][128], m[8], l[8]
 constexpr uint32_t kSpinLimit = 1u << 20;           // polls of a bounded wait
 constexpr uint32_t kSuspendNs = 2000;              // a failed poll may keep the thread parked this long
-constexpr int kMaxBatch = 2048;
+constexpr int kMaxBatch = 1024;
+constexpr int kSegCost = 2;                        // what starting a segment costs a warp, in records (Q load, partial tile)
 constexpr int kMaxCtas = 160;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
 constexpr int kMinRecords = 4;                    // fewest records a worker takes
 constexpr int kMaxDevices = 64;
@@ -57,7 +58,8 @@ struct AttnArgs {
     const int32_t *ctx;
     int batch;
     float sm_scale;
-    int32_t *cum;                   // workspace: pages before each sequence, batch + 1 entries (for the merge kernel)
+    int32_t *cum;                   // workspace: pages before each sequence, then pages + segment costs before each
+                                    // sequence, batch + 1 entries each (for the merge kernel)
     float *tiles;                   // workspace: partial tiles
 };
 
@@ -222,8 +224,9 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     uint8_t *scratch = ring + kStages * kRecord;                                  // kWarps x kScratch (BFP8 only)
     uint64_t *bars = reinterpret_cast<uint64_t *>(scratch + kWarps * Geo<kFmt>::scratch);   // full[kStages]
     int *stage_ok = reinterpret_cast<int *>(bars + kStages);                      // [kStages]
-    int *misc = stage_ok + kStages;                                               // [0] abort word, [16..] scan scratch
-    int *cum = misc + 16 + kThreads;                                              // [batch + 1]
+    int *misc = stage_ok + kStages;                                               // [0] abort word, [16..80) scan scratch
+    int *cum = misc + 16 + 64;                                                    // [batch + 1] pages before each sequence
+    int *ecum = cum + a.batch + 1;                                                // [batch + 1] same, plus kSegCost per non-empty sequence
     volatile int *abort_word = misc;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -238,45 +241,54 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     // The kernel is launched with programmatic stream serialisation: its CTAs may be placed while the previous
     // kernel of the stream drains.  Nothing that a predecessor could have written is read before this wait.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // exclusive prefix of pages per sequence: each thread owns `per` consecutive sequences, warps scan with
-    // shuffles, one warp scans the warp totals
+    // Exclusive prefixes per sequence of (pages) and of (pages + kSegCost if the sequence is not empty): each thread
+    // owns `per` consecutive sequences, warps scan with shuffles, one warp scans the warp totals.
     {
         const int per = (B + kThreads - 1) / kThreads;
         const int b0 = min(B, tid * per), b1 = min(B, b0 + per);
-        int mine = 0;
-        for (int b = b0; b < b1; ++b) mine += pages_of(a, b);
-        int incl = mine;                                   // inclusive scan inside the warp
+        int mine = 0, emine = 0;
+        for (int b = b0; b < b1; ++b) { const int n = pages_of(a, b); mine += n; emine += n ? n + kSegCost : 0; }
+        int incl = mine, eincl = emine;                    // inclusive scans inside the warp
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-            if (lane >= d) incl += v;
+            const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d), ev = __shfl_up_sync(0xFFFFFFFFu, eincl, d);
+            if (lane >= d) { incl += v; eincl += ev; }
         }
-        if (lane == 31) misc[16 + warp] = incl;
+        if (lane == 31) { misc[16 + warp] = incl; misc[16 + 32 + warp] = eincl; }
         __syncthreads();
         if (warp == 0) {
             int tot = lane < kWarps ? misc[16 + lane] : 0, run = tot;
+            int etot = lane < kWarps ? misc[16 + 32 + lane] : 0, erun = etot;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                const int v = __shfl_up_sync(0xFFFFFFFFu, run, d);
-                if (lane >= d) run += v;
+                const int v = __shfl_up_sync(0xFFFFFFFFu, run, d), ev = __shfl_up_sync(0xFFFFFFFFu, erun, d);
+                if (lane >= d) { run += v; erun += ev; }
             }
-            if (lane < kWarps) misc[16 + lane] = run - tot;              // pages before each warp's sequences
-            if (lane == kWarps - 1) cum[B] = run;
+            if (lane < kWarps) { misc[16 + lane] = run - tot; misc[16 + 32 + lane] = erun - etot; }
+            if (lane == kWarps - 1) { cum[B] = run; ecum[B] = erun; }
         }
         __syncthreads();
-        int run = misc[16 + warp] + incl - mine;
-        for (int b = b0; b < b1; ++b) { cum[b] = run; run += pages_of(a, b); }
+        int run = misc[16 + warp] + incl - mine, erun = misc[16 + 32 + warp] + eincl - emine;
+        for (int b = b0; b < b1; ++b) {
+            const int n = pages_of(a, b);
+            cum[b] = run; ecum[b] = erun;
+            run += n; erun += n ? n + kSegCost : 0;
+        }
         __syncthreads();
     }
     // let the merge kernel be scheduled already; it blocks in griddepcontrol.wait until this grid has finished
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (blockIdx.x == 0 && kMode == 0)
-        for (int b = tid; b <= B; b += kThreads) a.cum[b] = cum[b];
+        for (int b = tid; b <= B; b += kThreads) { a.cum[b] = cum[b]; a.cum[B + 1 + b] = ecum[b]; }
     // from here on the warps never synchronise with one another
     const int64_t W = (int64_t)Hkv * cum[B];
-    // Workers are numbered across SMs first.  Small batches use fewer workers, at least kMinRecords records
+    // The work list is cut by cost, not by record count: every (sequence, kv head) segment is charged kSegCost
+    // extra units at its start, so a warp whose range crosses a segment boundary (a second Q load, a second partial
+    // tile) gets that many records fewer.  WX is the list's length in cost units.
+    const int64_t WX = (int64_t)Hkv * ecum[B];
+    // Workers are numbered across SMs first.  Small batches use fewer workers, at least kMinRecords units
     // each, so that a segment is never cut into more partials than it is worth.
-    const int64_t NWK = max((int64_t)1, min((int64_t)gridDim.x * kWarps, W / kMinRecords));
+    const int64_t NWK = max((int64_t)1, min((int64_t)gridDim.x * kWarps, WX / kMinRecords));
     const int64_t u = (int64_t)warp * gridDim.x + blockIdx.x;      // this warp's worker index
 
     if (kMode == 0)                                               // empty sequences get rows of zeros
@@ -285,7 +297,20 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                 for (int i = lane; i < Hq * kHeadDim; i += 32) store_out(a, b * Hq * kHeadDim + i, 0.f);
 
     if (u >= NWK) return;
-    const int64_t wlo = u * W / NWK, whi = (u + 1) * W / NWK;
+    // number of records that lie before cost position p
+    auto records_before = [&](int64_t p) -> int64_t {
+        if (p >= WX) return W;
+        int lo = 0, hi = B - 1;
+        while (lo < hi) {   // largest b with Hkv*ecum[b] <= p: the (non-empty) sequence that holds p
+            const int mid = (lo + hi + 1) >> 1;
+            if ((int64_t)Hkv * ecum[mid] <= p) lo = mid; else hi = mid - 1;
+        }
+        const int n = cum[lo + 1] - cum[lo];
+        const int64_t off = p - (int64_t)Hkv * ecum[lo];
+        const int gg = (int)(off / (n + kSegCost)), r = (int)(off - (int64_t)gg * (n + kSegCost));
+        return (int64_t)Hkv * cum[lo] + (int64_t)gg * n + max(0, r - kSegCost);
+    };
+    const int64_t wlo = records_before(u * WX / NWK), whi = records_before((u + 1) * WX / NWK);
     if (wlo >= whi) return;
     const int Rw = (int)(whi - wlo);
 
@@ -724,10 +749,12 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int m
     if (h >= G) return;
     const int np = a.cum[b + 1] - a.cum[b];
     if (np == 0) return;                                         // rows of empty sequences were zeroed by the main kernel
-    const int64_t W = (int64_t)Hkv * a.cum[a.batch];
-    const int64_t NWK = max((int64_t)1, min((int64_t)max_workers, W / kMinRecords));
-    const int64_t ws = (int64_t)Hkv * a.cum[b] + (int64_t)g * np, we = ws + np;
-    const int64_t u0 = ((ws + 1) * NWK - 1) / W, u1 = (we * NWK - 1) / W;     // first and last worker of the segment
+    // the main kernel cut the work list by cost (kSegCost units at the start of every segment, then one per record)
+    const int32_t *ecum = a.cum + a.batch + 1;
+    const int64_t WX = (int64_t)Hkv * ecum[a.batch];
+    const int64_t NWK = max((int64_t)1, min((int64_t)max_workers, WX / kMinRecords));
+    const int64_t first = (int64_t)Hkv * ecum[b] + (int64_t)g * (np + kSegCost) + kSegCost;   // cost position of the first record
+    const int64_t u0 = ((first + 1) * NWK - 1) / WX, u1 = ((first + np) * NWK - 1) / WX;       // first and last worker of the segment
     if (u0 == u1) return;
     const float *t0 = a.tiles + (int64_t)blockIdx.x * kTileFloats;           // part i is at t0 + i * kTileFloats
     float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -809,11 +836,11 @@ template <int kFmt>
 static size_t attn_smem_bytes(int batch)
 {
     using G = Geo<kFmt>;
-    return (size_t)G::stages * G::record + (size_t)G::warps * G::scratch + G::stages * 8 + G::stages * 4 + (16 + G::threads) * 4 +
-           ((size_t)batch + 1) * 4;
+    return (size_t)G::stages * G::record + (size_t)G::warps * G::scratch + G::stages * 8 + G::stages * 4 + (16 + 64) * 4 +
+           ((size_t)batch + 1) * 8;
 }
 
-static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 4 + 255) & ~(size_t)255; }
+static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 8 + 255) & ~(size_t)255; }
 
 }  // namespace hma
 
@@ -939,7 +966,7 @@ extern "C" hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_
 // below until the process exits.
 namespace hma {
 constexpr int kStaticMaxSegments = 512;       // batch * num_kv_heads
-constexpr size_t kStaticWsBytes = 4096 + (size_t)(kMaxCtas * kWarps + kStaticMaxSegments) * kTileFloats * 4;   // 12.2 MiB
+constexpr size_t kStaticWsBytes = 8192 + (size_t)(kMaxCtas * kWarps + kStaticMaxSegments) * kTileFloats * 4;   // 12.2 MiB
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 static void *g_static_ws_ptr[kMaxDevices];    // device address of g_static_ws on each device, resolved on first use
 }  // namespace hma
