@@ -246,7 +246,20 @@ class Workload:
         e1.record()
         torch.cuda.synchronize(self.device)
         elems = 2 * self.L * T * self.hkv * 128
-        return e0.elapsed_time(e1) / 1e3 / reps, elems * (17 / 16 + 2), elems
+        fused = e0.elapsed_time(e1) / 1e3 / reps
+        # the elementwise strawman, layer by layer and tensor by tensor
+        def naive():
+            for l in range(self.L):
+                for which in (0, 1):
+                    self.hma.hma_bfp8_dequant_bf16_naive(cache, l, which, pages, 0, T, out[l, which])
+        naive()
+        torch.cuda.synchronize(self.device)
+        e0.record()
+        naive()
+        e1.record()
+        torch.cuda.synchronize(self.device)
+        self.naive_rebuild_s = e0.elapsed_time(e1) / 1e3
+        return fused, elems * (17 / 16 + 2), elems
 
 # ----------------------------------------------------------------------------- ranks
 def world():
@@ -405,6 +418,7 @@ def main():
     t_rb, rb_bytes, rb_elems = wl.time_rebuild()
     extra["rebuild_request"] = {"ms": t_rb * 1e3, "tokens": int(wl.lens[0]), "layers": wl.L, "gbs": rb_bytes / t_rb / 1e9,
                                 "frac_of_peak": rb_bytes / t_rb / 1e9 / peak, "calls": 1,
+                                "naive_elementwise_ms": wl.naive_rebuild_s * 1e3, "fused_speedup_over_naive": wl.naive_rebuild_s / t_rb,
                                 "what": "hma_bfp8_rebuild_request: one request, K and V, all layers, one launch (1.0625 B in + 2 B out per element)"}
     kv_step = wl.kv_bytes_per_layer("bfp8") * wl.L
     value = aggregate_value(wl.B, sec, ws)

@@ -236,6 +236,13 @@ hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t layer, int3
 hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const int32_t *page_ids, int64_t token_begin,
                                       int64_t n_tokens, void *out_bf16, void *stream);
 
+/* The "naive elementwise reconstruction" that section 3.3 measures the fused rebuild against (72 ms vs 1.5 ms on the
+ * paper's A100): same arguments and the same bits as hma_bfp8_dequant_bf16, computed one thread per element with byte
+ * loads.  A comparison point for the benchmark, not a product path. */
+hma_status_t hma_bfp8_dequant_bf16_naive(const hma_cache_t *cache, int32_t layer, int32_t which,
+                                         const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
+                                         void *out_bf16, void *stream);
+
 /* Flat variant: n_blocks blocks, exps[i] with mants[16*i .. 16*i+15] -> out_bf16[16*i ..] (device pointers). */
 hma_status_t hma_bfp8_dequant_blocks_bf16(const uint8_t *exps, const uint8_t *mants, int64_t n_blocks,
                                           void *out_bf16, void *stream);

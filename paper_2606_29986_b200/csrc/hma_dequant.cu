@@ -120,6 +120,32 @@ __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int wh
     }
 }
 
+// The elementwise strawman of section 3.3 ("naive elementwise reconstruction"): one thread per output element, byte
+// loads straight from the cache, integer bit assembly, two-byte stores.  Kept only as the comparison point.
+__global__ void __launch_bounds__(256) dequant_naive_kernel(CacheView cv, int which, const int32_t *__restrict__ page_ids,
+                                                            int64_t token_begin, int64_t n_tokens, uint16_t *__restrict__ out)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_tokens * cv.num_kv_heads * kHeadDim) return;
+    const int ch = (int)(i % kHeadDim), h = (int)((i / kHeadDim) % cv.num_kv_heads);
+    const int64_t gt = token_begin + i / ((int64_t)kHeadDim * cv.num_kv_heads);
+    const int tok = (int)(gt % kPageTokens);
+    const int32_t pid = page_ids[gt / kPageTokens - token_begin / kPageTokens];
+    uint32_t bits = 0;
+    if (pid >= 0 && pid < cv.num_pages) {
+        const uint8_t *rec = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)record_bytes(cv.format);
+        if (cv.format == HMA_KV_BFP8)
+            bits = which == 0 ? bfp8_to_bf16_bits(rec[bfp8_k_exp_off(tok, ch >> 4)], rec[bfp8_k_el_off(tok, ch)])
+                              : bfp8_to_bf16_bits(rec[bfp8_v_exp_off(tok, ch >> 4)], rec[bfp8_v_el_off(tok, ch)]);
+        else
+            bits = *reinterpret_cast<const uint16_t *>(rec + (which == 0 ? bf16_k_el_off(tok, ch) : bf16_v_el_off(tok, ch)));
+    } else {
+        atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_DEQUANT);
+    }
+    const int oc = which == 0 ? key_channel_of_query(ch, cv.key_layout) : ch;
+    out[(i / kHeadDim) * kHeadDim + oc] = (uint16_t)bits;
+}
+
 }  // namespace hma
 
 extern "C" hma_status_t hma_bfp8_dequant_blocks_bf16(const uint8_t *exps, const uint8_t *mants, int64_t n_blocks,
@@ -176,6 +202,25 @@ extern "C" hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const
     dim3 grid((unsigned)n_pages, (unsigned)cache->desc.num_kv_heads, (unsigned)(2 * cache->desc.num_layers));
     hma::dequant_paged_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, 0, page_ids, token_begin, n_tokens,
                                                                       (uint16_t *)out_bf16, cache->d_layers);
+    hma::count_launch();
+    HMA_CUDA_OK(cudaGetLastError());
+    return HMA_OK;
+}
+
+extern "C" hma_status_t hma_bfp8_dequant_bf16_naive(const hma_cache_t *cache, int32_t layer, int32_t which,
+                                                    const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
+                                                    void *out_bf16, void *stream)
+{
+    if (!cache || layer < 0 || layer >= cache->desc.num_layers || (which != 0 && which != 1) || token_begin < 0 || n_tokens < 0)
+        return HMA_ERR_INVALID_ARG;
+    if (n_tokens == 0) return HMA_OK;
+    if (!page_ids || !out_bf16) return HMA_ERR_INVALID_ARG;
+    const int64_t total = n_tokens * cache->desc.num_kv_heads * hma::kHeadDim;
+    if ((total + 255) / 256 > 0x7FFFFFFF) return HMA_ERR_INVALID_ARG;
+    hma::CacheView cv{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
+                      cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
+    hma::dequant_naive_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(cv, which, page_ids, token_begin,
+                                                                                                 n_tokens, (uint16_t *)out_bf16);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;

@@ -77,6 +77,8 @@ def lib():
         L.hma_decode_attention_simple.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
         L.hma_bfp8_dequant_bf16.restype = i32
         L.hma_bfp8_dequant_bf16.argtypes = [vp, i32, i32, vp, i64, i64, vp, vp]
+        L.hma_bfp8_dequant_bf16_naive.restype = i32
+        L.hma_bfp8_dequant_bf16_naive.argtypes = [vp, i32, i32, vp, i64, i64, vp, vp]
         L.hma_bfp8_rebuild_request.restype = i32
         L.hma_bfp8_rebuild_request.argtypes = [vp, vp, i64, i64, vp, vp]
         L.hma_bfp8_encode_rows.restype = i32
@@ -223,6 +225,12 @@ def hma_decode_attention_simple(cache, layer, q, out, block_table, context_lens,
 def hma_bfp8_dequant_bf16(cache, layer, which, page_ids, token_begin, n_tokens, out_bf16, stream=None):
     _check(lib().hma_bfp8_dequant_bf16(cache.handle, layer, which, _ptr(page_ids), token_begin, n_tokens,
                                        _ptr(out_bf16), _stream(stream)), "hma_bfp8_dequant_bf16")
+
+
+def hma_bfp8_dequant_bf16_naive(cache, layer, which, page_ids, token_begin, n_tokens, out_bf16, stream=None):
+    """Elementwise strawman of hma_bfp8_dequant_bf16 (same bits, one thread per element)."""
+    _check(lib().hma_bfp8_dequant_bf16_naive(cache.handle, layer, which, _ptr(page_ids), token_begin, n_tokens,
+                                             _ptr(out_bf16), _stream(stream)), "hma_bfp8_dequant_bf16_naive")
 
 
 def hma_bfp8_rebuild_request(cache, page_ids, token_begin, n_tokens, out_bf16, stream=None):

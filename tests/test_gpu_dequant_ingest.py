@@ -130,7 +130,12 @@ def test_whole_request_rebuild_in_one_launch(fmt):
         pages = sc.table[b, first:last + 1].contiguous()
         out = torch.zeros((3, 2, n, 4, 128), dtype=torch.bfloat16, device="cuda")
         hma.hma_bfp8_rebuild_request(sc.cache, pages, t0, n, out)
+        naive = torch.zeros_like(out)
+        for l in range(3):
+            for which in (0, 1):
+                hma.hma_bfp8_dequant_bf16_naive(sc.cache, l, which, pages, t0, n, naive[l, which])
         torch.cuda.synchronize()
+        assert torch.equal(naive, out)                     # the elementwise strawman produces the same bits
         got = bf16_bits(out)
         for l in range(3):
             wk = orc.relayout_keys_to_half_split(orc.decode_rowmajor_bf16(sc.k_wires[l][b][:, t0:t0 + n]))
