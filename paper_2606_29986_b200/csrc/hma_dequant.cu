@@ -8,13 +8,11 @@ namespace hma {
 // Four elements of one block -> four BF16 bit patterns, bit-exact for every (E, byte) pair.
 // The byte s<<7|m is first spread to the FP16 pattern s<<15|m, the FP16 subnormal +-m * 2^-24 (two integer
 // instructions per pair: section 3.3's "shifts, masks, ORs and a bitcast"); widening to fp32 and multiplying by
-// 2^(E-109), split in two exact power-of-two factors so that every E in 0..255 stays in range, gives
+// 2^(E-109) (one factor while it is a normal fp32 number, two exact power-of-two factors above that) gives
 // m * 2^(E-133) exactly (fp32 subnormals and overflow to Inf included); its upper 16 bits are the BF16 value.
 // The sign rides along, so m = 0 keeps its sign.
 __device__ __forceinline__ uint2 dequant4(uint32_t w, uint32_t E)
 {
-    const float s1 = __uint_as_float(((E >> 1) + 73u) << 23);           // 2^(floor(E/2) - 54)
-    const float s2 = __uint_as_float(((E - (E >> 1)) + 72u) << 23);     // 2^(ceil(E/2) - 55)
     uint32_t h01, h23;
     asm("prmt.b32 %0, %1, 0, 0x1100;" : "=r"(h01) : "r"(w));
     asm("prmt.b32 %0, %1, 0, 0x3322;" : "=r"(h23) : "r"(w));
@@ -22,8 +20,18 @@ __device__ __forceinline__ uint2 dequant4(uint32_t w, uint32_t E)
     h23 &= 0x807F807Fu;
     const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&h01));
     const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&h23));
-    const uint32_t b0 = __float_as_uint((f01.x * s1) * s2), b1 = __float_as_uint((f01.y * s1) * s2);
-    const uint32_t b2 = __float_as_uint((f23.x * s1) * s2), b3 = __float_as_uint((f23.y * s1) * s2);
+    uint32_t b0, b1, b2, b3;
+    if (E <= 236u) {
+        // 2^(E-109) is a normal fp32 number: one exact multiplication (results below 2^-126 are exact subnormals)
+        const float sc = __uint_as_float((E + 18u) << 23);
+        b0 = __float_as_uint(f01.x * sc); b1 = __float_as_uint(f01.y * sc);
+        b2 = __float_as_uint(f23.x * sc); b3 = __float_as_uint(f23.y * sc);
+    } else {
+        const float s1 = __uint_as_float(((E >> 1) + 73u) << 23);           // 2^(floor(E/2) - 54)
+        const float s2 = __uint_as_float(((E - (E >> 1)) + 72u) << 23);     // 2^(ceil(E/2) - 55)
+        b0 = __float_as_uint((f01.x * s1) * s2); b1 = __float_as_uint((f01.y * s1) * s2);
+        b2 = __float_as_uint((f23.x * s1) * s2); b3 = __float_as_uint((f23.y * s1) * s2);
+    }
     return make_uint2(__byte_perm(b0, b1, 0x7632), __byte_perm(b2, b3, 0x7632));
 }
 
@@ -43,9 +51,8 @@ __global__ void __launch_bounds__(256) dequant_blocks_kernel(const uint8_t *__re
 }
 
 // One CTA per (logical page of the request, kv head): the K or V half record is staged in shared memory, then each
-// thread rebuilds 4 consecutive channels of one token at a time and stores 8 bytes.  (One CTA per page covering all
+// thread rebuilds 8 consecutive channels of one token at a time and stores 16 bytes.  (One CTA per page covering all
 // heads was measured slower: too few threads in flight for a copy-like kernel.)
-constexpr int kDequantHeads = 1;
 // With `layers` set, blockIdx.z = 2 * layer + which selects the layer and the tensor, and the output is
 // [num_layers][2][n_tokens][Hkv][128]: the whole request in one launch.
 __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int which, const int32_t *__restrict__ page_ids,
@@ -57,7 +64,7 @@ __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int wh
         which = blockIdx.z & 1;
         out += (int64_t)blockIdx.z * n_tokens * cv.num_kv_heads * kHeadDim;
     }
-    __shared__ __align__(16) uint8_t recs[kDequantHeads][kBf16Half];
+    __shared__ __align__(16) uint8_t recs[1][kBf16Half];
     const int64_t first_page = token_begin / kPageTokens;
     const int64_t lp = first_page + blockIdx.x;
     const int32_t pid = page_ids[blockIdx.x];
@@ -77,44 +84,52 @@ __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int wh
             }
         }
         __syncthreads();
-        for (int item = threadIdx.x; item < kPageTokens * nh * 32; item += blockDim.x) {
-            const int c0 = (item & 31) * 4;                             // channels c0 .. c0+3
-            const int hh = (item >> 5) % nh, tok = (item >> 5) / nh;    // items ordered like the output: token, head, channel
+        for (int item = threadIdx.x; item < kPageTokens * 16; item += blockDim.x) {
+            const int tok = item >> 4, c0 = (item & 15) * 8;             // channels c0 .. c0+7 of token tok: half a block
             const int64_t gt = lp * kPageTokens + tok;
             if (gt < token_begin || gt >= token_begin + n_tokens) continue;
-            const uint8_t *rec = recs[hh];
-            uint2 o = make_uint2(0u, 0u);
+            const uint8_t *rec = recs[0];
+            uint2 lo = make_uint2(0u, 0u), hi = lo;                     // channels c0..c0+3 and c0+4..c0+7 as BF16 pairs
             if (!bad) {
                 // `rec` holds one half record: offsets below are relative to the start of that half
                 if (cv.format == HMA_KV_BFP8) {
-                    uint32_t w, E;
+                    uint32_t w0, w1, E;
                     if (which == 0) {
                         E = rec[bfp8_k_exp_off(tok, c0 >> 4)];
-                        w = *reinterpret_cast<const uint32_t *>(rec + bfp8_k_el_off(tok, c0));   // four channels are one word
+                        const uint8_t *p = rec + bfp8_k_el_off(tok, c0);           // four channels are one word, the next four 16 bytes on
+                        w0 = *reinterpret_cast<const uint32_t *>(p);
+                        w1 = *reinterpret_cast<const uint32_t *>(p + 16);
                     } else {
+                        // consecutive channels of a token sit 64 bytes apart, at the token's byte position
+                        const uint8_t *p = rec + (bfp8_v_el_off(tok, c0) - kBfp8Half);
                         E = rec[bfp8_v_exp_off(tok, c0 >> 4) - kBfp8Half];
-                        w = rec[bfp8_v_el_off(tok, c0) - kBfp8Half] | (rec[bfp8_v_el_off(tok, c0 + 1) - kBfp8Half] << 8) |
-                            (rec[bfp8_v_el_off(tok, c0 + 2) - kBfp8Half] << 16) |
-                            ((uint32_t)rec[bfp8_v_el_off(tok, c0 + 3) - kBfp8Half] << 24);
+                        w0 = p[0] | (p[64] << 8) | (p[128] << 16) | ((uint32_t)p[192] << 24);
+                        w1 = p[256] | (p[320] << 8) | (p[384] << 16) | ((uint32_t)p[448] << 24);
                     }
-                    o = dequant4(w, E);
+                    lo = dequant4(w0, E);
+                    hi = dequant4(w1, E);
                 } else if (which == 0) {
-                    o = *reinterpret_cast<const uint2 *>(rec + bf16_k_el_off(tok, c0));            // four channels are 8 bytes
+                    const uint8_t *p = rec + bf16_k_el_off(tok, c0);               // four channels are 8 bytes, the next four 16 bytes on
+                    lo = *reinterpret_cast<const uint2 *>(p);
+                    hi = *reinterpret_cast<const uint2 *>(p + 16);
                 } else {
-                    uint32_t e[4];
+                    uint32_t e[8];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) e[k] = *reinterpret_cast<const uint16_t *>(rec + bf16_v_el_off(tok, c0 + k) - kBf16Half);
-                    o = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
+                    for (int k = 0; k < 8; ++k) e[k] = *reinterpret_cast<const uint16_t *>(rec + bf16_v_el_off(tok, c0 + k) - kBf16Half);
+                    lo = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
+                    hi = make_uint2(e[4] | (e[5] << 16), e[6] | (e[7] << 16));
                 }
             }
-            uint16_t *row = out + ((gt - token_begin) * cv.num_kv_heads + h0 + hh) * kHeadDim;
+            uint16_t *row = out + ((gt - token_begin) * cv.num_kv_heads + blockIdx.y) * kHeadDim;
             if (relayout) {
                 // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout):
-                // cached channels c0, c0+2 go to c0/2, c0/2+1; cached channels c0+1, c0+3 to 64 + c0/2, 64 + c0/2 + 1
-                *reinterpret_cast<uint32_t *>(row + (c0 >> 1)) = (o.x & 0xFFFFu) | (o.y << 16);
-                *reinterpret_cast<uint32_t *>(row + 64 + (c0 >> 1)) = (o.x >> 16) | (o.y & 0xFFFF0000u);
+                // cached channels c0, c0+2, .. go to c0/2 .., cached channels c0+1, c0+3, .. to 64 + c0/2 ..
+                *reinterpret_cast<uint2 *>(row + (c0 >> 1)) =
+                    make_uint2((lo.x & 0xFFFFu) | (lo.y << 16), (hi.x & 0xFFFFu) | (hi.y << 16));
+                *reinterpret_cast<uint2 *>(row + 64 + (c0 >> 1)) =
+                    make_uint2((lo.x >> 16) | (lo.y & 0xFFFF0000u), (hi.x >> 16) | (hi.y & 0xFFFF0000u));
             } else {
-                *reinterpret_cast<uint2 *>(row + c0) = o;
+                *reinterpret_cast<uint4 *>(row + c0) = make_uint4(lo.x, lo.y, hi.x, hi.y);
             }
         }
     }
