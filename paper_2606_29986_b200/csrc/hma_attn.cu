@@ -4,9 +4,9 @@
 // Shape of the kernel
 //   * persistent grid, one CTA of 16 warps per SM (four warps per SM sub-partition, 128 registers each).
 //     All (sequence, kv head, page) records of the batch form one linear work list that is cut into
-//     equal contiguous ranges, one per *warp* (no tail effect, any mix of context lengths, no barrier
-//     between warps).  A warp that holds only part of a (sequence, kv head) segment writes a partial
-//     (max, sum, 128-vector) per q head; a small second kernel, launched with programmatic dependent
+//     contiguous ranges of equal cost, one per *warp* (any mix of context lengths, no barrier between
+//     warps; starting a segment is charged like two records).  A warp that holds only part of a
+//     (sequence, kv head) segment writes a partial (max, sum, 128-vector) per q head; a small second kernel, launched with programmatic dependent
 //     launch so that its launch latency hides behind the main kernel, merges the partials in worker
 //     order (fixed order, so results are bitwise repeatable).
 //   * every warp feeds itself: it keeps three 4352-byte page records in flight with 1-D bulk async
