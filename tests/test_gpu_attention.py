@@ -176,3 +176,43 @@ def test_argument_errors():
     with pytest.raises(hma.HmaError) as e:
         hma.hma_decode_attention(sc.cache, 0, sc.q.view(-1)[1:].view(torch.bfloat16), out, sc.table, sc.ctx, 0.1, sc.workspace)
     assert e.value.status == hma.HMA_ERR_ALIGNMENT
+
+
+def test_concurrent_ingest_on_a_side_stream_leaves_decode_untouched():
+    """A new request's layers land in spare pages on a side stream while decode runs: decode output stays bitwise the
+    same, and afterwards the new request attends and rebuilds correctly (section 3.2: transfer overlaps compute)."""
+    from oracle import oracle as orc
+    lens = [3000, 1500, 700, 4000]
+    new_T = 1000
+    sc = Scenario(lens, 32, 8, seed=111, permute=True, layers=2, extra_pages=(new_T + 15) // 16)
+    quiet = [bf16_bits(sc.attention(l, torch.bfloat16)) for l in range(2)]
+    kw = [synth.make_kv_wire(8, new_T, 7000 + l) for l in range(2)]
+    vw = [synth.make_kv_wire(8, new_T, 7100 + l) for l in range(2)]
+    kt = [[synth.rowmajor_to_tile32(w[2 * s:2 * s + 2].contiguous()).cuda() for s in range(4)] for w in kw]
+    vt = [[synth.rowmajor_to_tile32(w[2 * s:2 * s + 2].contiguous()).cuda() for s in range(4)] for w in vw]
+    spare = torch.from_numpy(np.ascontiguousarray(sc.spare)).cuda()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    outs = []
+    for rep in range(6):
+        for l in range(2):
+            hma.hma_kv_ingest_layer_shards(sc.cache, l, kt[l], vt[l], hma.HMA_WIRE_TILE32, [0, 2, 4, 6], [2] * 4, spare, 0, new_T, side)
+            out = torch.empty((len(lens), 32, 128), dtype=torch.bfloat16, device="cuda")
+            hma.hma_decode_attention(sc.cache, l, sc.q, out, sc.table, sc.ctx, 1.0 / np.sqrt(128.0), sc.workspace)
+            outs.append((l, out))
+    torch.cuda.synchronize()
+    for l, out in outs:
+        assert np.array_equal(bf16_bits(out), quiet[l])
+    assert hma.hma_error_flags(sc.cache) == 0
+    # the request that arrived meanwhile joins the batch
+    table = torch.full((1, spare.numel()), -1, dtype=torch.int32, device="cuda")
+    table[0] = spare
+    ctx = torch.tensor([new_T], dtype=torch.int32, device="cuda")
+    q = synth.make_q(1, 32, 112).cuda()
+    for l in range(2):
+        out = torch.empty((1, 32, 128), dtype=torch.float32, device="cuda")
+        hma.hma_decode_attention(sc.cache, l, q, out, table, ctx, 1.0 / np.sqrt(128.0), sc.workspace)
+        torch.cuda.synchronize()
+        ref64, _ = orc.decode_attention(bf16_bits(q), [kw[l].numpy()], [vw[l].numpy()], 8)
+        ma, rl = parity_metrics(out.cpu().numpy(), ref64)
+        assert ma <= 1e-2 and rl <= 2e-3
