@@ -216,3 +216,20 @@ def test_concurrent_ingest_on_a_side_stream_leaves_decode_untouched():
         ref64, _ = orc.decode_attention(bf16_bits(q), [kw[l].numpy()], [vw[l].numpy()], 8)
         ma, rl = parity_metrics(out.cpu().numpy(), ref64)
         assert ma <= 1e-2 and rl <= 2e-3
+
+
+def test_context_longer_than_the_block_table_is_clamped_and_many_kv_heads():
+    """context_lens beyond max_pages_per_seq * 16 are clamped to what the table can address; 16 kv heads work."""
+    from oracle import oracle as orc
+    sc = Scenario([64, 48], 32, 16, seed=121)
+    ctx = torch.tensor([10_000, 48], dtype=torch.int32, device="cuda")       # the table has 4 pages per sequence
+    out = torch.empty((2, 32, 128), dtype=torch.float32, device="cuda")
+    hma.hma_decode_attention(sc.cache, 0, sc.q, out, sc.table, ctx, 1.0 / np.sqrt(128.0), sc.workspace)
+    torch.cuda.synchronize()
+    ref64, _ = sc.oracle()
+    ma, rl = parity_metrics(out.cpu().numpy(), ref64)
+    assert ma <= 1e-2 and rl <= 2e-3 and hma.hma_error_flags(sc.cache) == 0
+    neg = torch.tensor([-5, 48], dtype=torch.int32, device="cuda")           # a negative length counts as empty
+    hma.hma_decode_attention(sc.cache, 0, sc.q, out, sc.table, neg, 1.0 / np.sqrt(128.0), sc.workspace)
+    torch.cuda.synchronize()
+    assert not out[0].any() and parity_metrics(out[1:].cpu().numpy(), ref64[1:])[1] <= 2e-3
