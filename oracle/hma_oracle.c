@@ -253,6 +253,65 @@ void orc_decode_attention(const uint16_t *q_bf16, const uint8_t *k_wire, const u
         }
 }
 
+/* Decode attention over a context whose first prefix_lens[b] tokens are BFP8 wire bytes (as above) and whose
+ * last tail_lens[b] tokens are plain BF16 values: KV made on the decode GPU, which the paper keeps in BF16
+ * (section 3.1), appended to the prefix that arrived from the prefill accelerator.  One softmax over all tokens.
+ *   k_tail, v_tail  BF16 bit patterns; sequence b starts at element tail_off[b], laid out [Hkv][tail_lens[b]][128]
+ * Keys of both parts are in the queries' head-dim order. */
+void orc_decode_attention_mixed(const uint16_t *q_bf16, const uint8_t *k_wire, const uint8_t *v_wire,
+                                const int64_t *wire_off, const int32_t *prefix_lens,
+                                const uint16_t *k_tail, const uint16_t *v_tail, const int64_t *tail_off,
+                                const int32_t *tail_lens, int32_t B, int32_t Hq, int32_t Hkv, double sm_scale,
+                                double *out_f64, uint16_t *out_bf16)
+{
+    const int G = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t h = 0; h < Hq; ++h) {
+            const int64_t T = prefix_lens[b], S = tail_lens[b], N = T + S;
+            const int32_t g = h / G;
+            double q[ORC_HEAD_DIM], o[ORC_HEAD_DIM];
+            for (int d = 0; d < ORC_HEAD_DIM; ++d) {
+                q[d] = orc_bf16_to_f64(q_bf16[((int64_t)b * Hq + h) * ORC_HEAD_DIM + d]);
+                o[d] = 0.0;
+            }
+            if (N > 0) {
+                const uint8_t *kr = k_wire + wire_off[b] + (int64_t)g * T * ORC_ROW_BYTES;
+                const uint8_t *vr = v_wire + wire_off[b] + (int64_t)g * T * ORC_ROW_BYTES;
+                const uint16_t *kt = k_tail + tail_off[b] + (int64_t)g * S * ORC_HEAD_DIM;
+                const uint16_t *vt = v_tail + tail_off[b] + (int64_t)g * S * ORC_HEAD_DIM;
+                double *s = (double *)malloc((size_t)N * sizeof(double));
+                double smax = -INFINITY;
+                for (int64_t t = 0; t < N; ++t) {
+                    double acc = 0.0;
+                    for (int d = 0; d < ORC_HEAD_DIM; ++d) {
+                        double kv = t < T ? bfp8_value(kr[t * ORC_ROW_BYTES + d / ORC_BLOCK], kr[t * ORC_ROW_BYTES + ORC_BLOCKS_PER_ROW + d])
+                                          : orc_bf16_to_f64(kt[(t - T) * ORC_HEAD_DIM + d]);
+                        acc += q[d] * kv;
+                    }
+                    s[t] = sm_scale * acc;
+                    if (s[t] > smax) smax = s[t];
+                }
+                double denom = 0.0;
+                for (int64_t t = 0; t < N; ++t) { s[t] = exp(s[t] - smax); denom += s[t]; }
+                for (int64_t t = 0; t < N; ++t) {
+                    double p = s[t] / denom;
+                    for (int d = 0; d < ORC_HEAD_DIM; ++d) {
+                        double vv = t < T ? bfp8_value(vr[t * ORC_ROW_BYTES + d / ORC_BLOCK], vr[t * ORC_ROW_BYTES + ORC_BLOCKS_PER_ROW + d])
+                                          : orc_bf16_to_f64(vt[(t - T) * ORC_HEAD_DIM + d]);
+                        o[d] += p * vv;
+                    }
+                }
+                free(s);
+            }
+            for (int d = 0; d < ORC_HEAD_DIM; ++d) {
+                int64_t idx = ((int64_t)b * Hq + h) * ORC_HEAD_DIM + d;
+                if (out_f64) out_f64[idx] = o[d];
+                if (out_bf16) out_bf16[idx] = orc_f64_to_bf16(o[d]);
+            }
+        }
+}
+
 int orc_num_threads(void)
 {
     int n = 1;

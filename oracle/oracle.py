@@ -173,6 +173,34 @@ def decode_attention(q_bf16, k_wires, v_wires, num_kv_heads, sm_scale=None, want
     return out64, out16
 
 
+def decode_attention_mixed(q_bf16, k_wires, v_wires, k_tails, v_tails, num_kv_heads, sm_scale=None):
+    """fp64 decode attention over BFP8 prefixes followed by BF16 tails.
+
+    k_wires, v_wires : list of B uint8 arrays [Hkv][T_b][136]
+    k_tails, v_tails : list of B uint16 arrays [Hkv][S_b][128] (BF16 bit patterns), S_b may be 0
+    returns (out_f64, out_bf16)."""
+    q_bf16 = np.ascontiguousarray(q_bf16, np.uint16)
+    B, Hq, D = q_bf16.shape
+    if sm_scale is None:
+        sm_scale = 1.0 / np.sqrt(HEAD_DIM)
+    lens = np.array([w.shape[1] for w in k_wires], np.int32)
+    tl = np.array([t.shape[1] for t in k_tails], np.int32)
+    offs = np.zeros(B, np.int64)
+    offs[1:] = np.cumsum([num_kv_heads * int(t) * ROW_BYTES for t in lens])[:-1]
+    toffs = np.zeros(B, np.int64)
+    toffs[1:] = np.cumsum([num_kv_heads * int(t) * HEAD_DIM for t in tl])[:-1]
+    kcat = np.concatenate([np.ascontiguousarray(w, np.uint8).reshape(-1) for w in k_wires] + [np.zeros(1, np.uint8)])
+    vcat = np.concatenate([np.ascontiguousarray(w, np.uint8).reshape(-1) for w in v_wires] + [np.zeros(1, np.uint8)])
+    ktc = np.concatenate([np.ascontiguousarray(t, np.uint16).reshape(-1) for t in k_tails] + [np.zeros(1, np.uint16)])
+    vtc = np.concatenate([np.ascontiguousarray(t, np.uint16).reshape(-1) for t in v_tails] + [np.zeros(1, np.uint16)])
+    out64 = np.empty((B, Hq, D), np.float64)
+    out16 = np.empty((B, Hq, D), np.uint16)
+    lib().orc_decode_attention_mixed(_p(q_bf16), _p(kcat), _p(vcat), _p(offs), _p(lens), _p(ktc), _p(vtc), _p(toffs), _p(tl),
+                                     ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(num_kv_heads),
+                                     ctypes.c_double(sm_scale), _p(out64), _p(out16))
+    return out64, out16
+
+
 def half_split_index(c):
     """Half-split position of interleaved-order channel c (the key re-layout of section 3.3)."""
     lib().orc_half_split_index.restype = ctypes.c_int32

@@ -154,3 +154,34 @@ def test_attention_with_interleaved_keys_equals_attention_in_one_layout():
     assert np.array_equal(o_int, o_same)
     o_plain, _ = orc.decode_attention(q, kw, vw, 2)
     assert not np.allclose(o_int, o_plain)                                     # and the flag does change the result
+
+
+def test_mixed_prefix_and_bf16_tail():
+    """BFP8 prefix + BF16 tail: equals the plain oracle when the tail is empty or when the tail holds the BF16 decode of
+    BFP8 bytes, and equals float64 library attention over the concatenated values."""
+    q, kw, vw = _case(2, 8, 2, [21, 7], 12)
+    empty = [np.zeros((2, 0, 128), np.uint16)] * 2
+    o_plain, b_plain = orc.decode_attention(q, kw, vw, 2, sm_scale=0.2)
+    o_mix, b_mix = orc.decode_attention_mixed(q, kw, vw, empty, empty, 2, sm_scale=0.2)
+    assert np.array_equal(o_plain, o_mix) and np.array_equal(b_plain, b_mix)
+    # split every sequence: the first part stays BFP8, the rest is handed over as its exact BF16 decode
+    cut = [9, 0]
+    kp = [w[:, :c] for w, c in zip(kw, cut)]
+    vp = [w[:, :c] for w, c in zip(vw, cut)]
+    kt = [orc.decode_rowmajor_bf16(w[:, c:]) for w, c in zip(kw, cut)]
+    vt = [orc.decode_rowmajor_bf16(w[:, c:]) for w, c in zip(vw, cut)]
+    o_split, _ = orc.decode_attention_mixed(q, kp, vp, kt, vt, 2, sm_scale=0.2)
+    assert np.allclose(o_split, o_plain, rtol=1e-13, atol=1e-15)
+    # a genuinely BF16 tail (values BFP8 cannot hold) against the float64 library routine
+    rng = np.random.default_rng(13)
+    tails = [(rng.standard_normal((2, s, 128)).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16) for s in (5, 12)]
+    tails_v = [(rng.standard_normal((2, s, 128)).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16) for s in (5, 12)]
+    o_m, _ = orc.decode_attention_mixed(q, kw, vw, tails, tails_v, 2, sm_scale=0.2)
+    for b in range(2):
+        K = np.concatenate([_np_values(kw[b]), _bf16_to_f64(tails[b])], axis=1)
+        V = np.concatenate([_np_values(vw[b]), _bf16_to_f64(tails_v[b])], axis=1)
+        Kt = torch.from_numpy(K).repeat_interleave(4, dim=0)
+        Vt = torch.from_numpy(V).repeat_interleave(4, dim=0)
+        Q = torch.from_numpy(_bf16_to_f64(q[b]))[:, None, :]
+        ref = torch.nn.functional.scaled_dot_product_attention(Q[None], Kt[None], Vt[None], scale=0.2)[0, :, 0].numpy()
+        assert np.allclose(o_m[b], ref, rtol=1e-10, atol=1e-12)
