@@ -228,6 +228,37 @@ class Workload:
         t = np.array([a.elapsed_time(b) for a, b in evs]) / 1e3
         return float(t.mean()), float(np.median(t)), float(t.min())
 
+    def time_mixed(self, tail_tokens=64, reps=3):
+        """hma_decode_attention_mixed: the BFP8 cache as prefix plus a BF16 cache holding `tail_tokens` decode-side tokens per
+        sequence (plain BF16 rows); mean seconds per call."""
+        hma = self.hma
+        lens = np.full(self.B, tail_tokens, np.int32)
+        table, num_pages, _ = synth.block_table(lens, True, 99)
+        tail = hma.KVCache(hma.make_desc(self.L, self.hq, self.hkv, num_pages, hma.HMA_KV_BF16), self.device)
+        ttable, tlens = torch.from_numpy(table).to(self.device), torch.from_numpy(lens).to(self.device)
+        g = torch.Generator(device=self.device)
+        g.manual_seed(99)
+        rows = torch.randn((self.hkv, tail_tokens, 128), generator=g, device=self.device).to(torch.bfloat16)
+        for l in range(self.L):
+            for b in range(self.B):
+                hma.hma_kv_ingest_layer(tail, l, rows, rows, hma.HMA_WIRE_BF16_ROWS, 0, self.hkv, ttable[b].contiguous(), 0, tail_tokens)
+        ws = torch.empty(2 * (hma.hma_decode_attention_workspace_bytes(self.caches["bfp8"].desc, self.B) + 256), dtype=torch.uint8,
+                         device=self.device)
+
+        def run():
+            for l in range(self.L):
+                hma.hma_decode_attention_mixed(self.caches["bfp8"], tail, l, self.q[l], self.out[l], self.table, self.ctx, ttable, tlens,
+                                               self.sm_scale, ws)
+        run()
+        torch.cuda.synchronize(self.device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record()
+        torch.cuda.synchronize(self.device)
+        return e0.elapsed_time(e1) / 1e3 / reps / self.L
+
     def time_rebuild(self, reps=3):
         """One-shot BFP8 -> BF16 rebuild of one whole request (sequence 0: every layer, K and V): seconds, bytes moved."""
         T = int(self.lens[0])
@@ -420,6 +451,10 @@ def main():
                                 "frac_of_peak": rb_bytes / t_rb / 1e9 / peak, "calls": 1,
                                 "naive_elementwise_ms": wl.naive_rebuild_s * 1e3, "fused_speedup_over_naive": wl.naive_rebuild_s / t_rb,
                                 "what": "hma_bfp8_rebuild_request: one request, K and V, all layers, one launch (1.0625 B in + 2 B out per element)"}
+    t_mixed = wl.time_mixed()
+    extra["mixed_prefix_tail"] = {"us_per_call": t_mixed * 1e6, "tail_tokens_per_sequence": 64,
+                                  "what": "hma_decode_attention_mixed: BFP8 prefix cache + BF16 cache with 64 decode-side tokens per sequence",
+                                  "overhead_vs_prefix_only": t_mixed / call_mean - 1.0}
     kv_step = wl.kv_bytes_per_layer("bfp8") * wl.L
     value = aggregate_value(wl.B, sec, ws)
     achieved = wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9

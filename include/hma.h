@@ -52,7 +52,7 @@ typedef enum {
 } hma_status_t;
 
 typedef enum { HMA_KV_BFP8 = 0, HMA_KV_BF16 = 1 } hma_kv_format_t;
-typedef enum { HMA_WIRE_TILE32 = 0, HMA_WIRE_ROWMAJOR = 1 } hma_wire_layout_t;
+typedef enum { HMA_WIRE_TILE32 = 0, HMA_WIRE_ROWMAJOR = 1, HMA_WIRE_BF16_ROWS = 2 } hma_wire_layout_t;
 typedef enum { HMA_OUT_BF16 = 0, HMA_OUT_F32 = 1 } hma_out_dtype_t;
 /* Head-dim order of the cached keys relative to the queries (section 3.3: the prefill accelerator writes post-RoPE
  * keys with rotary pairs interleaved, (2i, 2i+1); FlashAttention-style decoders use the half-split order, (i, i+64)).
@@ -121,6 +121,8 @@ void hma_cache_destroy(hma_cache_t *cache);
  *                   HMA_WIRE_TILE32:   [head][ceil(n_tokens/32)][4][1088 B]: a 32-token x 32-channel
  *                     tile = four 16x16 faces ordered (row half, column half); exponents at
  *                     face*16 + row%16, elements at 64 + face*256 + (row%16)*16 + col%16.
+ *                   HMA_WIRE_BF16_ROWS (BF16 caches only): [head][token][128] plain BF16 values, KV that was
+ *                     made on the decode GPU itself (the paper keeps decode in BF16, section 3.1).
  *                   Both pointers 16-byte aligned.
  *   page_ids        device int32: page_ids[i] = physical page of the request's logical page
  *                   floor(token_begin/16) + i; ceil((token_begin%16 + n_tokens)/16) entries.
@@ -203,6 +205,22 @@ hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer
                                          const int32_t *block_table, int32_t max_pages_per_seq,
                                          const int32_t *context_lens, int32_t batch, float sm_scale,
                                          void *stream);
+
+/*
+ * Decode attention over two caches: the first prefix_lens[b] tokens of sequence b are pages of `prefix` (the BFP8
+ * KV that arrived from the prefill accelerator), the next tail_lens[b] tokens are pages of `tail` (a BF16 cache
+ * holding the KV of tokens generated since, which the paper's decode side produces in BF16, section 3.1; the
+ * paper does not say where those live, this is one answer, hma_bfp8_encode_rows the other).  One softmax over
+ * both.  Same q/out/sm_scale conventions as hma_decode_attention; both caches must have the same head counts and
+ * HMA_KEYS_AS_QUERIES.  workspace: 2 * hma_decode_attention_workspace_bytes(desc, batch), rounded up to 256 each.
+ * Three launches: attention over each cache leaving partials, then a merge that completes the softmax.
+ */
+hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
+                                        const void *q, void *out, int32_t out_dtype,
+                                        const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,
+                                        const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens,
+                                        int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes,
+                                        void *stream);
 
 /* Bandwidth probe: streams exactly the page records hma_decode_attention would read (same block
  * tables, same work split, same bulk-copy ring) and does no arithmetic and no output.  Its time is

@@ -61,6 +61,7 @@ struct AttnArgs {
     int32_t *cum;                   // workspace: pages before each sequence, then pages + segment costs before each
                                     // sequence, batch + 1 entries each (for the merge kernel)
     float *tiles;                   // workspace: partial tiles
+    int always_partial;             // 1: never write `out`; every segment leaves partial tiles (two-cache attention)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -291,7 +292,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     const int64_t NWK = max((int64_t)1, min((int64_t)gridDim.x * kWarps, WX / kMinRecords));
     const int64_t u = (int64_t)warp * gridDim.x + blockIdx.x;      // this warp's worker index
 
-    if (kMode == 0)                                               // empty sequences get rows of zeros
+    if (kMode == 0 && !a.always_partial)                          // empty sequences get rows of zeros
         for (int64_t b = u; b < B; b += NWK)
             if (cum[b + 1] == cum[b])
                 for (int i = lane; i < Hq * kHeadDim; i += 32) store_out(a, b * Hq * kHeadDim + i, 0.f);
@@ -398,7 +399,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         np = cum[b + 1] - cum[b];
         T = min(a.ctx[b], a.max_pages * kPageTokens);
         tail = T - (np - 1) * kPageTokens;
-        whole = page == 0 && Rw - k >= np;
+        whole = page == 0 && Rw - k >= np && !a.always_partial;
         // Q fragments of this (sequence, kv head): FP16, one power-of-two scale per head
         float f[8][4];
         float amax = 0.f;
@@ -832,6 +833,91 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int m
     }
 }
 
+// Merge for attention over two caches (a BFP8 prefix and a BF16 tail of every sequence): both main kernels ran with
+// always_partial, so every segment of either cache left one partial tile per worker that touched it; the softmax is
+// completed over the parts of both, prefix parts first, in worker order.  One CTA per (sequence, kv head), one warp
+// per q head, four channels per lane.
+struct MergeSource {
+    const int32_t *cum;      // pages, then pages + segment costs, before each sequence
+    const float *tiles;
+    int max_workers;
+};
+
+__device__ __forceinline__ void segment_workers(const MergeSource &s, int batch, int Hkv, int b, int g, int64_t *u0, int *count)
+{
+    const int np = s.cum[b + 1] - s.cum[b];
+    *count = 0;
+    *u0 = 0;
+    if (np == 0) return;
+    const int32_t *ecum = s.cum + batch + 1;
+    const int64_t WX = (int64_t)Hkv * ecum[batch];
+    const int64_t NWK = max((int64_t)1, min((int64_t)s.max_workers, WX / kMinRecords));
+    const int64_t first = (int64_t)Hkv * ecum[b] + (int64_t)g * (np + kSegCost) + kSegCost;
+    *u0 = ((first + 1) * NWK - 1) / WX;
+    *count = (int)(((first + np) * NWK - 1) / WX - *u0 + 1);
+}
+
+__global__ void __launch_bounds__(256) attn_merge_mixed_kernel(const AttnArgs a, MergeSource sa, MergeSource sb)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
+    const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, h = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (h >= G) return;
+    int64_t ua, ub;
+    int pa, pb;
+    segment_workers(sa, a.batch, Hkv, b, g, &ua, &pa);
+    segment_workers(sb, a.batch, Hkv, b, g, &ub, &pb);
+    const int P = pa + pb;
+    auto part = [&](int j) -> const float * {
+        return j < pa ? sa.tiles + (ua + j + blockIdx.x) * kTileFloats : sb.tiles + (ub + (j - pa) + blockIdx.x) * kTileFloats;
+    };
+    float M = -INFINITY;
+    for (int c0 = 0; c0 < P; c0 += 32) {
+        float mm = c0 + lane < P ? __ldcg(part(c0 + lane) + 8 * kHeadDim + h) : -INFINITY;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, d));
+        M = fmaxf(M, mm);
+    }
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+    for (int c0 = 0; c0 < P; c0 += 32) {
+        float wgt = 0.f, dsum = 0.f;
+        if (c0 + lane < P) {
+            const float *pt = part(c0 + lane);
+            const float mm = __ldcg(pt + 8 * kHeadDim + h);
+            wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
+            dsum = wgt * __ldcg(pt + 8 * kHeadDim + 8 + h);
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) dsum += __shfl_xor_sync(0xFFFFFFFFu, dsum, d);     // fixed butterfly order
+        den += dsum;
+        const int cnt = min(32, P - c0);
+        for (int j0 = 0; j0 < cnt; j0 += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+                v[jj] = j0 + jj < cnt ? __ldcg(reinterpret_cast<const float4 *>(part(c0 + j0 + jj) + h * kHeadDim) + lane)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const float wj = __shfl_sync(0xFFFFFFFFu, wgt, (j0 + jj) & 31);
+                num.x = fmaf(wj, v[jj].x, num.x); num.y = fmaf(wj, v[jj].y, num.y);
+                num.z = fmaf(wj, v[jj].z, num.z); num.w = fmaf(wj, v[jj].w, num.w);
+            }
+        }
+    }
+    const float inv = den > 0.f ? 1.f / den : 0.f;       // no tokens in either cache: a row of zeros
+    const int64_t oi = ((int64_t)b * Hq + (int64_t)g * G + h) * kHeadDim + 4 * lane;
+    if (a.out_dtype == HMA_OUT_F32) {
+        reinterpret_cast<float4 *>(a.out)[oi >> 2] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+    } else {
+        const uint32_t lo = f32_to_bf16_rne(num.x * inv) | ((uint32_t)f32_to_bf16_rne(num.y * inv) << 16);
+        const uint32_t hi = f32_to_bf16_rne(num.z * inv) | ((uint32_t)f32_to_bf16_rne(num.w * inv) << 16);
+        reinterpret_cast<uint2 *>(a.out)[oi >> 2] = make_uint2(lo, hi);
+    }
+}
+
 template <int kFmt>
 static size_t attn_smem_bytes(int batch)
 {
@@ -854,7 +940,7 @@ extern "C" size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *d
 static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, const void *q, void *out, int32_t out_dtype,
                                      const int32_t *block_table, int32_t max_pages_per_seq, const int32_t *context_lens,
                                      int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes, void *stream,
-                                     int probe)
+                                     int probe, int always_partial = 0, hma::AttnArgs *args_out = nullptr, int *workers_out = nullptr)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || batch < 0 || max_pages_per_seq < 0) return HMA_ERR_INVALID_ARG;
     if (out_dtype != HMA_OUT_BF16 && out_dtype != HMA_OUT_F32) return HMA_ERR_INVALID_ARG;
@@ -900,6 +986,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.sm_scale = sm_scale;
     a.cum = (int32_t *)workspace;
     a.tiles = (float *)((uint8_t *)workspace + hma::cum_bytes(batch));
+    a.always_partial = always_partial;
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
     constexpr int tb = hma::Geo<HMA_KV_BFP8>::threads, tf = hma::Geo<HMA_KV_BF16>::threads;
@@ -921,7 +1008,9 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     else if (probe == 1) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BFP8>, a));
     else HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<2, HMA_KV_BFP8>, a));
     hma::count_launch();
-    if (probe) return HMA_OK;
+    if (args_out) *args_out = a;
+    if (workers_out) *workers_out = n_ctas * (bf16 ? hma::Geo<HMA_KV_BF16>::warps : hma::Geo<HMA_KV_BFP8>::warps);
+    if (probe || always_partial) return HMA_OK;
     cfg.gridDim = dim3((unsigned)(batch * cache->desc.num_kv_heads));
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = 0;
@@ -938,6 +1027,45 @@ extern "C" hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t l
 {
     return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
                             workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
+                                                   const void *q, void *out, int32_t out_dtype,
+                                                   const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,
+                                                   const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens,
+                                                   int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes,
+                                                   void *stream)
+{
+    if (!prefix || !tail) return HMA_ERR_INVALID_ARG;
+    if (prefix->desc.num_q_heads != tail->desc.num_q_heads || prefix->desc.num_kv_heads != tail->desc.num_kv_heads ||
+        prefix->desc.key_layout != HMA_KEYS_AS_QUERIES || tail->desc.key_layout != HMA_KEYS_AS_QUERIES)
+        return HMA_ERR_UNSUPPORTED_SHAPE;
+    if (layer < 0 || layer >= tail->desc.num_layers) return HMA_ERR_INVALID_ARG;
+    if (batch == 0) return HMA_OK;
+    const size_t half = (hma_decode_attention_workspace_bytes(&prefix->desc, batch) + 255) & ~(size_t)255;
+    if (!workspace) return HMA_ERR_INVALID_ARG;
+    if (workspace_bytes < 2 * half) return HMA_ERR_WORKSPACE_TOO_SMALL;
+    hma::AttnArgs aa, ab;
+    int wa = 0, wb = 0;
+    hma_status_t st = launch_attention(prefix, layer, q, out, out_dtype, prefix_table, prefix_max_pages, prefix_lens, batch, sm_scale,
+                                       workspace, half, stream, 0, 1, &aa, &wa);
+    if (st != HMA_OK) return st;
+    st = launch_attention(tail, layer, q, out, out_dtype, tail_table, tail_max_pages, tail_lens, batch, sm_scale,
+                          (uint8_t *)workspace + half, half, stream, 0, 1, &ab, &wb);
+    if (st != HMA_OK) return st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(batch * prefix->desc.num_kv_heads));
+    cfg.blockDim = dim3(256);
+    cfg.stream = (cudaStream_t)stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    hma::MergeSource sa{aa.cum, aa.tiles, wa}, sb{ab.cum, ab.tiles, wb};
+    HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_mixed_kernel, aa, sa, sb));
+    hma::count_launch();
+    return HMA_OK;
 }
 
 extern "C" hma_status_t hma_kv_read_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,

@@ -133,6 +133,35 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
     }
 }
 
+// Plain BF16 rows ([head][token][128], KV made on the decode GPU) into a BF16 cache: one CTA per (page, head).
+// K: two consecutive channels of a token are one word of the record; V: single elements (tokens pair up in a word).
+__global__ void __launch_bounds__(128) ingest_bf16_rows_kernel(CacheView cv, IngestArgs a)
+{
+    int shard = 0, hs = blockIdx.y;
+    while (shard + 1 < a.n_shards && hs >= a.head_count[shard]) hs -= a.head_count[shard++];
+    const int h = a.head_begin[shard] + hs;
+    const int64_t lp = a.token_begin / kPageTokens + blockIdx.x;
+    const int32_t pid = a.page_ids[blockIdx.x];
+    if (pid < 0 || pid >= cv.num_pages) {
+        if (threadIdx.x == 0) atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_INGEST);
+        return;
+    }
+    int lo = 0, hi = kPageTokens;
+    if (lp * kPageTokens < a.token_begin) lo = (int)(a.token_begin - lp * kPageTokens);
+    if ((lp + 1) * kPageTokens > a.token_begin + a.n_tokens) hi = (int)(a.token_begin + a.n_tokens - lp * kPageTokens);
+    uint8_t *rec = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)kBf16Record;
+    const uint16_t *kw = reinterpret_cast<const uint16_t *>(a.k_wire[shard]), *vw = reinterpret_cast<const uint16_t *>(a.v_wire[shard]);
+    for (int i = threadIdx.x; i < kPageTokens * 64; i += blockDim.x) {
+        const int tok = i >> 6, ch = (i & 63) * 2;
+        if (tok < lo || tok >= hi) continue;
+        const int64_t row = ((int64_t)hs * a.n_tokens + (lp * kPageTokens + tok - a.token_begin)) * kHeadDim;
+        *reinterpret_cast<uint32_t *>(rec + bf16_k_el_off(tok, ch)) = *reinterpret_cast<const uint32_t *>(kw + row + ch);
+        const uint32_t v2 = *reinterpret_cast<const uint32_t *>(vw + row + ch);
+        *reinterpret_cast<uint16_t *>(rec + bf16_v_el_off(tok, ch)) = (uint16_t)v2;
+        *reinterpret_cast<uint16_t *>(rec + bf16_v_el_off(tok, ch + 1)) = (uint16_t)(v2 >> 16);
+    }
+}
+
 }  // namespace hma
 
 static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_shards, const void *const *k_wires,
@@ -141,7 +170,8 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
                                   void *stream)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers) return HMA_ERR_INVALID_ARG;
-    if (wire_layout != HMA_WIRE_TILE32 && wire_layout != HMA_WIRE_ROWMAJOR) return HMA_ERR_INVALID_ARG;
+    if (wire_layout != HMA_WIRE_TILE32 && wire_layout != HMA_WIRE_ROWMAJOR && wire_layout != HMA_WIRE_BF16_ROWS) return HMA_ERR_INVALID_ARG;
+    if (wire_layout == HMA_WIRE_BF16_ROWS && cache->desc.format != HMA_KV_BF16) return HMA_ERR_INVALID_ARG;
     if (n_shards < 1 || n_shards > hma::kMaxShards || !k_wires || !v_wires || !head_begins || !head_counts) return HMA_ERR_INVALID_ARG;
     if (token_begin < 0 || n_tokens < 0) return HMA_ERR_INVALID_ARG;
     hma::IngestArgs a = {};
@@ -177,7 +207,8 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
     a.n_tokens = n_tokens;
     a.layout = wire_layout;
     dim3 grid((unsigned)n_pages, (unsigned)heads);
-    hma::ingest_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, a);
+    if (wire_layout == HMA_WIRE_BF16_ROWS) hma::ingest_bf16_rows_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, a);
+    else hma::ingest_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;

@@ -17,7 +17,7 @@ HMA_ERR_INVALID_ARG, HMA_ERR_UNSUPPORTED_SHAPE, HMA_ERR_ALIGNMENT = 1, 2, 3
 HMA_ERR_WORKSPACE_TOO_SMALL, HMA_ERR_CUDA, HMA_ERR_DEVICE_FLAGGED = 4, 5, 6
 HMA_ERR_STATIC_LIMIT = 7
 HMA_KV_BFP8, HMA_KV_BF16 = 0, 1
-HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR = 0, 1
+HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR, HMA_WIRE_BF16_ROWS = 0, 1, 2
 HMA_OUT_BF16, HMA_OUT_F32 = 0, 1
 HMA_KEYS_AS_QUERIES, HMA_KEYS_INTERLEAVED = 0, 1
 HMA_FLAG_BAD_PAGE_ATTENTION, HMA_FLAG_BAD_PAGE_INGEST, HMA_FLAG_BAD_PAGE_DEQUANT, HMA_FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
@@ -73,6 +73,8 @@ def lib():
         L.hma_kv_read_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
         L.hma_attention_alu_probe.restype = i32
         L.hma_attention_alu_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
+        L.hma_decode_attention_mixed.restype = i32
+        L.hma_decode_attention_mixed.argtypes = [vp, vp, i32, vp, vp, i32, vp, i32, vp, vp, i32, vp, i32, f32, vp, sz, vp]
         L.hma_decode_attention_simple.restype = i32
         L.hma_decode_attention_simple.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
         L.hma_bfp8_dequant_bf16.restype = i32
@@ -213,6 +215,17 @@ def hma_attention_alu_probe(cache, layer, block_table, context_lens, workspace, 
     _check(lib().hma_attention_alu_probe(cache.handle, layer, _ptr(block_table), block_table.shape[1], _ptr(context_lens),
                                          context_lens.shape[0], _ptr(workspace), workspace.numel() * workspace.element_size(),
                                          _stream(stream)), "hma_attention_alu_probe")
+
+
+def hma_decode_attention_mixed(prefix, tail, layer, q, out, prefix_table, prefix_lens, tail_table, tail_lens, sm_scale,
+                               workspace, stream=None):
+    """Attention over a BFP8 prefix cache and a BF16 tail cache (see include/hma.h)."""
+    out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
+    _check(lib().hma_decode_attention_mixed(prefix.handle, tail.handle, layer, _ptr(q), _ptr(out), out_dtype,
+                                            _ptr(prefix_table), prefix_table.shape[1], _ptr(prefix_lens),
+                                            _ptr(tail_table), tail_table.shape[1], _ptr(tail_lens), q.shape[0],
+                                            float(sm_scale), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                            _stream(stream)), "hma_decode_attention_mixed")
 
 
 def hma_decode_attention_simple(cache, layer, q, out, block_table, context_lens, sm_scale, stream=None):
