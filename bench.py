@@ -228,6 +228,28 @@ class Workload:
         t = np.array([a.elapsed_time(b) for a, b in evs]) / 1e3
         return float(t.mean()), float(np.median(t)), float(t.min())
 
+    def time_ingest(self, reps=5):
+        """GPU time of the ingest alone (device-resident wire, every layer of the arriving request), replayed from a CUDA
+        graph so that host launch overhead does not count; seconds per layer."""
+        s = torch.cuda.Stream(self.device)
+        s.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.stream(s):
+            self._ingest_all(self.wire_dev, s)
+            torch.cuda.synchronize(self.device)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                self._ingest_all(self.wire_dev, s)
+            g.replay()
+            torch.cuda.synchronize(self.device)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize(self.device)
+        torch.cuda.current_stream(self.device).wait_stream(s)
+        return e0.elapsed_time(e1) / 1e3 / reps / self.L
+
     def time_mixed(self, tail_tokens=64, reps=3):
         """hma_decode_attention_mixed: the BFP8 cache as prefix plus a BF16 cache holding `tail_tokens` decode-side tokens per
         sequence (plain BF16 rows); mean seconds per call."""
@@ -451,6 +473,12 @@ def main():
                                 "frac_of_peak": rb_bytes / t_rb / 1e9 / peak, "calls": 1,
                                 "naive_elementwise_ms": wl.naive_rebuild_s * 1e3, "fused_speedup_over_naive": wl.naive_rebuild_s / t_rb,
                                 "what": "hma_bfp8_rebuild_request: one request, K and V, all layers, one launch (1.0625 B in + 2 B out per element)"}
+    if wl.ingest_tokens:
+        t_ing = wl.time_ingest()
+        layer_bytes = 2 * 4 * wl.shard_bytes
+        extra["ingest_alone"] = {"us_per_layer": t_ing * 1e6, "gbs_read_plus_write": 2 * layer_bytes / t_ing / 1e9,
+                                 "frac_of_peak": 2 * layer_bytes / t_ing / 1e9 / peak,
+                                 "what": "hma_kv_ingest_layer_shards, one 8192-token layer (4 shards, TILE32), device-resident wire, CUDA-graph replay"}
     t_mixed = wl.time_mixed()
     extra["mixed_prefix_tail"] = {"us_per_call": t_mixed * 1e6, "tail_tokens_per_sequence": 64,
                                   "what": "hma_decode_attention_mixed: BFP8 prefix cache + BF16 cache with 64 decode-side tokens per sequence",

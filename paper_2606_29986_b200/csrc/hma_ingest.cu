@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
     if (lp * kPageTokens < a.token_begin) lo = (int)(a.token_begin - lp * kPageTokens);
     if ((lp + 1) * kPageTokens > a.token_begin + a.n_tokens) hi = (int)(a.token_begin + a.n_tokens - lp * kPageTokens);
     const bool row16 = a.layout == HMA_WIRE_TILE32;   // tile faces are 16-byte aligned; 136-byte rows only 8
+    const bool exp_fast = lo == 0 && hi == kPageTokens && (a.token_begin & 15) == 0;
     for (int item = threadIdx.x; item < 2 * kPageTokens * kBlocksPerRow; item += blockDim.x) {
         const int t = item >> 7 & 1, tok = (item >> 3) & 15, j = item & 7;
         if (tok < lo || tok >= hi) continue;
@@ -67,7 +68,26 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
             *reinterpret_cast<uint2 *>(dst) = *reinterpret_cast<const uint2 *>(w + mo);
             *reinterpret_cast<uint2 *>(dst + 8) = *reinterpret_cast<const uint2 *>(w + mo + 8);
         }
-        rows[t][tok][j] = w[eo];
+        if (!exp_fast) rows[t][tok][j] = w[eo];
+    }
+    if (exp_fast) {
+        // whole page, page-aligned in the wire: the exponents come in 16-byte (tile face) or 8-byte (row) pieces
+        const int64_t wt0 = lp * kPageTokens - a.token_begin;
+        if (row16 && threadIdx.x < 16) {
+            const int t = threadIdx.x >> 3, j = threadIdx.x & 7;
+            const uint8_t *w = t ? a.v_wire[shard] : a.k_wire[shard];
+            int64_t eo;
+            (void)wire_block_off(a.layout, a.n_tokens, hs, wt0, j, &eo);
+            const uint4 e = *reinterpret_cast<const uint4 *>(w + eo);
+            const uint32_t ew[4] = {e.x, e.y, e.z, e.w};
+#pragma unroll
+            for (int tok = 0; tok < kPageTokens; ++tok) rows[t][tok][j] = (uint8_t)(ew[tok >> 2] >> (8 * (tok & 3)));
+        } else if (!row16 && threadIdx.x < 32) {
+            const int t = threadIdx.x >> 4, tok = threadIdx.x & 15;
+            const uint8_t *w = t ? a.v_wire[shard] : a.k_wire[shard];
+            *reinterpret_cast<uint2 *>(&rows[t][tok][0]) =
+                *reinterpret_cast<const uint2 *>(w + ((int64_t)hs * a.n_tokens + wt0 + tok) * kRowBytes);
+        }
     }
     __syncthreads();
     uint8_t *rec = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)record_bytes(cv.format);
@@ -99,17 +119,28 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
             put(rv + w, val, vmask(tq));
         }
         for (int wi = threadIdx.x; wi < 512; wi += blockDim.x) {
+            // K elements: four consecutive channels of one token are one word of the record
             const int c = wi >> 7, lane = (wi >> 2) & 31, w4 = wi & 3, g = lane >> 2, tq = lane & 3;
-            {   // K elements: four consecutive channels of one token
-                const int tok = g + 8 * (c & 1), ch = 16 * (4 * (c >> 1) + w4) + 4 * tq;
-                put(rk + 32 + wi, *reinterpret_cast<const uint32_t *>(&rows[0][tok][16 + ch]), tok >= lo && tok < hi ? 0xFFFFFFFFu : 0u);
-            }
-            {   // V elements: one channel of four tokens
-                const int ch = 16 * (2 * c + (w4 >> 1)) + g + 8 * (w4 & 1);
-                const uint32_t val = rows[1][2 * tq][16 + ch] | (rows[1][2 * tq + 1][16 + ch] << 8) |
-                                     (rows[1][2 * tq + 8][16 + ch] << 16) | ((uint32_t)rows[1][2 * tq + 9][16 + ch] << 24);
-                put(rv + 32 + wi, val, vmask(tq));
-            }
+            const int tok = g + 8 * (c & 1), ch = 16 * (4 * (c >> 1) + w4) + 4 * tq;
+            put(rk + 32 + wi, *reinterpret_cast<const uint32_t *>(&rows[0][tok][16 + ch]), tok >= lo && tok < hi ? 0xFFFFFFFFu : 0u);
+        }
+        for (int it = threadIdx.x; it < 128; it += blockDim.x) {
+            // V elements: a 4-token x 4-channel block is read as four words (one per token) and transposed in registers
+            // into four words of the record (one per channel)
+            const int tq = it >> 5, ch0 = (it & 31) * 4;
+            const uint32_t w0 = *reinterpret_cast<const uint32_t *>(&rows[1][2 * tq][16 + ch0]);
+            const uint32_t w1 = *reinterpret_cast<const uint32_t *>(&rows[1][2 * tq + 1][16 + ch0]);
+            const uint32_t w2 = *reinterpret_cast<const uint32_t *>(&rows[1][2 * tq + 8][16 + ch0]);
+            const uint32_t w3 = *reinterpret_cast<const uint32_t *>(&rows[1][2 * tq + 9][16 + ch0]);
+            const uint32_t a01 = __byte_perm(w0, w1, 0x5140), b01 = __byte_perm(w0, w1, 0x7362);
+            const uint32_t a23 = __byte_perm(w2, w3, 0x5140), b23 = __byte_perm(w2, w3, 0x7362);
+            const uint32_t o4[4] = {__byte_perm(a01, a23, 0x5410), __byte_perm(a01, a23, 0x7632), __byte_perm(b01, b23, 0x5410),
+                                    __byte_perm(b01, b23, 0x7632)};
+            const int j = ch0 >> 4, cb0 = ch0 & 15;
+            const int wi0 = (j >> 1) * 128 + ((cb0 & 7) * 4 + tq) * 4 + (j & 1) * 2 + (cb0 >> 3);
+            const uint32_t m = vmask(tq);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) put(rv + 32 + wi0 + 16 * i, o4[i], m);
         }
     } else {
         // BF16 cache: decode while scattering; a word holds two elements
