@@ -46,3 +46,16 @@ def test_binding_names_match_header():
         if name in ("hma_cache_create", "hma_cache_destroy", "hma_status_string"):
             continue      # wrapped by KVCache / status_string
         assert hasattr(hma, name), name
+
+
+def test_header_is_plain_c():
+    """include/hma.h compiles as C99 on its own (no CUDA or C++ types in the signatures)."""
+    import subprocess
+    import tempfile
+    with tempfile.NamedTemporaryFile("w", suffix=".c", delete=False) as f:
+        f.write('#include "hma.h"\nint main(void) { hma_cache_desc_t d; (void)d; return HMA_OK; }\n')
+        path = f.name
+    r = subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-fsyntax-only", "-I", os.path.join(ROOT, "include"), path],
+                       capture_output=True, text=True)
+    os.unlink(path)
+    assert r.returncode == 0, r.stderr
