@@ -30,9 +30,9 @@ from paper_2606_29986_b200 import synth  # noqa: E402
 DEFAULT_WORKLOAD = "qwen3-32b-b32-ctx8k"
 BFP8_ROW = 272      # bytes per (token, kv head): K 136 + V 136
 BF16_ROW = 512
-# DRAM bytes per launch of the attention kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum);
-# see profiles/.  Keyed by workload; None where no capture exists.
-NCU_TRAFFIC_BYTES = {"qwen3-32b-b32-ctx8k": 575_400_000}    # profiles/attn_kernel_bfp8_qwen3-32b-b32-ctx8k_ncu_full.md
+# DRAM bytes per launch of the attention kernel as one ncu capture of this workload counted them
+# (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists.
+NCU_TRAFFIC_BYTES = {"qwen3-32b-b32-ctx8k": 575_000_000}
 
 
 def measured_peak():
@@ -104,8 +104,7 @@ class Workload:
             self.caches["bf16"] = hma.KVCache(hma.make_desc(self.L, self.hq, self.hkv, self.num_pages, hma.HMA_KV_BF16), device)
         self.q = [synth.make_q(self.B, self.hq, seed + l, device) for l in range(self.L)]
         self.out = torch.empty((self.L, self.B, self.hq, 128), dtype=torch.bfloat16, device=device)
-        ws = hma.hma_decode_attention_workspace_bytes(self.caches["bfp8"].desc, self.B)
-        self.workspace = torch.empty(ws, dtype=torch.uint8, device=device)
+        self.workspace = hma.new_workspace(self.caches["bfp8"].desc, self.B, device)
         self.sample_wires = {}       # (layer, b) -> (k_wire, v_wire) numpy: wire bytes of a few sequences, for the parity tests
         keep = {(0, 0), (self.L - 1, self.B - 1), (0, int(np.argmin(self.lens))), (self.L - 1, int(np.argmax(self.lens)))}
         for l in range(self.L):
@@ -208,25 +207,41 @@ class Workload:
         barrier()
         return max_over_ranks(e0.elapsed_time(e1) / 1e3) / steps      # seconds per step
 
-    def time_layer_calls(self, fmt, reps, probe=False):
-        """Average duration of one hma_decode_attention call, CUDA events around every call on its stream."""
+    def time_calls(self, kinds, passes, fmt="bfp8"):
+        """Duration of single calls, CUDA events around every call on its stream.  `kinds` lists what to time
+        ("attn": hma_decode_attention, "probe": hma_kv_read_probe, "alu": hma_attention_alu_probe, "hbm": a plain
+        contiguous read of the layer's bytes); the kinds are interleaved call by call, layer after layer, so that
+        every kind sees the same clocks and the same cold L2.  Returns kind -> (mean, median, min) in seconds."""
         cache = self.caches[fmt]
-        evs = []
-        for r in range(reps):
+        if not hasattr(self, "sink"):
+            self.sink = torch.zeros(1, dtype=torch.int32, device=self.device)
+        evs = {k: [] for k in kinds}
+        for r in range(passes):
             for l in range(self.L):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                if probe == "alu":
-                    self.hma.hma_attention_alu_probe(cache, l, self.table, self.ctx, self.workspace)
-                elif probe:
-                    self.hma.hma_kv_read_probe(cache, l, self.table, self.ctx, self.workspace)
-                else:
-                    self.hma.hma_decode_attention(cache, l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, self.workspace)
-                b.record()
-                evs.append((a, b))
+                for kind in kinds:
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    if kind == "alu":
+                        self.hma.hma_attention_alu_probe(cache, l, self.table, self.ctx, self.workspace)
+                    elif kind == "probe":
+                        self.hma.hma_kv_read_probe(cache, l, self.table, self.ctx, self.workspace)
+                    elif kind == "hbm":
+                        self.hma.hma_hbm_read_probe(cache.layers[l], self.sink)
+                    else:
+                        self.hma.hma_decode_attention(cache, l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, self.workspace)
+                    b.record()
+                    evs[kind].append((a, b))
         torch.cuda.synchronize(self.device)
-        t = np.array([a.elapsed_time(b) for a, b in evs]) / 1e3
-        return float(t.mean()), float(np.median(t)), float(t.min())
+        res = {}
+        for kind in kinds:
+            t = np.array([a.elapsed_time(b) for a, b in evs[kind]]) / 1e3
+            res[kind] = (float(t.mean()), float(np.median(t)), float(t.min()))
+        return res
+
+    def time_layer_calls(self, fmt, reps, probe=False):
+        """Average duration of one hma_decode_attention call (or of one probe call), back to back."""
+        kind = "alu" if probe == "alu" else "probe" if probe else "attn"
+        return self.time_calls([kind], reps, fmt)[kind]
 
     def time_ingest(self, reps=5):
         """GPU time of the ingest alone (device-resident wire, every layer of the arriving request), replayed from a CUDA
@@ -264,8 +279,7 @@ class Workload:
         for l in range(self.L):
             for b in range(self.B):
                 hma.hma_kv_ingest_layer(tail, l, rows, rows, hma.HMA_WIRE_BF16_ROWS, 0, self.hkv, ttable[b].contiguous(), 0, tail_tokens)
-        ws = torch.empty(2 * (hma.hma_decode_attention_workspace_bytes(self.caches["bfp8"].desc, self.B) + 256), dtype=torch.uint8,
-                         device=self.device)
+        ws = hma.new_workspace(self.caches["bfp8"].desc, self.B, self.device, copies=2)
 
         def run():
             for l in range(self.L):
@@ -424,16 +438,23 @@ def main():
     sampler.start()
     time.sleep(0.3)
     # per-call duration of the dominant kernel (decode attention), CUDA events around each call
+    # (back to back, as inside a decode pass), then the two read ceilings interleaved with it call by call
     wl.time_layer_calls("bfp8", 1)
-    call_mean, call_med, call_min = wl.time_layer_calls("bfp8", 3)
-    wl.time_layer_calls("bfp8", 1, probe=True)
-    probe_mean, probe_med, probe_min = wl.time_layer_calls("bfp8", 3, probe=True)
+    call_mean, call_med, call_min = wl.time_layer_calls("bfp8", 5)
+    wl.time_calls(["attn", "probe", "hbm"], 1)
+    ceil = wl.time_calls(["attn", "probe", "hbm"], 5)
+    probe_mean, probe_med, probe_min = ceil["probe"]
+    hbm_mean, hbm_med, hbm_min = ceil["hbm"]
+    inter_mean, inter_med, inter_min = ceil["attn"]
     if args.kernel_only:
         wl.time_layer_calls("bfp8", 1, probe="alu")
         alu_mean = wl.time_layer_calls("bfp8", 3, probe="alu")[0]
         res = {"alu_probe_us_per_call": alu_mean * 1e6, "workload": args.workload, "layers_built": wl.L, "bfp8_us_per_call": [call_mean * 1e6, call_med * 1e6, call_min * 1e6],
-               "bfp8_gbs": wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9, "probe_us_per_call": probe_mean * 1e6,
-               "probe_gbs": wl.kv_bytes_per_layer("bfp8") / probe_mean / 1e9}
+               "bfp8_gbs": wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9, "probe_us_per_call": [probe_mean * 1e6, probe_med * 1e6, probe_min * 1e6],
+               "probe_gbs": wl.kv_bytes_per_layer("bfp8") / probe_med / 1e9,
+               "bfp8_us_per_call_interleaved": [inter_mean * 1e6, inter_med * 1e6, inter_min * 1e6],
+               "hbm_read_us": [hbm_mean * 1e6, hbm_med * 1e6, hbm_min * 1e6],
+               "hbm_read_gbs": wl.caches["bfp8"].layers[0].numel() / hbm_med / 1e9}
         if "bf16" in wl.caches:
             wl.time_layer_calls("bf16", 1)
             m, md, mn = wl.time_layer_calls("bf16", 2)
@@ -462,8 +483,8 @@ def main():
     sec_e2e_mapped = wl.time_steps(max(2, args.steps // 4), 3, host=True, staged=False) if wl.ingest_tokens else sec_e2e
     extra = {}
     if "bf16" in wl.caches:
-        k = max(1, args.steps // 10)
-        sec_bf16 = wl.time_steps(k, 3 if k > 1 else 1, fmt="bf16", ingest=False)
+        k = max(5, args.steps // 4)
+        sec_bf16 = wl.time_steps(k, 3, fmt="bf16", ingest=False)
         extra["bf16_kv"] = {"tokens_per_s": aggregate_value(wl.B, sec_bf16, ws), "ms_per_step": sec_bf16 * 1e3,
                             "kv_gbs": wl.kv_bytes_per_layer("bf16") * wl.L / sec_bf16 / 1e9, "steps": k,
                             "bfp8_speedup": sec_bf16 / sec_decode_only}
@@ -507,8 +528,16 @@ def main():
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": "of " + peak_kind, "frac_of_8000": achieved / 8000.0,
                      "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                     "probe_gbs": wl.kv_bytes_per_layer("bfp8") / probe_mean / 1e9,
-                     "frac_of_probe": probe_mean / call_mean,
+                     "probe_gbs": wl.kv_bytes_per_layer("bfp8") / probe_med / 1e9,
+                     "frac_of_probe": probe_med / inter_med,
+                     "hbm_read_gbs": wl.caches["bfp8"].layers[0].numel() / hbm_med / 1e9,
+                     "frac_of_hbm_read": (wl.kv_bytes_per_layer("bfp8") / inter_med) / (wl.caches["bfp8"].layers[0].numel() / hbm_med),
+                     "ceilings": {"what": "hma_decode_attention, hma_kv_read_probe (same records, no arithmetic) and hma_hbm_read_probe "
+                                          "(plain contiguous read of the layer) interleaved call by call, 5 passes over all layers; "
+                                          "[mean, median, min] us per call",
+                                  "attention_us": [inter_mean * 1e6, inter_med * 1e6, inter_min * 1e6],
+                                  "kv_read_probe_us": [probe_mean * 1e6, probe_med * 1e6, probe_min * 1e6],
+                                  "hbm_read_us": [hbm_mean * 1e6, hbm_med * 1e6, hbm_min * 1e6]},
                      "kernel": "hma_decode_attention (attn_kernel<0,0> + attn_merge_kernel)",
                      "bytes_per_launch": wl.kv_bytes_per_layer("bfp8"), "us_per_launch_mean": call_mean * 1e6,
                      "us_per_launch_median": call_med * 1e6, "us_per_launch_min": call_min * 1e6},

@@ -8,10 +8,11 @@
  *   hma_kv_ingest_layer     scatter one layer of arriving wire bytes into the paged cache
  *                           (consumer half of the compute-transfer pipeline, section 3.2)
  *   hma_decode_attention    GQA paged decode attention reading raw BFP8 pages (section 3.3)
- *   hma_bfp8_dequant_bf16   one-shot BFP8 -> BF16 rebuild of a request's KV (section 3.3, the
- *                           "fused kernel rebuilds a whole request's KV")
+ *   hma_bfp8_dequant_bf16   one-shot BFP8 -> BF16 rebuild of a request's KV (the whole-request
+ *                           reconstruction kernel of section 3.3)
  *
- * BFP8 as read here (the paper gives only "per-block shared exponent" and "7-bit mantissa"):
+ * BFP8 as read here (section 3.3 fixes only that a block shares one exponent and that mantissas
+ * have 7 bits):
  * a block is 16 consecutive head-dim channels of one (token, kv head); it has one exponent byte E
  * (bias 127) and 16 element bytes b = s<<7 | m;  value = (-1)^s * m * 2^(E-133).  Every such
  * value with E <= 254 is exactly a BF16 number.
@@ -47,7 +48,7 @@ typedef enum {
     HMA_ERR_ALIGNMENT = 3,
     HMA_ERR_WORKSPACE_TOO_SMALL = 4,
     HMA_ERR_CUDA = 5,
-    HMA_ERR_DEVICE_FLAGGED = 6,
+    /* 6 is not used */
     HMA_ERR_STATIC_LIMIT = 7      /* the request does not fit the library's built-in scratch array */
 } hma_status_t;
 
@@ -67,6 +68,8 @@ typedef enum { HMA_KEYS_AS_QUERIES = 0, HMA_KEYS_INTERLEAVED = 1 } hma_key_layou
 #define HMA_FLAG_BAD_PAGE_DEQUANT   4u  /* page id outside [0, num_pages): output rows zeroed    */
 #define HMA_FLAG_WAIT_TIMEOUT       8u  /* a bounded wait inside a kernel ran out                */
 #define HMA_FLAG_BAD_VALUE_ENCODE  16u  /* hma_bfp8_encode_rows met NaN/Inf: encoded as zero      */
+#define HMA_FLAG_EXPONENT_RANGE   32u  /* attention met a V block exponent above 250, or a softmax
+                                          sum that is not finite (K exponents that overflow fp32)   */
 
 typedef struct {
     int32_t num_layers;
@@ -83,7 +86,7 @@ typedef struct {
 typedef struct hma_cache hma_cache_t;   /* opaque; host-side metadata only */
 
 /*
- * Paged KV cache (paper Fig. 2 step 3: "raw BFP8 pages in HBM").
+ * Paged KV cache holding the arriving bytes undecoded (paper Fig. 2 step 3).
  *
  * One layer is `num_pages` pages; a page holds 16 tokens of every kv head; the record of one
  * (page, kv head) is contiguous: K part then V part.
@@ -112,7 +115,7 @@ void hma_cache_destroy(hma_cache_t *cache);
 /*
  * Ingest one layer of one request (sections 3.2 and 3.3: host-to-device copy and the
  * tiled -> paged layout conversion that merges per-chip shards).  Pure byte movement on a BFP8
- * cache; on a BF16 cache the same call decodes while scattering (the "standalone consumer pass"
+ * cache; on a BF16 cache the same call decodes while scattering (the separate consumer-side dequantization pass
  * of section 2.3, used to fill the baseline cache with identical values).
  *
  *   k_wire, v_wire  device or pinned: raw wire bytes of heads [head_begin, head_begin+head_count)
@@ -135,7 +138,7 @@ hma_status_t hma_kv_ingest_layer(hma_cache_t *cache, int32_t layer,
                                  const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
                                  void *stream);
 
-/* The same for several producer shards in one launch (section 3.3: "merges the per-chip KV shards"; Table 2
+/* The same for several producer shards in one launch (the shard merge of section 3.3; Table 2
  * runs Qwen3-32B prefill as one TP=4 group, so a layer arrives as four head ranges).  k_wires, v_wires,
  * head_begins, head_counts are host arrays of n_shards (1..8) entries; shard i carries heads
  * [head_begins[i], head_begins[i]+head_counts[i]) in the wire layout described above; head ranges must not
@@ -159,7 +162,8 @@ hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32
  *   workspace    device, 256-byte aligned, >= hma_decode_attention_workspace_bytes(...) bytes;
  *                contents need no initialisation and are clobbered
  *   batch        at most 1024 (HMA_ERR_UNSUPPORTED_SHAPE beyond)
- * Accuracy: fp32 accumulation; element exponents above 250 are outside the supported range.
+ * Accuracy: fp32 accumulation.  Block exponents above 250 (values beyond 2^117) are outside the supported
+ * range: the call still returns, HMA_FLAG_EXPONENT_RANGE is raised and the affected rows are not meaningful.
  * Launches: two kernels per call (attention, then a small merge of the per-worker partials), both with
  * programmatic stream serialisation; each waits on the grid dependency before it reads any input, so the
  * usual stream order holds whatever kernel precedes the call.  The first call on a device sets the kernels'
@@ -222,21 +226,6 @@ hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cac
                                         int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes,
                                         void *stream);
 
-/* Bandwidth probe: streams exactly the page records hma_decode_attention would read (same block
- * tables, same work split, same bulk-copy ring) and does no arithmetic and no output.  Its time is
- * the ceiling the attention kernel's memory pipeline can reach (section 2.2: decode is memory-bound).
- * BFP8 caches only.  Workspace as for hma_decode_attention. */
-hma_status_t hma_kv_read_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
-                               int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
-                               void *workspace, size_t workspace_bytes, void *stream);
-
-/* Diagnostic twin of the probe: the arithmetic of every record on whatever shared memory holds, with no
- * loads and no output; its time is the attention kernel's instruction-issue floor.  The paper has no
- * counterpart; it exists so that the benchmark can say which of the two floors binds. */
-hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
-                                     int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
-                                     void *workspace, size_t workspace_bytes, void *stream);
-
 /*
  * One-shot reconstruction (section 3.3): tokens [token_begin, token_begin+n_tokens) of a request,
  * tensor `which` (0 = K, 1 = V), all kv heads -> row-major BF16 [n_tokens][num_kv_heads][128].
@@ -248,13 +237,13 @@ hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t layer, int3
                                    const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
                                    void *out_bf16, void *stream);
 
-/* The whole request in one launch (section 3.3: "a fused kernel rebuilds a whole request's KV"): every layer, K and V,
+/* The whole request in one launch (the whole-request reconstruction of section 3.3): every layer, K and V,
  * -> out_bf16 [num_layers][2 (K, V)][n_tokens][num_kv_heads][128] (device, 16-byte aligned), with the same decode,
  * key re-layout and page_ids convention as hma_bfp8_dequant_bf16. */
 hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const int32_t *page_ids, int64_t token_begin,
                                       int64_t n_tokens, void *out_bf16, void *stream);
 
-/* The "naive elementwise reconstruction" that section 3.3 measures the fused rebuild against (72 ms vs 1.5 ms on the
+/* The elementwise strawman that section 3.3 measures the fused rebuild against (72 ms vs 1.5 ms on the
  * paper's A100): same arguments and the same bits as hma_bfp8_dequant_bf16, computed one thread per element with byte
  * loads.  A comparison point for the benchmark, not a product path. */
 hma_status_t hma_bfp8_dequant_bf16_naive(const hma_cache_t *cache, int32_t layer, int32_t which,
@@ -287,6 +276,33 @@ const char *hma_last_cuda_error(void);
 
 /* Number of kernels this library has launched in the calling process (for launch accounting). */
 int64_t hma_launch_count(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * Instrumentation.  Nothing below is on the decode path; the benchmark uses these entry points to
+ * say which ceiling binds (the paper has no counterpart; section 2.2 only states that decode is
+ * memory-bound).
+ * ------------------------------------------------------------------------------------------------ */
+
+/* Bandwidth probe: streams exactly the page records hma_decode_attention would read (same block
+ * tables, same work split, same bulk-copy ring) and does no arithmetic and no output.  Its time is
+ * the ceiling the attention kernel's memory pipeline can reach (section 2.2: decode is memory-bound).
+ * BFP8 caches only.  Workspace as for hma_decode_attention. */
+hma_status_t hma_kv_read_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
+                               int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/* Diagnostic twin of the probe: the arithmetic of every record on whatever shared memory holds, with no
+ * loads and no output; its time is the attention kernel's instruction-issue floor.  The paper has no
+ * counterpart; it exists so that the benchmark can say which of the two floors binds. */
+hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,
+                                     int32_t max_pages_per_seq, const int32_t *context_lens, int32_t batch,
+                                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* A plain contiguous read of `bytes` bytes of device memory (16-byte aligned) with streaming loads: the simplest
+ * read-only ceiling of the GPU's memory system, for comparison with hma_kv_read_probe.  `sink4` is a device word
+ * the kernel may add to (it practically never does; it keeps the loads alive). */
+hma_status_t hma_hbm_read_probe(const void *src, size_t bytes, void *sink4, void *stream);
+
 
 #ifdef __cplusplus
 }

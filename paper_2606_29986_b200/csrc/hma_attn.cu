@@ -6,9 +6,11 @@
 //     All (sequence, kv head, page) records of the batch form one linear work list that is cut into
 //     contiguous ranges of equal cost, one per *warp* (any mix of context lengths, no barrier between
 //     warps; starting a segment is charged like two records).  A warp that holds only part of a
-//     (sequence, kv head) segment writes a partial (max, sum, 128-vector) per q head; a small second kernel, launched with programmatic dependent
-//     launch so that its launch latency hides behind the main kernel, merges the partials in worker
-//     order (fixed order, so results are bitwise repeatable).
+//     (sequence, kv head) segment leaves a partial (max, sum, 128-vector) per q head in its own ring slots; when
+//     every warp of the CTA is done the CTA combines, in warp order, the partials that belong to one segment.  A
+//     segment that lies inside one CTA is finished there; one that several CTAs share goes to global memory as one
+//     partial per CTA, and the CTA that arrives last (an arrival counter per segment in the workspace) merges them
+//     in CTA order.  Every order is fixed, so results are bitwise repeatable; there is no second kernel.
 //   * every warp feeds itself: it keeps three 4352-byte page records in flight with 1-D bulk async
 //     copies (cp.async.bulk + mbarrier transaction counts) and re-arms a ring slot as soon as its
 //     Q.K^T phase has pulled the record's words into registers.
@@ -39,12 +41,14 @@ struct Geo {
     static constexpr int record = kFmt == HMA_KV_BFP8 ? kBfp8Record : kBf16Record;
     static constexpr int scratch = kFmt == HMA_KV_BFP8 ? kScratch : 0;
 };
-constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile: o[8][128], m[8], l[8]
+constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile in global memory: o[8][128], m[8], l[8]
+constexpr int kPieceStride = kHeadDim + 4;        // floats per head of a partial parked in a ring slot (bank-conflict-free)
+constexpr int kPieceFloats = 8 * kPieceStride + 16;   // 1072 floats = 4288 B: fits the smallest ring slot (4352 B)
 constexpr uint32_t kSpinLimit = 1u << 20;           // polls of a bounded wait
 constexpr uint32_t kSuspendNs = 2000;              // a failed poll may keep the thread parked this long
 constexpr int kMaxBatch = 1024;
 constexpr int kSegCost = 2;                        // what starting a segment costs a warp, in records (Q load, partial tile)
-constexpr int kMaxCtas = 160;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
+constexpr int kMaxCtas = 192;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
 constexpr int kMinRecords = 4;                    // fewest records a worker takes
 constexpr int kMaxDevices = 64;
 
@@ -58,11 +62,42 @@ struct AttnArgs {
     const int32_t *ctx;
     int batch;
     float sm_scale;
+    int32_t *counters;              // workspace: one arrival counter per (sequence, kv head); zero between calls
     int32_t *cum;                   // workspace: pages before each sequence, then pages + segment costs before each
-                                    // sequence, batch + 1 entries each (for the merge kernel)
-    float *tiles;                   // workspace: partial tiles
-    int always_partial;             // 1: never write `out`; every segment leaves partial tiles (two-cache attention)
+                                    // sequence, batch + 1 entries each (written for the two-cache merge kernel only)
+    float *tiles;                   // workspace: per-CTA partial tiles; CTA c's partial of segment s is tile c + s
+    float *tails;                   // workspace: one tile per segment, for the warp that holds the segment's end and goes on
+    int always_partial;             // 1: never write `out`; every segment leaves per-CTA partial tiles (two-cache attention)
+#ifdef HMA_TRACE
+    unsigned long long *trace;      // workspace, after the tiles: kTraceWords words per worker (see trace_stamp)
+#endif
 };
+
+// Per-warp timing instrumentation, compiled in only with -DHMA_TRACE (a separate library image; the default build
+// carries none of it).  Each worker writes kTraceWords 64-bit words after the partial tiles of the workspace:
+//   0 SM id   1 after the grid-dependency wait   2 end of the prologue   3 first record landed
+//   4 end of the record loop   5 after the last partial/output store   6 records taken   7 unused
+//   8 CTA-level reduction begins (all warps of the CTA are done)   9 its segments are reduced
+//   10 arrivals on the shared segments' counters are done   11 the CTA leaves   12 walk begins   13-15 first segments done
+// Words 1-5 are %globaltimer nanoseconds; words 8-15 are the SM's cycle counter (only differences inside a CTA mean anything).
+constexpr int kTraceWords = 16;
+#ifdef HMA_TRACE
+__device__ __forceinline__ unsigned long long trace_now()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ unsigned trace_smid()
+{
+    unsigned v;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(v));
+    return v;
+}
+#define HMA_TRACE_STAMP(a, u, i, v)  do { if ((threadIdx.x & 31) == 0) (a).trace[(u) * kTraceWords + (i)] = (v); } while (0)
+#else
+#define HMA_TRACE_STAMP(a, u, i, v)  do { } while (0)
+#endif
 
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -210,7 +245,239 @@ __device__ __forceinline__ void store_out(const AttnArgs &a, int64_t idx, float 
     else reinterpret_cast<uint16_t *>(a.out)[idx] = f32_to_bf16_rne(v);
 }
 
+// How the work list (WX cost units) is dealt out: `nwk` workers (warps) over the first `ctas` CTAs of the grid.
+struct Split {
+    int64_t nwk;
+    int64_t ctas;
+};
+__host__ __device__ inline Split make_split(int64_t WX, int grid_ctas, int warps_per_cta)
+{
+    Split s;
+    s.nwk = WX / kMinRecords;
+    if (s.nwk > (int64_t)grid_ctas * warps_per_cta) s.nwk = (int64_t)grid_ctas * warps_per_cta;
+    if (s.nwk < 1) s.nwk = 1;
+    s.ctas = s.nwk < grid_ctas ? s.nwk : grid_ctas;
+    return s;
+}
+// CTA that holds worker u, and the CTAs [c0, c0 + count) whose records meet segment (b, g) of np records; `first` is the
+// cost position of the segment's first record.
+__host__ __device__ inline int64_t cta_of_worker(const Split &s, int64_t u) { return ((u + 1) * s.ctas - 1) / s.nwk; }
+__host__ __device__ inline void segment_ctas(const Split &s, int64_t WX, int64_t first, int np, int64_t *c0, int *count)
+{
+    const int64_t u0 = ((first + 1) * s.nwk - 1) / WX, u1 = ((first + np) * s.nwk - 1) / WX;   // first and last worker
+    *c0 = cta_of_worker(s, u0);
+    *count = (int)(cta_of_worker(s, u1) - *c0 + 1);
+}
+
 // ---------------------------------------------------------------- the kernel
+// ---------------------------------------------------------------- CTA-level reduction and cross-CTA merge
+// Runs once per CTA after all of its warps have parked their last partial (a function of its own so that its
+// registers do not weigh on the record loop).
+struct EpilogueArgs {       // what the reduction needs of AttnArgs, by value (registers, not a stack copy of the parameters)
+    void *out;
+    float *tiles, *tails;
+    int32_t *counters;
+    int out_dtype, always_partial, batch;
+    struct { int num_kv_heads, num_q_heads; } cv;
+#ifdef HMA_TRACE
+    unsigned long long *trace;      // this warp's trace words
+#endif
+};
+#ifdef HMA_TRACE
+#define HMA_TRACE_EPI(a, i)  do { if ((threadIdx.x & 31) == 0) (a).trace[i] = (unsigned long long)clock64(); } while (0)   /* SM cycles: cheap to read */
+#else
+#define HMA_TRACE_EPI(a, i)  do { } while (0)
+#endif
+__device__ __forceinline__ void store_pair(void *out, int out_dtype, int64_t oi, float x, float y)
+{
+    if (out_dtype == HMA_OUT_F32) *reinterpret_cast<float2 *>(reinterpret_cast<float *>(out) + oi) = make_float2(x, y);
+    else *reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(out) + oi) = f32_to_bf16_rne(x) | ((uint32_t)f32_to_bf16_rne(y) << 16);
+}
+
+template <int kFmt>
+__device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *ring, const long long *wr, const int *wseg,
+                                          const int *cum, const int *ecum, int *misc)
+{
+    constexpr int kWarps = Geo<kFmt>::warps, kThreads = Geo<kFmt>::threads, kRecord = Geo<kFmt>::record;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv, B = a.batch;
+    const bool aborted = misc[0] != 0;            // outputs of this CTA are void (and flagged); arrivals still happen
+    HMA_TRACE_EPI(a, 8);
+    // lane i of every warp holds the record range of warp i
+    const long long my_lo = lane < kWarps ? wr[2 * lane] : 0, my_hi = lane < kWarps ? wr[2 * lane + 1] : 0;
+    const unsigned have = __ballot_sync(0xFFFFFFFFu, my_lo < my_hi);
+    if (have == 0) return;
+    const long long clo = __shfl_sync(0xFFFFFFFFu, my_lo, __ffs(have) - 1), chi = __shfl_sync(0xFFFFFFFFu, my_hi, 31 - __clz(have));
+    const uint32_t ring_s = smem_u32(ring);
+    const int sb0 = wseg[2 * (__ffs(have) - 1)], sg0 = wseg[2 * (__ffs(have) - 1) + 1];     // segment of the CTA's first record
+    // Calls fn(sb, sg, npb, whole_seg, members, has_tail, tail_warp) for every segment of the CTA's range that is not
+    // finished already (one warp holding it entirely).  `members`: the warps whose last partial (ring slot 0) belongs
+    // to the segment; has_tail: in addition, after the members in order, the tail tile in ring slot 1 of tail_warp.
+    auto walk = [&](auto &&fn) {
+        int sb = sb0, sg = sg0, npb = cum[sb0 + 1] - cum[sb0];
+        for (;;) {
+            const long long s_lo = (long long)Hkv * cum[sb] + (long long)sg * npb, s_hi = s_lo + npb;
+            if (s_lo >= chi) break;
+            const long long lo = max(s_lo, clo), hi = min(s_hi, chi);
+            unsigned mem = __ballot_sync(0xFFFFFFFFu, my_lo < my_hi && my_lo < hi && my_hi > lo);     // warps with records of this segment
+            const int i1 = 31 - __clz(mem);
+            const bool one_warp_whole = (mem & (mem - 1)) == 0 && __shfl_sync(0xFFFFFFFFu, my_lo <= s_lo && my_hi >= s_hi, i1);
+            if (!one_warp_whole) {
+                // the last warp of the group may have gone on into the next segment: its partial is the segment's tail tile
+                const bool tail_in_global = __shfl_sync(0xFFFFFFFFu, my_hi > s_hi, i1);
+                if (tail_in_global) mem &= ~(1u << i1);
+                fn(sb, sg, npb, lo == s_lo && hi == s_hi, mem, tail_in_global, i1);
+            }
+            if (++sg == Hkv) {
+                sg = 0;
+                do { ++sb; } while (sb < B && cum[sb + 1] == cum[sb]);
+                if (sb >= B) break;
+                npb = cum[sb + 1] - cum[sb];
+            }
+        }
+    };
+    HMA_TRACE_EPI(a, 12);
+    int n_groups = 0;
+    int n_open = 0;                               // segments this CTA shares with other CTAs (at most its first and last)
+    walk([&](int sb, int sg, int npb, bool whole_seg, unsigned mem, bool tail_in_global, int tail_warp) {
+        const int64_t seg = (int64_t)sb * Hkv + sg;
+        if (!aborted) {
+            const uint32_t gtail = ring_s + (tail_warp * kDepth + 1) * kRecord;      // dense tile layout, in the ring slot 1 of the warp that wrote it
+            const int i0 = mem ? __ffs(mem) - 1 : 0, i1 = mem ? 31 - __clz(mem) : -1;
+#ifdef HMA_EXP_NOREDUCE
+            if (false)
+#endif
+            for (int idx = tid; idx < 8 * (kHeadDim / 2); idx += kThreads) {
+                // a warp works on one head: lane i weighs the partial of warp i, lane kWarps the tail tile
+                const int h = idx / (kHeadDim / 2), ch = 2 * (idx % (kHeadDim / 2));
+                if (h >= G) break;
+                float mine_m = -INFINITY, mine_l = 0.f;
+                if (lane < kWarps && (mem >> lane & 1u)) {
+                    const uint32_t pc = ring_s + lane * kDepth * kRecord + (8 * kPieceStride + h) * 4;
+                    mine_m = __uint_as_float(lds32(pc)); mine_l = __uint_as_float(lds32(pc + 32));
+                } else if (lane == kWarps && tail_in_global) {
+                    mine_m = __uint_as_float(lds32(gtail + (8 * kHeadDim + h) * 4)); mine_l = __uint_as_float(lds32(gtail + (8 * kHeadDim + 8 + h) * 4));
+                }
+                float M = mine_m;
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
+                const float mine_w = mine_m == -INFINITY ? 0.f : ex2f(mine_m - M);
+                float den = mine_w * mine_l;
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, d);      // fixed butterfly order
+                float2 vt = make_float2(0.f, 0.f);
+                if (tail_in_global)
+                    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(vt.x), "=f"(vt.y) : "r"(gtail + (h * kHeadDim + ch) * 4));
+                float nx = 0.f, ny = 0.f;
+                for (int i = i0; i <= i1; i += 4) {            // in warp order, four loads in flight
+                    float2 v[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        v[j] = make_float2(0.f, 0.f);
+                        if (mem >> (i + j) & 1u)
+                            asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v[j].x), "=f"(v[j].y)
+                                         : "r"(ring_s + (i + j) * kDepth * kRecord + (h * kPieceStride + ch) * 4));
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float wgt = __shfl_sync(0xFFFFFFFFu, mine_w, (i + j) & 31);      // 0 for a warp that is no member
+                        nx = fmaf(wgt, v[j].x, nx); ny = fmaf(wgt, v[j].y, ny);
+                    }
+                }
+                {
+                    const float wgt = __shfl_sync(0xFFFFFFFFu, mine_w, kWarps);
+                    nx = fmaf(wgt, vt.x, nx); ny = fmaf(wgt, vt.y, ny);
+                }
+#ifdef HMA_EXP_NOSTORE
+                if (nx == 1.2345f)
+#endif
+                if (whole_seg && !a.always_partial) {
+                    const float inv = den > 0.f ? 1.f / den : 0.f;
+                    store_pair(a.out, a.out_dtype, ((int64_t)sb * Hq + (int64_t)sg * G + h) * kHeadDim + ch, nx * inv, ny * inv);
+                } else {
+                    float *tp = a.tiles + ((int64_t)blockIdx.x + seg) * kTileFloats;
+                    *reinterpret_cast<float2 *>(tp + h * kHeadDim + ch) = make_float2(nx, ny);
+                    if (ch == 0) { tp[8 * kHeadDim + h] = M; tp[8 * kHeadDim + 8 + h] = den; }
+                }
+            }
+        }
+        if (!whole_seg && !a.always_partial && n_open < 2) {
+#ifdef HMA_EXP_NODIV
+            if (tid == 32 * n_open) { misc[4 + 4 * n_open] = 2; misc[5 + 4 * n_open] = 0; misc[6 + 4 * n_open] = sb; misc[7 + 4 * n_open] = sg; }
+            if (false) {
+#else
+            if (tid == 32 * n_open) {
+#endif
+                // this thread will register the CTA on the segment's arrival counter: which CTAs share the segment
+                const int64_t WX = (int64_t)Hkv * ecum[B];
+                const Split sp = make_split(WX, (int)gridDim.x, kWarps);
+                const int64_t first = (int64_t)Hkv * ecum[sb] + (int64_t)sg * (npb + kSegCost) + kSegCost;   // cost position of the first record
+                int64_t c0;
+                int parts;
+                segment_ctas(sp, WX, first, npb, &c0, &parts);
+                misc[4 + 4 * n_open] = parts; misc[5 + 4 * n_open] = (int)c0;
+                misc[6 + 4 * n_open] = sb; misc[7 + 4 * n_open] = sg;
+            }
+            ++n_open;
+        }
+        if (n_groups < 3) HMA_TRACE_EPI(a, 13 + n_groups);
+        ++n_groups;
+    });
+    HMA_TRACE_EPI(a, 9);
+    if (n_open == 0) return;                      // the same for every thread of the CTA
+    // Arrival: the CTA's tile stores happen before the barrier, the release of the arriving thread's atomic carries
+    // them (cumulativity) to whoever acquires the counter after the last arrival.
+    __syncthreads();
+    if ((tid & 31) == 0 && (tid >> 5) < n_open) {
+        const int k = tid >> 5;
+        int32_t *ctr = a.counters + (int64_t)misc[6 + 4 * k] * Hkv + misc[7 + 4 * k];
+        int prev;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(ctr) : "memory");
+        const bool last = prev == misc[4 + 4 * k] - 1;
+        if (last) *ctr = 0;                       // everybody has arrived: leave the counter ready for the next call
+        else misc[4 + 4 * k] = 0;
+    }
+    __syncthreads();
+    HMA_TRACE_EPI(a, 10);
+    for (int k = 0; k < n_open; ++k) {
+        const int parts = misc[4 + 4 * k];
+        if (parts == 0) continue;                 // another CTA will arrive later and finish this segment
+        const int ob = misc[6 + 4 * k], og = misc[7 + 4 * k];
+        const float *t0 = a.tiles + ((int64_t)misc[5 + 4 * k] + (int64_t)ob * Hkv + og) * kTileFloats;       // part i is at t0 + i * kTileFloats
+        for (int idx = tid; idx < 8 * (kHeadDim / 2); idx += kThreads) {
+            const int h = idx / (kHeadDim / 2), ch = 2 * (idx % (kHeadDim / 2));
+            if (h >= G) break;
+            // parts in CTA order, four at a time (one trip to L2 for the usual two to four parts), running maximum
+            float M = -INFINITY, nx = 0.f, ny = 0.f, den = 0.f;
+            for (int p0 = 0; p0 < parts; p0 += 4) {
+                float mi[4], li[4];
+                float2 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float *tp = t0 + (int64_t)(p0 + j) * kTileFloats;
+                    const bool ok = p0 + j < parts;
+                    mi[j] = ok ? __ldcg(tp + 8 * kHeadDim + h) : -INFINITY;
+                    li[j] = ok ? __ldcg(tp + 8 * kHeadDim + 8 + h) : 0.f;
+                    v[j] = ok ? __ldcg(reinterpret_cast<const float2 *>(tp + h * kHeadDim + ch)) : make_float2(0.f, 0.f);
+                }
+                const float Mn = fmaxf(fmaxf(fmaxf(mi[0], mi[1]), fmaxf(mi[2], mi[3])), M);
+                const float keep = M == -INFINITY ? 0.f : ex2f(M - Mn);
+                nx *= keep; ny *= keep; den *= keep;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float wgt = mi[j] == -INFINITY ? 0.f : ex2f(mi[j] - Mn);
+                    nx = fmaf(wgt, v[j].x, nx); ny = fmaf(wgt, v[j].y, ny);
+                    den = fmaf(wgt, li[j], den);
+                }
+                M = Mn;
+            }
+            const float inv = den > 0.f ? 1.f / den : 0.f;
+            store_pair(a.out, a.out_dtype, ((int64_t)ob * Hq + (int64_t)og * G + h) * kHeadDim + ch, nx * inv, ny * inv);
+        }
+    }
+    HMA_TRACE_EPI(a, 11);
+}
+
 // kMode 0: attention.  1: stream the records through the ring, no arithmetic (bandwidth probe).
 // 2: the arithmetic of every record on whatever the ring holds, nothing loaded or written (issue-rate probe).
 extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -225,8 +492,10 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     uint8_t *scratch = ring + kStages * kRecord;                                  // kWarps x kScratch (BFP8 only)
     uint64_t *bars = reinterpret_cast<uint64_t *>(scratch + kWarps * Geo<kFmt>::scratch);   // full[kStages]
     int *stage_ok = reinterpret_cast<int *>(bars + kStages);                      // [kStages]
-    int *misc = stage_ok + kStages;                                               // [0] abort word, [16..80) scan scratch
-    int *cum = misc + 16 + 64;                                                    // [batch + 1] pages before each sequence
+    int *misc = stage_ok + kStages;                                               // [0] abort word, [4..12) epilogue, [16..80) scan scratch
+    long long *wr = reinterpret_cast<long long *>(misc + 16 + 64);                // [kWarps][2] record range of each warp
+    int *wseg = reinterpret_cast<int *>(wr + 2 * kWarps);                         // [kWarps][2] sequence and kv head of its first record
+    int *cum = wseg + 2 * kWarps;                                                 // [batch + 1] pages before each sequence
     int *ecum = cum + a.batch + 1;                                                // [batch + 1] same, plus kSegCost per non-empty sequence
     volatile int *abort_word = misc;
 
@@ -242,6 +511,9 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     // The kernel is launched with programmatic stream serialisation: its CTAs may be placed while the previous
     // kernel of the stream drains.  Nothing that a predecessor could have written is read before this wait.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef HMA_TRACE
+    const unsigned long long tr_wait = trace_now();
+#endif
     // Exclusive prefixes per sequence of (pages) and of (pages + kSegCost if the sequence is not empty): each thread
     // owns `per` consecutive sequences, warps scan with shuffles, one warp scans the warp totals.
     {
@@ -277,27 +549,36 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         }
         __syncthreads();
     }
-    // let the merge kernel be scheduled already; it blocks in griddepcontrol.wait until this grid has finished
+#ifdef HMA_TRACE
+    const unsigned long long tr_pro = trace_now();
+#endif
+    // the next kernel of the stream may be placed as SMs free up; it waits on this grid by itself
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (blockIdx.x == 0 && kMode == 0)
+    if (blockIdx.x == 0 && kMode == 0 && a.always_partial)
         for (int b = tid; b <= B; b += kThreads) { a.cum[b] = cum[b]; a.cum[B + 1 + b] = ecum[b]; }
-    // from here on the warps never synchronise with one another
+    // from here to the CTA-level reduction at the end the warps never synchronise with one another
     const int64_t W = (int64_t)Hkv * cum[B];
     // The work list is cut by cost, not by record count: every (sequence, kv head) segment is charged kSegCost
-    // extra units at its start, so a warp whose range crosses a segment boundary (a second Q load, a second partial
-    // tile) gets that many records fewer.  WX is the list's length in cost units.
+    // extra units at its start, so a warp whose range crosses a segment boundary (a second Q load, a second partial)
+    // gets that many records fewer.  WX is the list's length in cost units.
     const int64_t WX = (int64_t)Hkv * ecum[B];
-    // Workers are numbered across SMs first.  Small batches use fewer workers, at least kMinRecords units
-    // each, so that a segment is never cut into more partials than it is worth.
-    const int64_t NWK = max((int64_t)1, min((int64_t)gridDim.x * kWarps, WX / kMinRecords));
-    const int64_t u = (int64_t)warp * gridDim.x + blockIdx.x;      // this warp's worker index
+    // Small batches use fewer workers, at least kMinRecords units each, so that a segment is never cut into more
+    // partials than it is worth.  Workers are dealt to the CTAs in contiguous runs (CTA c holds workers
+    // [c * NWK / C, (c + 1) * NWK / C) of the C CTAs in use), so a CTA owns one contiguous range of records.
+    const Split sp = make_split(WX, (int)gridDim.x, kWarps);
+    const int64_t NWK = sp.nwk;
+    const int64_t ubase = (int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * NWK / sp.ctas : NWK;
+    const int nmine = (int64_t)blockIdx.x < sp.ctas ? (int)(((int64_t)blockIdx.x + 1) * NWK / sp.ctas - ubase) : 0;
+    const int64_t u = ubase + warp;                                 // this warp's worker index (if warp < nmine)
+    if (lane == 0) { wr[2 * warp] = 0; wr[2 * warp + 1] = 0; }      // no records until shown otherwise
 
+    do {    // ---- this warp's share of the work list; `break` leaves for the CTA-level reduction ----
+    if (warp >= nmine) break;
     if (kMode == 0 && !a.always_partial)                          // empty sequences get rows of zeros
         for (int64_t b = u; b < B; b += NWK)
             if (cum[b + 1] == cum[b])
                 for (int i = lane; i < Hq * kHeadDim; i += 32) store_out(a, b * Hq * kHeadDim + i, 0.f);
 
-    if (u >= NWK) return;
     // number of records that lie before cost position p
     auto records_before = [&](int64_t p) -> int64_t {
         if (p >= WX) return W;
@@ -312,8 +593,12 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         return (int64_t)Hkv * cum[lo] + (int64_t)gg * n + max(0, r - kSegCost);
     };
     const int64_t wlo = records_before(u * WX / NWK), whi = records_before((u + 1) * WX / NWK);
-    if (wlo >= whi) return;
+    if (wlo >= whi) break;
     const int Rw = (int)(whi - wlo);
+    HMA_TRACE_STAMP(a, u, 0, (unsigned long long)trace_smid());
+    HMA_TRACE_STAMP(a, u, 1, tr_wait);
+    HMA_TRACE_STAMP(a, u, 2, tr_pro);
+    HMA_TRACE_STAMP(a, u, 6, (unsigned long long)Rw);
 
     // the segment (b, g) and page that hold record wlo
     int b, g, page, np;
@@ -330,6 +615,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         g = (int)(off / np);
         page = (int)(off - (int64_t)g * np);
     }
+    if (lane == 0) { wr[2 * warp] = wlo; wr[2 * warp + 1] = whi; wseg[2 * warp] = b; wseg[2 * warp + 1] = g; }
 
     // ---- the warp's own feed: three ring slots; record addresses are worked out 32 at a time, one per lane ----
     const uint32_t full0 = smem_u32(bars + warp * kDepth);
@@ -394,12 +680,13 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     int Rmine = 0;                                 // reference exponent of V channel block (lane & 7)
     int T = 0, tail = kPageTokens;
     bool whole = false;                            // this warp holds every record of the current segment
+    int64_t tail_seg = -1;                         // segment whose end this warp held before going on (its tail tile is in global memory)
 
     auto begin_segment = [&](int k) {
         np = cum[b + 1] - cum[b];
         T = min(a.ctx[b], a.max_pages * kPageTokens);
         tail = T - (np - 1) * kPageTokens;
-        whole = page == 0 && Rw - k >= np && !a.always_partial;
+        whole = page == 0 && Rw - k >= np;
         // Q fragments of this (sequence, kv head): FP16, one power-of-two scale per head
         float f[8][4];
         float amax = 0.f;
@@ -457,7 +744,12 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         Rmine = 0;
     };
 
-    auto finish_segment = [&]() {
+    // The warp is done with its records of the current segment.  A segment it held entirely is finished here (written
+    // to `out`, or as a partial tile for the two-cache merge).  Otherwise the partial (o, m, l) waits for the CTA-level
+    // reduction: in the warp's ring slot 0 if these were the warp's last records (the ring is idle by then), else (the
+    // warp goes on into the next segment, so it held the end of this one, and only one warp does) in the segment's
+    // tail tile in global memory, which the warp copies back into its ring slot 1 once its ring is idle.
+    auto finish_segment = [&](bool at_end) {
         if (kMode == 1) return;
         if (kBfp8) {
             // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
@@ -469,9 +761,11 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         }
         const float l0 = lacc[0], l1 = lacc[1];
         const int h0 = 2 * t4, h1 = 2 * t4 + 1;
+        // a softmax sum that is not finite: scores overflowed fp32 (K exponents beyond the supported range)
+        if (!(l0 < INFINITY) || !(l1 < INFINITY)) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);
         const int64_t ob = ((int64_t)b * Hq + (int64_t)g * G) * kHeadDim;
         if (kMode == 2 && a.batch >= 0) return;    // the issue-rate probe never stores, but keeps its arithmetic live
-        if (whole) {
+        if (whole && !a.always_partial) {
             const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -482,15 +776,26 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                 }
             return;
         }
-        const int64_t seg = (int64_t)b * Hkv + g;
-        float *tp = a.tiles + (u + seg) * kTileFloats;
+        float *tp;
+        int hs;           // floats between heads
+        if (whole) {      // two-cache attention: nobody else touches this segment, its tile goes straight to global memory
+            tp = a.tiles + ((int64_t)blockIdx.x + (int64_t)b * Hkv + g) * kTileFloats;
+            hs = kHeadDim;
+        } else if (at_end) {
+            tp = reinterpret_cast<float *>(ring + (warp * kDepth) * kRecord);
+            hs = kPieceStride;
+        } else {
+            tail_seg = (int64_t)b * Hkv + g;
+            tp = a.tails + tail_seg * kTileFloats;
+            hs = kHeadDim;
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tp[((c & 1) ? h1 : h0) * kHeadDim + 16 * j + gq + 8 * (c >> 1)] = o[j][c];
+            for (int c = 0; c < 4; ++c) tp[((c & 1) ? h1 : h0) * hs + 16 * j + gq + 8 * (c >> 1)] = o[j][c];
         if (gq == 0) {
-            tp[8 * kHeadDim + h0] = m0; tp[8 * kHeadDim + h1] = m1;
-            tp[8 * kHeadDim + 8 + h0] = l0; tp[8 * kHeadDim + 8 + h1] = l1;
+            tp[8 * hs + h0] = m0; tp[8 * hs + h1] = m1;
+            tp[8 * hs + 8 + h0] = l0; tp[8 * hs + 8 + h1] = l1;
         }
     };
 
@@ -502,7 +807,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     for (int k = 0; k < Rw; ++k) {
         if (left == 0) {
             if (k > 0) {
-                finish_segment();
+                finish_segment(false);
                 page = 0;
                 if (++g == Hkv) {
                     g = 0;
@@ -520,6 +825,9 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         if (kMode < 2) {
             alive = mbar_wait(full0 + 8 * slot, par, abort_word, a.cv.flags);
             if (!alive) break;
+#ifdef HMA_TRACE
+            if (k == 0) HMA_TRACE_STAMP(a, u, 3, trace_now());
+#endif
         }
         if (++slot == kDepth) { slot = 0; par ^= 1u; }
         const bool ok = kMode == 2 || stage_ok[s_idx] != 0;
@@ -555,6 +863,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                     emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
                     emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
                     const int Rnew = max(Rmine, emax);
+                    if (Rnew > 250) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);   // beyond the supported range
     #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
@@ -729,132 +1038,71 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
             }
         }
     }
-    if (alive) finish_segment();
-    else if (lane == 0 && kMode < 2) {
+    HMA_TRACE_STAMP(a, u, 4, trace_now());
+    if (alive) {
+        finish_segment(true);
+        if (tail_seg >= 0 && kMode == 0) {
+            // the last tail tile this warp wrote (it can only be shared with other warps if it was the warp's first
+            // segment, and a warp writes at most one such) comes back from L2 into ring slot 1, same layout
+            __syncwarp();
+            const uint4 *src = reinterpret_cast<const uint4 *>(a.tails + tail_seg * kTileFloats);
+            const uint32_t dst = ring0 + kRecord;
+            uint4 v[(kTileFloats * 4 / 16 + 31) / 32];
+#pragma unroll
+            for (int i = 0; i < (kTileFloats * 4 / 16 + 31) / 32; ++i)
+                if (lane + 32 * i < kTileFloats * 4 / 16) v[i] = __ldcg(src + lane + 32 * i);
+#pragma unroll
+            for (int i = 0; i < (kTileFloats * 4 / 16 + 31) / 32; ++i)
+                if (lane + 32 * i < kTileFloats * 4 / 16) sts128(dst + (lane + 32 * i) * 16, v[i].x, v[i].y, v[i].z, v[i].w);
+        }
+    }
+    HMA_TRACE_STAMP(a, u, 5, trace_now());
+    if (!alive && lane == 0 && kMode < 2) {
         // a wait ran out: give the copies still in flight a bounded chance to land before the warp leaves
         for (int s = 0; s < kDepth; ++s)
             for (uint32_t it = 0; it < (1u << 16) && !mbar_try_wait(full0 + 8 * s, 0) && !mbar_try_wait(full0 + 8 * s, 1); ++it) {}
     }
-}
+    } while (0);
 
-// ---------------------------------------------------------------- cross-split merge
-// One CTA per (sequence, kv head), one warp per q head, four channels per lane.  Segments that a single worker
-// held entirely were written by the main kernel.  Lane i of a chunk holds (m, l) of part i, so the weights of up
-// to 32 parts come from one round of loads; the 128-vectors are then fetched four parts at a time.
-__global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a, int max_workers)
-{
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may be placed; it waits by itself
-    asm volatile("griddepcontrol.wait;" ::: "memory");               // the main kernel's tiles are complete and visible
-    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
-    const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, h = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (h >= G) return;
-    const int np = a.cum[b + 1] - a.cum[b];
-    if (np == 0) return;                                         // rows of empty sequences were zeroed by the main kernel
-    // the main kernel cut the work list by cost (kSegCost units at the start of every segment, then one per record)
-    const int32_t *ecum = a.cum + a.batch + 1;
-    const int64_t WX = (int64_t)Hkv * ecum[a.batch];
-    const int64_t NWK = max((int64_t)1, min((int64_t)max_workers, WX / kMinRecords));
-    const int64_t first = (int64_t)Hkv * ecum[b] + (int64_t)g * (np + kSegCost) + kSegCost;   // cost position of the first record
-    const int64_t u0 = ((first + 1) * NWK - 1) / WX, u1 = ((first + np) * NWK - 1) / WX;       // first and last worker of the segment
-    if (u0 == u1) return;
-    const float *t0 = a.tiles + (int64_t)blockIdx.x * kTileFloats;           // part i is at t0 + i * kTileFloats
-    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-    float den = 0.f;
-    const int P = (int)(u1 - u0 + 1);
-    if (P <= 16) {
-        // common case: every load of the merge is issued before any is used (one trip to L2)
-        float4 v[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-            v[j] = j < P ? __ldcg(reinterpret_cast<const float4 *>(t0 + (u0 + j) * kTileFloats + h * kHeadDim) + lane)
-                         : make_float4(0.f, 0.f, 0.f, 0.f);
-        float mm = -INFINITY, ll = 0.f;
-        if (lane < P) {
-            mm = __ldcg(t0 + (u0 + lane) * kTileFloats + 8 * kHeadDim + h);
-            ll = __ldcg(t0 + (u0 + lane) * kTileFloats + 8 * kHeadDim + 8 + h);
-        }
-        float M = mm;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
-        const float wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
-        den = wgt * ll;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, d);          // fixed butterfly order
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const float wj = __shfl_sync(0xFFFFFFFFu, wgt, j);
-            num.x = fmaf(wj, v[j].x, num.x); num.y = fmaf(wj, v[j].y, num.y);
-            num.z = fmaf(wj, v[j].z, num.z); num.w = fmaf(wj, v[j].w, num.w);
-        }
-    } else {
-        float M = -INFINITY;
-        for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
-            const int64_t i = c0 + lane;
-            float mm = i <= u1 ? __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h) : -INFINITY;
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, d));
-            M = fmaxf(M, mm);
-        }
-        for (int64_t c0 = u0; c0 <= u1; c0 += 32) {
-            const int64_t i = c0 + lane;
-            float wgt = 0.f, dsum = 0.f;
-            if (i <= u1) {
-                const float mm = __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + h);
-                wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
-                dsum = wgt * __ldcg(t0 + i * kTileFloats + 8 * kHeadDim + 8 + h);
-            }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) dsum += __shfl_xor_sync(0xFFFFFFFFu, dsum, d);     // fixed butterfly order
-            den += dsum;
-            const int cnt = (int)min((int64_t)32, u1 - c0 + 1);
-            for (int j0 = 0; j0 < cnt; j0 += 4) {
-                float4 v[4];
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj)
-                    v[jj] = j0 + jj < cnt ? __ldcg(reinterpret_cast<const float4 *>(t0 + (c0 + j0 + jj) * kTileFloats + h * kHeadDim) + lane)
-                                          : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    const float wj = __shfl_sync(0xFFFFFFFFu, wgt, (j0 + jj) & 31);
-                    num.x = fmaf(wj, v[jj].x, num.x); num.y = fmaf(wj, v[jj].y, num.y);
-                    num.z = fmaf(wj, v[jj].z, num.z); num.w = fmaf(wj, v[jj].w, num.w);
-                }
-            }
-        }
-    }
-    const float inv = den > 0.f ? 1.f / den : 0.f;
-    const int64_t oi = ((int64_t)b * Hq + (int64_t)g * G + h) * kHeadDim + 4 * lane;
-    if (a.out_dtype == HMA_OUT_F32) {
-        reinterpret_cast<float4 *>(a.out)[oi >> 2] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
-    } else {
-        const uint32_t lo = f32_to_bf16_rne(num.x * inv) | ((uint32_t)f32_to_bf16_rne(num.y * inv) << 16);
-        const uint32_t hi = f32_to_bf16_rne(num.z * inv) | ((uint32_t)f32_to_bf16_rne(num.w * inv) << 16);
-        reinterpret_cast<uint2 *>(a.out)[oi >> 2] = make_uint2(lo, hi);
+    __syncthreads();
+#ifdef HMA_EXP_NOEPI
+    if (false) {
+#else
+    if (kMode == 0) {
+#endif
+        EpilogueArgs e;
+        e.out = a.out; e.tiles = a.tiles; e.tails = a.tails; e.counters = a.counters;
+        e.out_dtype = a.out_dtype; e.always_partial = a.always_partial; e.batch = a.batch;
+        e.cv.num_kv_heads = a.cv.num_kv_heads; e.cv.num_q_heads = a.cv.num_q_heads;
+#ifdef HMA_TRACE
+        e.trace = a.trace + (((int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * sp.nwk / sp.ctas : 0) + warp) * kTraceWords;
+#endif
+        cta_epilogue<kFmt>(e, ring, wr, wseg, cum, ecum, misc);
     }
 }
 
 // Merge for attention over two caches (a BFP8 prefix and a BF16 tail of every sequence): both main kernels ran with
-// always_partial, so every segment of either cache left one partial tile per worker that touched it; the softmax is
-// completed over the parts of both, prefix parts first, in worker order.  One CTA per (sequence, kv head), one warp
+// always_partial, so every segment of either cache left one partial tile per CTA that touched it; the softmax is
+// completed over the parts of both, prefix parts first, in CTA order.  One CTA per (sequence, kv head), one warp
 // per q head, four channels per lane.
 struct MergeSource {
     const int32_t *cum;      // pages, then pages + segment costs, before each sequence
     const float *tiles;
-    int max_workers;
+    int grid_ctas;           // CTAs the main kernel was launched with
+    int warps;               // warps per CTA of that kernel
 };
 
-__device__ __forceinline__ void segment_workers(const MergeSource &s, int batch, int Hkv, int b, int g, int64_t *u0, int *count)
+__device__ __forceinline__ void segment_parts(const MergeSource &s, int batch, int Hkv, int b, int g, int64_t *c0, int *count)
 {
     const int np = s.cum[b + 1] - s.cum[b];
     *count = 0;
-    *u0 = 0;
+    *c0 = 0;
     if (np == 0) return;
     const int32_t *ecum = s.cum + batch + 1;
     const int64_t WX = (int64_t)Hkv * ecum[batch];
-    const int64_t NWK = max((int64_t)1, min((int64_t)s.max_workers, WX / kMinRecords));
+    const Split sp = make_split(WX, s.grid_ctas, s.warps);
     const int64_t first = (int64_t)Hkv * ecum[b] + (int64_t)g * (np + kSegCost) + kSegCost;
-    *u0 = ((first + 1) * NWK - 1) / WX;
-    *count = (int)(((first + np) * NWK - 1) / WX - *u0 + 1);
+    segment_ctas(sp, WX, first, np, c0, count);
 }
 
 __global__ void __launch_bounds__(256) attn_merge_mixed_kernel(const AttnArgs a, MergeSource sa, MergeSource sb)
@@ -866,8 +1114,8 @@ __global__ void __launch_bounds__(256) attn_merge_mixed_kernel(const AttnArgs a,
     if (h >= G) return;
     int64_t ua, ub;
     int pa, pb;
-    segment_workers(sa, a.batch, Hkv, b, g, &ua, &pa);
-    segment_workers(sb, a.batch, Hkv, b, g, &ub, &pb);
+    segment_parts(sa, a.batch, Hkv, b, g, &ua, &pa);
+    segment_parts(sb, a.batch, Hkv, b, g, &ub, &pb);
     const int P = pa + pb;
     auto part = [&](int j) -> const float * {
         return j < pa ? sa.tiles + (ua + j + blockIdx.x) * kTileFloats : sb.tiles + (ub + (j - pa) + blockIdx.x) * kTileFloats;
@@ -923,24 +1171,40 @@ static size_t attn_smem_bytes(int batch)
 {
     using G = Geo<kFmt>;
     return (size_t)G::stages * G::record + (size_t)G::warps * G::scratch + G::stages * 8 + G::stages * 4 + (16 + 64) * 4 +
-           ((size_t)batch + 1) * 8;
+           (size_t)G::warps * 24 + ((size_t)batch + 1) * 8;
 }
 
+// Workspace layout: arrival counters | cum (two-cache merge only) | per-CTA tiles | per-segment tail tiles [| trace]
 static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 8 + 255) & ~(size_t)255; }
+static size_t counter_bytes(int batch, int hkv) { return ((size_t)batch * hkv * 4 + 255) & ~(size_t)255; }
+static size_t cta_tiles(int batch, int hkv) { return (size_t)kMaxCtas + (size_t)batch * hkv; }
 
 }  // namespace hma
 
 extern "C" size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *desc, int32_t batch)
 {
     if (!desc || batch < 0 || desc->num_kv_heads <= 0) return 0;
-    return hma::cum_bytes(batch) +
-           ((size_t)hma::kMaxCtas * hma::kWarps + (size_t)batch * desc->num_kv_heads) * hma::kTileFloats * 4;
+    const int hkv = desc->num_kv_heads;
+    size_t bytes = hma::counter_bytes(batch, hkv) + hma::cum_bytes(batch) +
+                   (hma::cta_tiles(batch, hkv) + (size_t)batch * hkv) * hma::kTileFloats * 4;
+#ifdef HMA_TRACE
+    bytes += (size_t)hma::kMaxCtas * hma::kWarps * hma::kTraceWords * 8;
+#endif
+    return bytes;
+}
+
+extern "C" hma_status_t hma_decode_attention_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!workspace) return HMA_ERR_INVALID_ARG;
+    if ((uintptr_t)workspace & 255u) return HMA_ERR_ALIGNMENT;
+    HMA_CUDA_OK(cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream));
+    return HMA_OK;
 }
 
 static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, const void *q, void *out, int32_t out_dtype,
                                      const int32_t *block_table, int32_t max_pages_per_seq, const int32_t *context_lens,
                                      int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes, void *stream,
-                                     int probe, int always_partial = 0, hma::AttnArgs *args_out = nullptr, int *workers_out = nullptr)
+                                     int probe, int always_partial = 0, hma::AttnArgs *args_out = nullptr, int *ctas_out = nullptr)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || batch < 0 || max_pages_per_seq < 0) return HMA_ERR_INVALID_ARG;
     if (out_dtype != HMA_OUT_BF16 && out_dtype != HMA_OUT_F32) return HMA_ERR_INVALID_ARG;
@@ -957,6 +1221,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     int dev = 0;
     HMA_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= hma::kMaxDevices) return HMA_ERR_UNSUPPORTED_SHAPE;
+    if (dev != cache->device) return HMA_ERR_INVALID_ARG;     // the handle's pointers belong to the device it was made on
     {
         std::lock_guard<std::mutex> guard(setup_lock);
         if (!sm_count[dev]) {
@@ -984,14 +1249,20 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.ctx = context_lens;
     a.batch = batch;
     a.sm_scale = sm_scale;
-    a.cum = (int32_t *)workspace;
-    a.tiles = (float *)((uint8_t *)workspace + hma::cum_bytes(batch));
+    const int hkv = cache->desc.num_kv_heads;
+    a.counters = (int32_t *)workspace;
+    a.cum = (int32_t *)((uint8_t *)workspace + hma::counter_bytes(batch, hkv));
+    a.tiles = (float *)((uint8_t *)a.cum + hma::cum_bytes(batch));
+    a.tails = a.tiles + hma::cta_tiles(batch, hkv) * hma::kTileFloats;
     a.always_partial = always_partial;
+#ifdef HMA_TRACE
+    a.trace = (unsigned long long *)(a.tails + (size_t)batch * hkv * hma::kTileFloats);
+#endif
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
     constexpr int tb = hma::Geo<HMA_KV_BFP8>::threads, tf = hma::Geo<HMA_KV_BF16>::threads;
-    // Both kernels are launched with programmatic stream serialisation: each may be placed on the SMs while its
-    // predecessor drains, and each waits on the grid dependency itself before it reads anything.
+    // The kernel is launched with programmatic stream serialisation: it may be placed on the SMs while its
+    // predecessor drains, and it waits on the grid dependency itself before it reads anything.
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -1009,14 +1280,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     else HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<2, HMA_KV_BFP8>, a));
     hma::count_launch();
     if (args_out) *args_out = a;
-    if (workers_out) *workers_out = n_ctas * (bf16 ? hma::Geo<HMA_KV_BF16>::warps : hma::Geo<HMA_KV_BFP8>::warps);
-    if (probe || always_partial) return HMA_OK;
-    cfg.gridDim = dim3((unsigned)(batch * cache->desc.num_kv_heads));
-    cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = 0;
-    HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_kernel, a,
-                                   n_ctas * (bf16 ? hma::Geo<HMA_KV_BF16>::warps : hma::Geo<HMA_KV_BFP8>::warps)));
-    hma::count_launch();
+    if (ctas_out) *ctas_out = n_ctas;
     return HMA_OK;
 }
 
@@ -1062,7 +1326,9 @@ extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, co
     cfg.stream = (cudaStream_t)stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    hma::MergeSource sa{aa.cum, aa.tiles, wa}, sb{ab.cum, ab.tiles, wb};
+    hma::MergeSource sa{aa.cum, aa.tiles, wa, hma::Geo<HMA_KV_BFP8>::warps}, sb{ab.cum, ab.tiles, wb, hma::Geo<HMA_KV_BF16>::warps};
+    if (prefix->desc.format != HMA_KV_BFP8) sa.warps = hma::Geo<HMA_KV_BF16>::warps;
+    if (tail->desc.format == HMA_KV_BFP8) sb.warps = hma::Geo<HMA_KV_BFP8>::warps;
     HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_mixed_kernel, aa, sa, sb));
     hma::count_launch();
     return HMA_OK;
@@ -1094,7 +1360,7 @@ extern "C" hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_
 // below until the process exits.
 namespace hma {
 constexpr int kStaticMaxSegments = 512;       // batch * num_kv_heads
-constexpr size_t kStaticWsBytes = 8192 + (size_t)(kMaxCtas * kWarps + kStaticMaxSegments) * kTileFloats * 4;   // 12.2 MiB
+constexpr size_t kStaticWsBytes = 2048 + 8192 + (size_t)(kMaxCtas + 2 * kStaticMaxSegments) * kTileFloats * 4;   // 4.8 MiB
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 static void *g_static_ws_ptr[kMaxDevices];    // device address of g_static_ws on each device, resolved on first use
 }  // namespace hma
@@ -1110,13 +1376,19 @@ extern "C" hma_status_t hma_decode_attention_static(const hma_cache_t *cache, in
     int dev = 0;
     HMA_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= hma::kMaxDevices) return HMA_ERR_STATIC_LIMIT;
-    if (!hma::g_static_ws_ptr[dev]) {
-        // In host code the array's name is only a handle: the device address has to be asked for, with the
-        // device that will run the kernels current.
-        void *p = nullptr;
-        HMA_CUDA_OK(cudaGetSymbolAddress(&p, hma::g_static_ws));
-        hma::g_static_ws_ptr[dev] = p;
+    void *ws = nullptr;
+    {
+        static std::mutex static_lock;
+        std::lock_guard<std::mutex> guard(static_lock);
+        if (!hma::g_static_ws_ptr[dev]) {
+            // In host code the array's name is only a handle: the device address has to be asked for, with the
+            // device that will run the kernels current.
+            void *p = nullptr;
+            HMA_CUDA_OK(cudaGetSymbolAddress(&p, hma::g_static_ws));
+            hma::g_static_ws_ptr[dev] = p;
+        }
+        ws = hma::g_static_ws_ptr[dev];
     }
     return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
-                            hma::g_static_ws_ptr[dev], hma::kStaticWsBytes, stream, 0);
+                            ws, hma::kStaticWsBytes, stream, 0);
 }

@@ -100,6 +100,7 @@ extern "C" hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, in
                                                     const int32_t *context_lens, int32_t batch, float sm_scale, void *stream)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || batch < 0 || max_pages_per_seq < 0) return HMA_ERR_INVALID_ARG;
+    if (!hma::on_cache_device(cache)) return HMA_ERR_INVALID_ARG;
     if (out_dtype != HMA_OUT_BF16 && out_dtype != HMA_OUT_F32) return HMA_ERR_INVALID_ARG;
     if (batch == 0) return HMA_OK;
     if (!q || !out || !block_table || !context_lens) return HMA_ERR_INVALID_ARG;

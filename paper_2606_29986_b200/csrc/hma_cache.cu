@@ -89,7 +89,6 @@ extern "C" const char *hma_status_string(int32_t status)
         case HMA_ERR_ALIGNMENT: return "misaligned pointer";
         case HMA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case HMA_ERR_CUDA: return "CUDA runtime error";
-        case HMA_ERR_DEVICE_FLAGGED: return "device flagged an anomaly";
         case HMA_ERR_STATIC_LIMIT: return "request exceeds the built-in scratch array of hma_decode_attention_static";
         default: return "unknown status";
     }

@@ -94,7 +94,15 @@ struct hma_cache {
     int device;
 };
 
-namespace hma { void note_cuda_error(cudaError_t e); }
+namespace hma {
+void note_cuda_error(cudaError_t e);
+// A handle holds pointers of the device it was created on: every launch path refuses to run with another device current.
+inline bool on_cache_device(const hma_cache *c)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == c->device;
+}
+}  // namespace hma
 
 #define HMA_CUDA_OK(expr)                          \
     do {                                           \

@@ -7,7 +7,7 @@ namespace hma {
 
 // Four elements of one block -> four BF16 bit patterns, bit-exact for every (E, byte) pair.
 // The byte s<<7|m is first spread to the FP16 pattern s<<15|m, the FP16 subnormal +-m * 2^-24 (two integer
-// instructions per pair: section 3.3's "shifts, masks, ORs and a bitcast"); widening to fp32 and multiplying by
+// instructions per pair: the integer-only decode of section 3.3); widening to fp32 and multiplying by
 // 2^(E-109) (one factor while it is a normal fp32 number, two exact power-of-two factors above that) gives
 // m * 2^(E-133) exactly (fp32 subnormals and overflow to Inf included); its upper 16 bits are the BF16 value.
 // The sign rides along, so m = 0 keeps its sign.
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int wh
     }
 }
 
-// The elementwise strawman of section 3.3 ("naive elementwise reconstruction"): one thread per output element, byte
+// The elementwise strawman of section 3.3: one thread per output element, byte
 // loads straight from the cache, integer bit assembly, two-byte stores.  Kept only as the comparison point.
 __global__ void __launch_bounds__(256) dequant_naive_kernel(CacheView cv, int which, const int32_t *__restrict__ page_ids,
                                                             int64_t token_begin, int64_t n_tokens, uint16_t *__restrict__ out)
@@ -184,6 +184,7 @@ extern "C" hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t 
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || (which != 0 && which != 1) || token_begin < 0 || n_tokens < 0)
         return HMA_ERR_INVALID_ARG;
+    if (!hma::on_cache_device(cache)) return HMA_ERR_INVALID_ARG;
     if (n_tokens == 0) return HMA_OK;
     if (!page_ids || !out_bf16) return HMA_ERR_INVALID_ARG;
     if ((uintptr_t)out_bf16 & 15u) return HMA_ERR_ALIGNMENT;
@@ -205,6 +206,7 @@ extern "C" hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const
                                                  int64_t n_tokens, void *out_bf16, void *stream)
 {
     if (!cache || token_begin < 0 || n_tokens < 0) return HMA_ERR_INVALID_ARG;
+    if (!hma::on_cache_device(cache)) return HMA_ERR_INVALID_ARG;
     if (n_tokens == 0) return HMA_OK;
     if (!page_ids || !out_bf16) return HMA_ERR_INVALID_ARG;
     if ((uintptr_t)out_bf16 & 15u) return HMA_ERR_ALIGNMENT;
@@ -228,6 +230,7 @@ extern "C" hma_status_t hma_bfp8_dequant_bf16_naive(const hma_cache_t *cache, in
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || (which != 0 && which != 1) || token_begin < 0 || n_tokens < 0)
         return HMA_ERR_INVALID_ARG;
+    if (!hma::on_cache_device(cache)) return HMA_ERR_INVALID_ARG;
     if (n_tokens == 0) return HMA_OK;
     if (!page_ids || !out_bf16) return HMA_ERR_INVALID_ARG;
     const int64_t total = n_tokens * cache->desc.num_kv_heads * hma::kHeadDim;

@@ -63,6 +63,7 @@ extern "C" hma_status_t hma_bfp8_encode_rows(const hma_cache_t *cache, const voi
                                              void *wire_rowmajor, void *stream)
 {
     if (!cache || n_rows < 0 || (x_is_bf16 != 0 && x_is_bf16 != 1)) return HMA_ERR_INVALID_ARG;
+    if (!hma::on_cache_device(cache)) return HMA_ERR_INVALID_ARG;
     if (n_rows == 0) return HMA_OK;
     if (!x || !wire_rowmajor) return HMA_ERR_INVALID_ARG;
     if (((uintptr_t)x & 15u) || ((uintptr_t)wire_rowmajor & 7u)) return HMA_ERR_ALIGNMENT;

@@ -201,19 +201,17 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
                                   void *stream)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers) return HMA_ERR_INVALID_ARG;
+    if (!hma::on_cache_device(cache)) return HMA_ERR_INVALID_ARG;
     if (wire_layout != HMA_WIRE_TILE32 && wire_layout != HMA_WIRE_ROWMAJOR && wire_layout != HMA_WIRE_BF16_ROWS) return HMA_ERR_INVALID_ARG;
     if (wire_layout == HMA_WIRE_BF16_ROWS && cache->desc.format != HMA_KV_BF16) return HMA_ERR_INVALID_ARG;
     if (n_shards < 1 || n_shards > hma::kMaxShards || !k_wires || !v_wires || !head_begins || !head_counts) return HMA_ERR_INVALID_ARG;
     if (token_begin < 0 || n_tokens < 0) return HMA_ERR_INVALID_ARG;
     hma::IngestArgs a = {};
     int heads = 0;
-    unsigned seen = 0;
     for (int s = 0; s < n_shards; ++s) {
         if (head_begins[s] < 0 || head_counts[s] <= 0 || head_begins[s] + head_counts[s] > cache->desc.num_kv_heads) return HMA_ERR_INVALID_ARG;
-        for (int h = head_begins[s]; h < head_begins[s] + head_counts[s]; ++h) {
-            if (seen & (1u << (h & 31))) return HMA_ERR_INVALID_ARG;     // two shards may not write the same head
-            seen |= 1u << (h & 31);
-        }
+        for (int t = 0; t < s; ++t)                                      // two shards may not write the same head
+            if (head_begins[s] < head_begins[t] + head_counts[t] && head_begins[t] < head_begins[s] + head_counts[s]) return HMA_ERR_INVALID_ARG;
         a.k_wire[s] = (const uint8_t *)k_wires[s];
         a.v_wire[s] = (const uint8_t *)v_wires[s];
         a.head_begin[s] = head_begins[s];

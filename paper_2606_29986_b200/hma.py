@@ -14,14 +14,14 @@ _LIB_PATH = os.path.join(_HERE, "libhma.so")
 
 HMA_OK = 0
 HMA_ERR_INVALID_ARG, HMA_ERR_UNSUPPORTED_SHAPE, HMA_ERR_ALIGNMENT = 1, 2, 3
-HMA_ERR_WORKSPACE_TOO_SMALL, HMA_ERR_CUDA, HMA_ERR_DEVICE_FLAGGED = 4, 5, 6
+HMA_ERR_WORKSPACE_TOO_SMALL, HMA_ERR_CUDA = 4, 5
 HMA_ERR_STATIC_LIMIT = 7
 HMA_KV_BFP8, HMA_KV_BF16 = 0, 1
 HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR, HMA_WIRE_BF16_ROWS = 0, 1, 2
 HMA_OUT_BF16, HMA_OUT_F32 = 0, 1
 HMA_KEYS_AS_QUERIES, HMA_KEYS_INTERLEAVED = 0, 1
 HMA_FLAG_BAD_PAGE_ATTENTION, HMA_FLAG_BAD_PAGE_INGEST, HMA_FLAG_BAD_PAGE_DEQUANT, HMA_FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
-HMA_FLAG_BAD_VALUE_ENCODE = 16
+HMA_FLAG_BAD_VALUE_ENCODE, HMA_FLAG_EXPONENT_RANGE = 16, 32
 
 
 class CacheDesc(ctypes.Structure):
@@ -46,9 +46,11 @@ def lib():
     """The loaded C-ABI library.  Raises if libhma.so is missing (build it with build.py)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(_LIB_PATH):
-            raise ImportError("libhma.so is not built: run `python -m paper_2606_29986_b200.build`")
-        L = ctypes.CDLL(_LIB_PATH)
+        # HMA_LIBRARY selects another build of the same sources (the instrumented libhma_trace.so), nothing else
+        path = os.environ.get("HMA_LIBRARY") or _LIB_PATH
+        if not os.path.exists(path):
+            raise ImportError("%s is not built: run `python -m paper_2606_29986_b200.build`" % os.path.basename(path))
+        L = ctypes.CDLL(path)
         vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
         L.hma_cache_layer_bytes.restype = sz
         L.hma_cache_layer_bytes.argtypes = [ctypes.POINTER(CacheDesc)]
@@ -63,6 +65,8 @@ def lib():
                                                  ctypes.POINTER(i32), ctypes.POINTER(i32), vp, i64, i64, vp]
         L.hma_decode_attention_workspace_bytes.restype = sz
         L.hma_decode_attention_workspace_bytes.argtypes = [ctypes.POINTER(CacheDesc), i32]
+        L.hma_decode_attention_workspace_init.restype = i32
+        L.hma_decode_attention_workspace_init.argtypes = [vp, sz, vp]
         L.hma_decode_attention.restype = i32
         L.hma_decode_attention.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp, sz, vp]
         L.hma_decode_attention_static.restype = i32
@@ -71,6 +75,8 @@ def lib():
         L.hma_decode_attention_static_limit_bytes.argtypes = []
         L.hma_kv_read_probe.restype = i32
         L.hma_kv_read_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
+        L.hma_hbm_read_probe.restype = i32
+        L.hma_hbm_read_probe.argtypes = [vp, sz, vp, vp]
         L.hma_attention_alu_probe.restype = i32
         L.hma_attention_alu_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
         L.hma_decode_attention_mixed.restype = i32
@@ -181,6 +187,22 @@ def hma_decode_attention_workspace_bytes(desc, batch):
     return int(lib().hma_decode_attention_workspace_bytes(ctypes.byref(desc), batch))
 
 
+def hma_decode_attention_workspace_init(workspace, stream=None):
+    """Zero-fills a workspace (required once before its first use; calls leave it ready for the next one)."""
+    _check(lib().hma_decode_attention_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "hma_decode_attention_workspace_init")
+
+
+def new_workspace(desc, batch, device="cuda", copies=1):
+    """A torch uint8 tensor sized for hma_decode_attention on `batch` sequences (`copies` = 2 for the two-cache call,
+    each half rounded up to 256 bytes) and initialised through hma_decode_attention_workspace_init."""
+    n = (hma_decode_attention_workspace_bytes(desc, batch) + 255) // 256 * 256
+    ws = torch.empty(copies * n, dtype=torch.uint8, device=device)
+    with torch.cuda.device(ws.device):
+        hma_decode_attention_workspace_init(ws)
+    return ws
+
+
 def hma_decode_attention(cache, layer, q, out, block_table, context_lens, sm_scale, workspace, stream=None):
     out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
     _check(lib().hma_decode_attention(cache.handle, layer, _ptr(q), _ptr(out), out_dtype, _ptr(block_table),
@@ -215,6 +237,11 @@ def hma_attention_alu_probe(cache, layer, block_table, context_lens, workspace, 
     _check(lib().hma_attention_alu_probe(cache.handle, layer, _ptr(block_table), block_table.shape[1], _ptr(context_lens),
                                          context_lens.shape[0], _ptr(workspace), workspace.numel() * workspace.element_size(),
                                          _stream(stream)), "hma_attention_alu_probe")
+
+
+def hma_hbm_read_probe(src, sink, stream=None):
+    """Contiguous streaming read of the whole tensor `src` (a read-only memory ceiling); `sink` is a 4-byte device tensor."""
+    _check(lib().hma_hbm_read_probe(_ptr(src), src.numel() * src.element_size(), _ptr(sink), _stream(stream)), "hma_hbm_read_probe")
 
 
 def hma_decode_attention_mixed(prefix, tail, layer, q, out, prefix_table, prefix_lens, tail_table, tail_lens, sm_scale,

@@ -1,0 +1,86 @@
+"""Per-warp timing of the attention kernel, from the instrumented build of the library (-DHMA_TRACE).
+
+    python -m paper_2606_29986_b200.trace [--workload NAME] [--layers N] [--reps R]
+
+Builds libhma_trace.so if needed, runs hma_decode_attention on a benchmark workload with that image, reads the
+time stamps every worker (warp) left behind its partial tiles, and prints a summary: when warps start, when their
+first record lands, when they leave the record loop, how that spreads inside an SM and between SMs.  The default
+library carries none of the instrumentation; the numbers printed here are about where time goes, not bench values.
+"""
+import argparse
+import os
+import sys
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+TRACE_WORDS = 16
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="qwen3-32b-b32-ctx8k")
+    ap.add_argument("--layers", type=int, default=4)
+    ap.add_argument("--reps", type=int, default=5)
+    args = ap.parse_args()
+
+    from paper_2606_29986_b200 import build
+    os.environ["HMA_LIBRARY"] = os.environ.get("HMA_LIBRARY") or build.build(trace=True)
+    sys.path.insert(0, ROOT)
+    import torch
+    import bench
+    from paper_2606_29986_b200 import hma
+    dev = torch.device("cuda", 0)
+    wl = bench.Workload(args.workload, dev, with_bf16=False, with_ingest=False, layers=args.layers)
+    ws_bytes = hma.hma_decode_attention_workspace_bytes(wl.caches["bfp8"].desc, wl.B)
+    n_workers = 192 * 16
+    trace_off = ws_bytes - n_workers * TRACE_WORDS * 8
+    assert wl.workspace.numel() >= ws_bytes
+
+    def run(l):
+        wl.workspace[trace_off:ws_bytes].zero_()
+        # two calls back to back: the second one starts the way a call inside a decode pass does
+        hma.hma_decode_attention(wl.caches["bfp8"], (l + 1) % wl.L, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wl.workspace)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        hma.hma_decode_attention(wl.caches["bfp8"], l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wl.workspace)
+        e1.record()
+        torch.cuda.synchronize()
+        tr = wl.workspace[trace_off:ws_bytes].view(torch.int64).cpu().numpy().reshape(-1, TRACE_WORDS).copy()
+        return tr[tr[:, 1] > 0], e0.elapsed_time(e1) * 1e3
+
+    for i in range(3):
+        run(i % wl.L)
+    rows = []
+    for rep in range(args.reps):
+        tr, call_us = run(rep % wl.L)
+        t0 = tr[:, 1].min()
+        us = lambda col: (tr[:, col] - t0) / 1e3
+        smid, wait, pro, first, loop_end, done, recs = tr[:, 0], us(1), us(2), us(3), us(4), us(5), tr[:, 6]
+        epi = tr[:, 8] > 0
+        cyc = lambda a, b: ((tr[:, a] - tr[:, b])[epi & (tr[:, a] > 0) & (tr[:, b] > 0)] / 1.9e3)      # us at about 1.9 GHz
+        sms = np.unique(smid)
+        sm_end = np.array([loop_end[smid == s].max() for s in sms])
+        sm_mean = np.array([loop_end[smid == s].mean() for s in sms])
+        within = np.array([loop_end[smid == s].max() - loop_end[smid == s].min() for s in sms])
+        rows.append(dict(call_us=call_us, workers=len(tr), sms=len(sms), enter_spread=wait.max(), prologue_end=pro.mean(),
+                         first_mean=first.mean(), first_max=first.max(), end_min=loop_end.min(), end_mean=loop_end.mean(),
+                         end_p90=np.percentile(loop_end, 90), end_max=loop_end.max(), done_max=done.max(),
+                         sm_mean_min=sm_mean.min(), sm_mean_max=sm_mean.max(), sm_mean_std=sm_mean.std(),
+                         epi_walk_setup_us=cyc(12, 8).mean(), epi_seg1_us=cyc(13, 12).mean(), epi_seg2_us=cyc(14, 13).mean(),
+                         epi_seg3_us=cyc(15, 14).mean(), epi_reduce_us=cyc(9, 8).mean(), epi_arrive_us=cyc(10, 9).mean(),
+                         epi_merge_us=cyc(11, 10).mean(), epi_total_us_mean=cyc(11, 8).mean(), epi_total_us_max=cyc(11, 8).max(),
+                         within_mean=within.mean(), within_max=within.max(), recs_min=int(recs.min()), recs_max=int(recs.max()),
+                         slow=[int(x) for x in sms[np.argsort(sm_end)[-8:]]]))
+    keys = [k for k in rows[0] if k != "slow"]
+    print("workload %s, %d layers built, %d traced calls (all times in us after the first warp passed the grid-dependency wait)" %
+          (args.workload, wl.L, len(rows)))
+    print("| quantity | " + " | ".join("call %d" % i for i in range(len(rows))) + " |")
+    print("|---|" + "---|" * len(rows))
+    for k in keys:
+        print("| %s | " % k + " | ".join(("%.2f" % r[k]) if isinstance(r[k], float) else str(r[k]) for r in rows) + " |")
+    print("SMs whose last warp leaves the loop last, per call:", [r["slow"] for r in rows])
+
+
+if __name__ == "__main__":
+    main()

@@ -53,8 +53,7 @@ class Scenario:
                     hma.hma_kv_ingest_layer_shards(self.cache, l, kss, vss, wire_layout, [s * hs for s in range(shards)],
                                                    [hs] * shards, pages, 0, T)
         torch.cuda.synchronize()
-        ws = hma.hma_decode_attention_workspace_bytes(self.desc, self.B)
-        self.workspace = torch.empty(ws, dtype=torch.uint8, device=device)
+        self.workspace = hma.new_workspace(self.desc, self.B, device)
 
     def attention(self, layer=0, out_dtype=torch.bfloat16, simple=False, sm_scale=None, q=None):
         q = self.q if q is None else q

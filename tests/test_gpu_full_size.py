@@ -49,7 +49,7 @@ def test_longest_supported_context_and_limits():
     out = torch.zeros_like(q)
     tbl = torch.zeros((big, 1), dtype=torch.int32, device="cuda")
     ctx = torch.zeros(big, dtype=torch.int32, device="cuda")
-    ws = torch.empty(hma.hma_decode_attention_workspace_bytes(sc.desc, big), dtype=torch.uint8, device="cuda")
+    ws = hma.new_workspace(sc.desc, big)
     with pytest.raises(hma.HmaError) as e:
         hma.hma_decode_attention(sc.cache, 0, q, out, tbl, ctx, 0.1, ws)
     assert e.value.status == hma.HMA_ERR_UNSUPPORTED_SHAPE

@@ -45,7 +45,7 @@ def test_bfp8_prefix_plus_bf16_tail(hq, hkv):
     tail_lens = [5, 0, 40, 130, 17]
     sc = Scenario(prefix_lens, hq, hkv, seed=300 + hq, permute=True)
     tail, ttable, tlens, ks, vs = _tail_scenario(sc, tail_lens, 301 + hq)
-    ws = torch.empty(2 * (hma.hma_decode_attention_workspace_bytes(sc.desc, sc.B) + 256), dtype=torch.uint8, device="cuda")
+    ws = hma.new_workspace(sc.desc, sc.B, copies=2)
     ref64, _ = orc.decode_attention_mixed(bf16_bits(sc.q), sc.k_wires[0], sc.v_wires[0], ks, vs, hkv)
     outs = {}
     for dt in (torch.float32, torch.bfloat16):
