@@ -29,7 +29,7 @@
  *   - errors: invalid arguments return a status and enqueue nothing.  Device-side anomalies never
  *     trap: a page id outside [0, num_pages) is skipped and a bit is set in the cache's flag word.
  *   - supported geometry: head_dim 128, 16 tokens per page, 16-element blocks,
- *     num_q_heads / num_kv_heads in 1..8.
+ *     num_q_heads / num_kv_heads in 1..8, at most 64 kv heads.
  */
 #ifndef HMA_H
 #define HMA_H
@@ -159,17 +159,23 @@ hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32
  *   out          device, [batch][num_q_heads][128] BF16 or F32 per out_dtype
  *   block_table  device int32 [batch][max_pages_per_seq]
  *   context_lens device int32 [batch]; every entry <= max_pages_per_seq*16
- *   workspace    device, 256-byte aligned, >= hma_decode_attention_workspace_bytes(...) bytes;
- *                contents need no initialisation and are clobbered
+ *   workspace    device, 256-byte aligned, >= hma_decode_attention_workspace_bytes(...) bytes.  It must have been
+ *                zero-filled once (hma_decode_attention_workspace_init, or any memset to 0) before the first call that
+ *                uses it: it holds one arrival counter per (sequence, kv head) on which the CTAs that share a segment
+ *                meet.  Every call leaves the counters at zero again, so one workspace serves any number of calls, of
+ *                any shape it is large enough for; the rest of it is clobbered.  A call that reports
+ *                HMA_FLAG_WAIT_TIMEOUT may leave counters behind: zero the workspace again before its next use.
+ *                Calls that may overlap on the GPU need a workspace each.
  *   batch        at most 1024 (HMA_ERR_UNSUPPORTED_SHAPE beyond)
  * Accuracy: fp32 accumulation.  Block exponents above 250 (values beyond 2^117) are outside the supported
  * range: the call still returns, HMA_FLAG_EXPONENT_RANGE is raised and the affected rows are not meaningful.
- * Launches: two kernels per call (attention, then a small merge of the per-worker partials), both with
- * programmatic stream serialisation; each waits on the grid dependency before it reads any input, so the
- * usual stream order holds whatever kernel precedes the call.  The first call on a device sets the kernels'
- * shared-memory attributes.
+ * Launches: one kernel per call (the cross-split reduction happens inside it), with programmatic stream
+ * serialisation; it waits on the grid dependency before it reads any input, so the usual stream order holds
+ * whatever kernel precedes the call.  The first call on a device sets the kernels' shared-memory attributes.
  */
 size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *desc, int32_t batch);
+/* Zero-fills a workspace on `stream` (see hma_decode_attention: needed once per workspace, before its first use). */
+hma_status_t hma_decode_attention_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,
                                   const void *q, void *out, int32_t out_dtype,
                                   const int32_t *block_table, int32_t max_pages_per_seq,
@@ -180,7 +186,7 @@ hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,
  * hma_decode_attention for callers that cannot allocate.  (The paper has no counterpart: this exists for
  * the way the library gets embedded, not for the method.)  A decode loop that fixed its memory pool at
  * start-up, or code running where the host framework forbids allocation, has no workspace to pass; here
- * the scratch is a 12.2 MiB array that is part of the library image on every GPU that loads it
+ * the scratch is a 5.1 MiB array that is part of the library image on every GPU that loads it
  * (hma_decode_attention_static_limit_bytes returns the exact size).  The call allocates and frees nothing.
  *
  *   - same arguments and results as hma_decode_attention, without the workspace pair; the outputs of the
@@ -190,9 +196,10 @@ hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,
  *     enqueues nothing.
  *   - the first call on each device looks up the array's device address (with that device current) and sets
  *     kernel attributes; make that first call outside any stream capture.
- *   - all calls on a device share the one array.  Nothing in it has to start at zero and a call never reads
- *     what an earlier call left, but two calls that overlap on the GPU (different streams) race on it:
- *     keep such calls on one stream or order them with events.
+ *   - all calls on a device share the one array.  Its arrival counters start at zero (the loader zero-fills the
+ *     array) and every call returns them to zero; nothing else in it is read before it is written.  Two calls
+ *     that overlap on the GPU (different streams) race on it: keep such calls on one stream or order them with
+ *     events.
  */
 size_t hma_decode_attention_static_limit_bytes(void);
 hma_status_t hma_decode_attention_static(const hma_cache_t *cache, int32_t layer,
@@ -216,8 +223,9 @@ hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer
  * holding the KV of tokens generated since, which the paper's decode side produces in BF16, section 3.1; the
  * paper does not say where those live, this is one answer, hma_bfp8_encode_rows the other).  One softmax over
  * both.  Same q/out/sm_scale conventions as hma_decode_attention; both caches must have the same head counts and
- * HMA_KEYS_AS_QUERIES.  workspace: 2 * hma_decode_attention_workspace_bytes(desc, batch), rounded up to 256 each.
- * Three launches: attention over each cache leaving partials, then a merge that completes the softmax.
+ * HMA_KEYS_AS_QUERIES.  workspace: 2 * hma_decode_attention_workspace_bytes(desc, batch), rounded up to 256 each
+ * (no zero-filling needed for this call).
+ * Three launches: attention over each cache leaving one partial per CTA and segment, then a merge that completes the softmax.
  */
 hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
                                         const void *q, void *out, int32_t out_dtype,
@@ -303,6 +311,17 @@ hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_t layer, co
  * the kernel may add to (it practically never does; it keeps the loads alive). */
 hma_status_t hma_hbm_read_probe(const void *src, size_t bytes, void *sink4, void *stream);
 
+
+#ifdef HMA_TRACE
+/* Only in the instrumented build of the library (compiled with -DHMA_TRACE; the default build has neither this entry
+ * point nor the per-warp time stamps).  Failure drill for the bounded waits inside the attention kernel: in the next
+ * hma_decode_attention launch of this process, record number `record` of the launch's work list (records are counted
+ * sequence by sequence, kv head by kv head, page by page) is announced to its arrival barrier as 16 bytes longer than
+ * the copy that fills it, and waits give up after `spin_limit` polls.  The copy lands in full, the barrier never
+ * completes, the waiting warp gives up, raises HMA_FLAG_WAIT_TIMEOUT and the kernel returns: nothing faults and nothing
+ * hangs.  Outputs of the segments that CTA worked on are void. */
+hma_status_t hma_trace_arm_timeout_drill(int64_t record, uint32_t spin_limit);
+#endif
 
 #ifdef __cplusplus
 }

@@ -44,6 +44,7 @@ struct Geo {
 constexpr int kTileFloats = 8 * kHeadDim + 16;    // partial tile in global memory: o[8][128], m[8], l[8]
 constexpr int kPieceStride = kHeadDim + 4;        // floats per head of a partial parked in a ring slot (bank-conflict-free)
 constexpr int kPieceFloats = 8 * kPieceStride + 16;   // 1072 floats = 4288 B: fits the smallest ring slot (4352 B)
+static_assert(kPieceFloats * 4 <= kBfp8Record && kTileFloats * 4 <= kBfp8Record, "a parked partial must fit a ring slot");
 constexpr uint32_t kSpinLimit = 1u << 20;           // polls of a bounded wait
 constexpr uint32_t kSuspendNs = 2000;              // a failed poll may keep the thread parked this long
 constexpr int kMaxBatch = 1024;
@@ -70,13 +71,15 @@ struct AttnArgs {
     int always_partial;             // 1: never write `out`; every segment leaves per-CTA partial tiles (two-cache attention)
 #ifdef HMA_TRACE
     unsigned long long *trace;      // workspace, after the tiles: kTraceWords words per worker (see trace_stamp)
+    long long drill_record;         // timeout drill: this record of the work list is announced 16 bytes too long (-1: none)
+    uint32_t spin_limit;            // polls of a bounded wait (the drill shortens it)
 #endif
 };
 
 // Per-warp timing instrumentation, compiled in only with -DHMA_TRACE (a separate library image; the default build
 // carries none of it).  Each worker writes kTraceWords 64-bit words after the partial tiles of the workspace:
 //   0 SM id   1 after the grid-dependency wait   2 end of the prologue   3 first record landed
-//   4 end of the record loop   5 after the last partial/output store   6 records taken   7 unused
+//   4 end of the record loop   5 after the last partial/output store   6 records taken   7 kernel entry (before the wait)
 //   8 CTA-level reduction begins (all warps of the CTA are done)   9 its segments are reduced
 //   10 arrivals on the shared segments' counters are done   11 the CTA leaves   12 walk begins   13-15 first segments done
 // Words 1-5 are %globaltimer nanoseconds; words 8-15 are the SM's cycle counter (only differences inside a CTA mean anything).
@@ -127,9 +130,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait: gives up after kSpinLimit polls (or when another thread of the CTA already gave up),
 // raises the CTA's abort word and the device flag, and returns false.  Nothing spins forever.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_word, uint32_t *flags)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_word, uint32_t *flags, uint32_t limit = kSpinLimit)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_word) return false;
     }
@@ -288,194 +291,210 @@ struct EpilogueArgs {       // what the reduction needs of AttnArgs, by value (r
 #else
 #define HMA_TRACE_EPI(a, i)  do { } while (0)
 #endif
-__device__ __forceinline__ void store_pair(void *out, int out_dtype, int64_t oi, float x, float y)
+// ---- group descriptors: what the CTA-level reduction has to do, worked out once per CTA right after the warps know
+// their ranges (everybody is waiting for first data then), so that nothing of it is on the critical path at the end
+constexpr int kMaxGroups = 32;       // more than a CTA can have: a group holds a boundary between two of its (at most 16) warps, or one of its own ends
+constexpr int kGroupInts = 6;        // sequence, kv head, member mask, flags (1 whole segment, 2 has tail, tail warp << 8), parts, first CTA
+
+// One full warp plans the groups of the CTA.  A group is a segment of the CTA's record range that no single warp held
+// entirely: `members` are the warps whose last partial (ring slot 0) belongs to it; a warp that held the segment's end
+// and went on contributes its tail tile (ring slot 1) after them.  If the CTA holds only part of the segment,
+// parts = number of CTAs that share it, first CTA = the lowest.  gstate[0] = number of groups.
+template <int kFmt>
+__device__ __noinline__ void plan_groups(int always_partial, int Hkv, int B, const long long *wr, const int *wseg, const int *cum,
+                                         const int *ecum, int *gdesc, int *gstate)
 {
-    if (out_dtype == HMA_OUT_F32) *reinterpret_cast<float2 *>(reinterpret_cast<float *>(out) + oi) = make_float2(x, y);
-    else *reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(out) + oi) = f32_to_bf16_rne(x) | ((uint32_t)f32_to_bf16_rne(y) << 16);
+    constexpr int kWarps = Geo<kFmt>::warps;
+    const int lane = threadIdx.x & 31;
+    const long long my_lo = lane < kWarps ? wr[2 * lane] : 0, my_hi = lane < kWarps ? wr[2 * lane + 1] : 0;   // lane i: range of warp i
+    const unsigned have = __ballot_sync(0xFFFFFFFFu, my_lo < my_hi);
+    if (have == 0) {
+        if (lane == 0) gstate[0] = 0;
+        return;
+    }
+    const long long clo = __shfl_sync(0xFFFFFFFFu, my_lo, __ffs(have) - 1), chi = __shfl_sync(0xFFFFFFFFu, my_hi, 31 - __clz(have));
+    int sb = wseg[2 * (__ffs(have) - 1)], sg = wseg[2 * (__ffs(have) - 1) + 1];     // segment of the CTA's first record
+    int npb = cum[sb + 1] - cum[sb], n = 0;
+    for (;;) {
+        const long long s_lo = (long long)Hkv * cum[sb] + (long long)sg * npb, s_hi = s_lo + npb;
+        if (s_lo >= chi || n == kMaxGroups) break;
+        const long long lo = max(s_lo, clo), hi = min(s_hi, chi);
+        unsigned mem = __ballot_sync(0xFFFFFFFFu, my_lo < my_hi && my_lo < hi && my_hi > lo);     // warps with records of this segment
+        const int i1 = 31 - __clz(mem);
+        const bool one_warp_whole = (mem & (mem - 1)) == 0 && __shfl_sync(0xFFFFFFFFu, my_lo <= s_lo && my_hi >= s_hi, i1);
+        if (!one_warp_whole) {
+            const bool has_tail = __shfl_sync(0xFFFFFFFFu, my_hi > s_hi, i1);     // the last warp went on into the next segment
+            if (has_tail) mem &= ~(1u << i1);
+            const bool whole_seg = lo == s_lo && hi == s_hi;
+            if (lane == 0) {
+                int parts = 0;
+                int64_t c0 = 0;
+                if (!whole_seg && !always_partial) {
+                    const int64_t WX = (int64_t)Hkv * ecum[B];
+                    const Split sp = make_split(WX, (int)gridDim.x, kWarps);
+                    const int64_t first = (int64_t)Hkv * ecum[sb] + (int64_t)sg * (npb + kSegCost) + kSegCost;   // cost position of the first record
+                    segment_ctas(sp, WX, first, npb, &c0, &parts);
+                }
+                int *d = gdesc + n * kGroupInts;
+                d[0] = sb; d[1] = sg; d[2] = (int)mem; d[3] = (whole_seg ? 1 : 0) | (has_tail ? 2 : 0) | (i1 << 8);
+                d[4] = parts; d[5] = (int)c0;
+            }
+            ++n;
+        }
+        if (++sg == Hkv) {
+            sg = 0;
+            do { ++sb; } while (sb < B && cum[sb + 1] == cum[sb]);
+            if (sb >= B) break;
+            npb = cum[sb + 1] - cum[sb];
+        }
+    }
+    if (lane == 0) gstate[0] = n;
 }
 
-template <int kFmt>
-__device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *ring, const long long *wr, const int *wseg,
-                                          const int *cum, const int *ecum, int *misc)
+__device__ __forceinline__ void store_quad(void *out, int out_dtype, int64_t oi, float x, float y, float z, float w)
 {
-    constexpr int kWarps = Geo<kFmt>::warps, kThreads = Geo<kFmt>::threads, kRecord = Geo<kFmt>::record;
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv, B = a.batch;
+    if (out_dtype == HMA_OUT_F32) *reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + oi) = make_float4(x, y, z, w);
+    else
+        *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(out) + oi) =
+            make_uint2(f32_to_bf16_rne(x) | ((uint32_t)f32_to_bf16_rne(y) << 16), f32_to_bf16_rne(z) | ((uint32_t)f32_to_bf16_rne(w) << 16));
+}
+__device__ __forceinline__ float4 lds_f4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
+// ---------------------------------------------------------------- CTA-level reduction and cross-CTA merge
+// Runs once per CTA after all of its warps have parked their last partial (a function of its own so that its
+// registers do not weigh on the record loop).  Work items are (group, q head): one warp each, four channels per
+// lane; lane i weighs the partial of warp i (lane kWarps: the tail tile), so the weights of a group cost one round of
+// loads and two shuffle reductions, and the 128-vectors are then summed in warp order, four loads in flight.
+template <int kFmt>
+__device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *ring,
+                                          int *misc, const int *gdesc, const int *gstate)
+{
+    constexpr int kWarps = Geo<kFmt>::warps, kRecord = Geo<kFmt>::record;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
     const bool aborted = misc[0] != 0;            // outputs of this CTA are void (and flagged); arrivals still happen
     HMA_TRACE_EPI(a, 8);
-    // lane i of every warp holds the record range of warp i
-    const long long my_lo = lane < kWarps ? wr[2 * lane] : 0, my_hi = lane < kWarps ? wr[2 * lane + 1] : 0;
-    const unsigned have = __ballot_sync(0xFFFFFFFFu, my_lo < my_hi);
-    if (have == 0) return;
-    const long long clo = __shfl_sync(0xFFFFFFFFu, my_lo, __ffs(have) - 1), chi = __shfl_sync(0xFFFFFFFFu, my_hi, 31 - __clz(have));
     const uint32_t ring_s = smem_u32(ring);
-    const int sb0 = wseg[2 * (__ffs(have) - 1)], sg0 = wseg[2 * (__ffs(have) - 1) + 1];     // segment of the CTA's first record
-    // Calls fn(sb, sg, npb, whole_seg, members, has_tail, tail_warp) for every segment of the CTA's range that is not
-    // finished already (one warp holding it entirely).  `members`: the warps whose last partial (ring slot 0) belongs
-    // to the segment; has_tail: in addition, after the members in order, the tail tile in ring slot 1 of tail_warp.
-    auto walk = [&](auto &&fn) {
-        int sb = sb0, sg = sg0, npb = cum[sb0 + 1] - cum[sb0];
-        for (;;) {
-            const long long s_lo = (long long)Hkv * cum[sb] + (long long)sg * npb, s_hi = s_lo + npb;
-            if (s_lo >= chi) break;
-            const long long lo = max(s_lo, clo), hi = min(s_hi, chi);
-            unsigned mem = __ballot_sync(0xFFFFFFFFu, my_lo < my_hi && my_lo < hi && my_hi > lo);     // warps with records of this segment
-            const int i1 = 31 - __clz(mem);
-            const bool one_warp_whole = (mem & (mem - 1)) == 0 && __shfl_sync(0xFFFFFFFFu, my_lo <= s_lo && my_hi >= s_hi, i1);
-            if (!one_warp_whole) {
-                // the last warp of the group may have gone on into the next segment: its partial is the segment's tail tile
-                const bool tail_in_global = __shfl_sync(0xFFFFFFFFu, my_hi > s_hi, i1);
-                if (tail_in_global) mem &= ~(1u << i1);
-                fn(sb, sg, npb, lo == s_lo && hi == s_hi, mem, tail_in_global, i1);
-            }
-            if (++sg == Hkv) {
-                sg = 0;
-                do { ++sb; } while (sb < B && cum[sb + 1] == cum[sb]);
-                if (sb >= B) break;
-                npb = cum[sb + 1] - cum[sb];
-            }
-        }
-    };
-    HMA_TRACE_EPI(a, 12);
-    int n_groups = 0;
     int n_open = 0;                               // segments this CTA shares with other CTAs (at most its first and last)
-    walk([&](int sb, int sg, int npb, bool whole_seg, unsigned mem, bool tail_in_global, int tail_warp) {
-        const int64_t seg = (int64_t)sb * Hkv + sg;
-        if (!aborted) {
-            const uint32_t gtail = ring_s + (tail_warp * kDepth + 1) * kRecord;      // dense tile layout, in the ring slot 1 of the warp that wrote it
-            const int i0 = mem ? __ffs(mem) - 1 : 0, i1 = mem ? 31 - __clz(mem) : -1;
-#ifdef HMA_EXP_NOREDUCE
-            if (false)
-#endif
-            for (int idx = tid; idx < 8 * (kHeadDim / 2); idx += kThreads) {
-                // a warp works on one head: lane i weighs the partial of warp i, lane kWarps the tail tile
-                const int h = idx / (kHeadDim / 2), ch = 2 * (idx % (kHeadDim / 2));
-                if (h >= G) break;
+    {
+        const int n = gstate[0];
+        if (!aborted)
+            for (int item = warp; item < n * 8; item += kWarps) {
+                const int h = item & 7;
+                if (h >= G) continue;
+                const int *d = gdesc + (item >> 3) * kGroupInts;
+                const int sb = d[0], sg = d[1];
+                const unsigned mem = (unsigned)d[2];
+                const bool whole_seg = d[3] & 1, has_tail = d[3] & 2;
+                const uint32_t gtail = ring_s + ((d[3] >> 8) * kDepth + 1) * kRecord;      // dense tile layout
                 float mine_m = -INFINITY, mine_l = 0.f;
                 if (lane < kWarps && (mem >> lane & 1u)) {
                     const uint32_t pc = ring_s + lane * kDepth * kRecord + (8 * kPieceStride + h) * 4;
                     mine_m = __uint_as_float(lds32(pc)); mine_l = __uint_as_float(lds32(pc + 32));
-                } else if (lane == kWarps && tail_in_global) {
+                } else if (lane == kWarps && has_tail) {
                     mine_m = __uint_as_float(lds32(gtail + (8 * kHeadDim + h) * 4)); mine_l = __uint_as_float(lds32(gtail + (8 * kHeadDim + 8 + h) * 4));
                 }
+                // every 128-vector load is issued before the weights are needed; summed in warp order, the tail tile last
+                float4 v[kWarps + 1];
+#pragma unroll
+                for (int i = 0; i < kWarps; ++i) {
+                    v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (mem >> i & 1u) v[i] = lds_f4(ring_s + i * kDepth * kRecord + (h * kPieceStride + 4 * lane) * 4);
+                }
+                v[kWarps] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (has_tail) v[kWarps] = lds_f4(gtail + (h * kHeadDim + 4 * lane) * 4);
                 float M = mine_m;
 #pragma unroll
-                for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
+                for (int dd = 16; dd > 0; dd >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, dd));
                 const float mine_w = mine_m == -INFINITY ? 0.f : ex2f(mine_m - M);
                 float den = mine_w * mine_l;
 #pragma unroll
-                for (int d = 16; d > 0; d >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, d);      // fixed butterfly order
-                float2 vt = make_float2(0.f, 0.f);
-                if (tail_in_global)
-                    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(vt.x), "=f"(vt.y) : "r"(gtail + (h * kHeadDim + ch) * 4));
-                float nx = 0.f, ny = 0.f;
-                for (int i = i0; i <= i1; i += 4) {            // in warp order, four loads in flight
-                    float2 v[4];
+                for (int dd = 16; dd > 0; dd >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, dd);      // fixed butterfly order
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        v[j] = make_float2(0.f, 0.f);
-                        if (mem >> (i + j) & 1u)
-                            asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v[j].x), "=f"(v[j].y)
-                                         : "r"(ring_s + (i + j) * kDepth * kRecord + (h * kPieceStride + ch) * 4));
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float wgt = __shfl_sync(0xFFFFFFFFu, mine_w, (i + j) & 31);      // 0 for a warp that is no member
-                        nx = fmaf(wgt, v[j].x, nx); ny = fmaf(wgt, v[j].y, ny);
-                    }
+                for (int i = 0; i <= kWarps; ++i) {
+                    const float wgt = __shfl_sync(0xFFFFFFFFu, mine_w, i);      // 0 for a warp that is no member
+                    acc.x = fmaf(wgt, v[i].x, acc.x); acc.y = fmaf(wgt, v[i].y, acc.y);
+                    acc.z = fmaf(wgt, v[i].z, acc.z); acc.w = fmaf(wgt, v[i].w, acc.w);
                 }
-                {
-                    const float wgt = __shfl_sync(0xFFFFFFFFu, mine_w, kWarps);
-                    nx = fmaf(wgt, vt.x, nx); ny = fmaf(wgt, vt.y, ny);
-                }
-#ifdef HMA_EXP_NOSTORE
-                if (nx == 1.2345f)
-#endif
                 if (whole_seg && !a.always_partial) {
                     const float inv = den > 0.f ? 1.f / den : 0.f;
-                    store_pair(a.out, a.out_dtype, ((int64_t)sb * Hq + (int64_t)sg * G + h) * kHeadDim + ch, nx * inv, ny * inv);
+                    store_quad(a.out, a.out_dtype, ((int64_t)sb * Hq + (int64_t)sg * G + h) * kHeadDim + 4 * lane, acc.x * inv, acc.y * inv,
+                               acc.z * inv, acc.w * inv);
                 } else {
-                    float *tp = a.tiles + ((int64_t)blockIdx.x + seg) * kTileFloats;
-                    *reinterpret_cast<float2 *>(tp + h * kHeadDim + ch) = make_float2(nx, ny);
-                    if (ch == 0) { tp[8 * kHeadDim + h] = M; tp[8 * kHeadDim + 8 + h] = den; }
+                    float *tp = a.tiles + ((int64_t)blockIdx.x + (int64_t)sb * Hkv + sg) * kTileFloats;
+                    *reinterpret_cast<float4 *>(tp + h * kHeadDim + 4 * lane) = acc;
+                    if (lane == 0) { tp[8 * kHeadDim + h] = M; tp[8 * kHeadDim + 8 + h] = den; }
                 }
             }
-        }
-        if (!whole_seg && !a.always_partial && n_open < 2) {
-#ifdef HMA_EXP_NODIV
-            if (tid == 32 * n_open) { misc[4 + 4 * n_open] = 2; misc[5 + 4 * n_open] = 0; misc[6 + 4 * n_open] = sb; misc[7 + 4 * n_open] = sg; }
-            if (false) {
-#else
-            if (tid == 32 * n_open) {
-#endif
-                // this thread will register the CTA on the segment's arrival counter: which CTAs share the segment
-                const int64_t WX = (int64_t)Hkv * ecum[B];
-                const Split sp = make_split(WX, (int)gridDim.x, kWarps);
-                const int64_t first = (int64_t)Hkv * ecum[sb] + (int64_t)sg * (npb + kSegCost) + kSegCost;   // cost position of the first record
-                int64_t c0;
-                int parts;
-                segment_ctas(sp, WX, first, npb, &c0, &parts);
-                misc[4 + 4 * n_open] = parts; misc[5 + 4 * n_open] = (int)c0;
-                misc[6 + 4 * n_open] = sb; misc[7 + 4 * n_open] = sg;
+        for (int g = 0; g < n; ++g) {                 // note the shared segments (the same in every thread)
+            const int *d = gdesc + g * kGroupInts;
+            if (d[4] > 0 && n_open < 2) {
+                if (tid == 0) { misc[4 + 4 * n_open] = d[4]; misc[5 + 4 * n_open] = d[5]; misc[6 + 4 * n_open] = d[0]; misc[7 + 4 * n_open] = d[1]; }
+                ++n_open;
             }
-            ++n_open;
         }
-        if (n_groups < 3) HMA_TRACE_EPI(a, 13 + n_groups);
-        ++n_groups;
-    });
+    }
     HMA_TRACE_EPI(a, 9);
     if (n_open == 0) return;                      // the same for every thread of the CTA
     // Arrival: the CTA's tile stores happen before the barrier, the release of the arriving thread's atomic carries
     // them (cumulativity) to whoever acquires the counter after the last arrival.
     __syncthreads();
-    if ((tid & 31) == 0 && (tid >> 5) < n_open) {
-        const int k = tid >> 5;
-        int32_t *ctr = a.counters + (int64_t)misc[6 + 4 * k] * Hkv + misc[7 + 4 * k];
+    if (lane == 0 && warp < n_open) {
+        int32_t *ctr = a.counters + (int64_t)misc[6 + 4 * warp] * Hkv + misc[7 + 4 * warp];
         int prev;
         asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(ctr) : "memory");
-        const bool last = prev == misc[4 + 4 * k] - 1;
+        const bool last = prev == misc[4 + 4 * warp] - 1;
         if (last) *ctr = 0;                       // everybody has arrived: leave the counter ready for the next call
-        else misc[4 + 4 * k] = 0;
+        else misc[4 + 4 * warp] = 0;
     }
     __syncthreads();
     HMA_TRACE_EPI(a, 10);
-    for (int k = 0; k < n_open; ++k) {
+    for (int item = warp; item < n_open * 8; item += kWarps) {
+        const int k = item >> 3, h = item & 7;
         const int parts = misc[4 + 4 * k];
-        if (parts == 0) continue;                 // another CTA will arrive later and finish this segment
+        if (parts == 0 || h >= G) continue;       // another CTA will arrive later and finish this segment
         const int ob = misc[6 + 4 * k], og = misc[7 + 4 * k];
         const float *t0 = a.tiles + ((int64_t)misc[5 + 4 * k] + (int64_t)ob * Hkv + og) * kTileFloats;       // part i is at t0 + i * kTileFloats
-        for (int idx = tid; idx < 8 * (kHeadDim / 2); idx += kThreads) {
-            const int h = idx / (kHeadDim / 2), ch = 2 * (idx % (kHeadDim / 2));
-            if (h >= G) break;
-            // parts in CTA order, four at a time (one trip to L2 for the usual two to four parts), running maximum
-            float M = -INFINITY, nx = 0.f, ny = 0.f, den = 0.f;
-            for (int p0 = 0; p0 < parts; p0 += 4) {
-                float mi[4], li[4];
-                float2 v[4];
+        // parts in CTA order, four at a time (one trip to L2 for the usual two to four parts), running maximum
+        float M = -INFINITY, den = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p0 = 0; p0 < parts; p0 += 4) {
+            float mi[4], li[4];
+            float4 v[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float *tp = t0 + (int64_t)(p0 + j) * kTileFloats;
-                    const bool ok = p0 + j < parts;
-                    mi[j] = ok ? __ldcg(tp + 8 * kHeadDim + h) : -INFINITY;
-                    li[j] = ok ? __ldcg(tp + 8 * kHeadDim + 8 + h) : 0.f;
-                    v[j] = ok ? __ldcg(reinterpret_cast<const float2 *>(tp + h * kHeadDim + ch)) : make_float2(0.f, 0.f);
-                }
-                const float Mn = fmaxf(fmaxf(fmaxf(mi[0], mi[1]), fmaxf(mi[2], mi[3])), M);
-                const float keep = M == -INFINITY ? 0.f : ex2f(M - Mn);
-                nx *= keep; ny *= keep; den *= keep;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float wgt = mi[j] == -INFINITY ? 0.f : ex2f(mi[j] - Mn);
-                    nx = fmaf(wgt, v[j].x, nx); ny = fmaf(wgt, v[j].y, ny);
-                    den = fmaf(wgt, li[j], den);
-                }
-                M = Mn;
+            for (int j = 0; j < 4; ++j) {
+                const float *tp = t0 + (int64_t)(p0 + j) * kTileFloats;
+                const bool ok = p0 + j < parts;
+                mi[j] = ok ? __ldcg(tp + 8 * kHeadDim + h) : -INFINITY;
+                li[j] = ok ? __ldcg(tp + 8 * kHeadDim + 8 + h) : 0.f;
+                v[j] = ok ? __ldcg(reinterpret_cast<const float4 *>(tp + h * kHeadDim) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            const float inv = den > 0.f ? 1.f / den : 0.f;
-            store_pair(a.out, a.out_dtype, ((int64_t)ob * Hq + (int64_t)og * G + h) * kHeadDim + ch, nx * inv, ny * inv);
+            const float Mn = fmaxf(fmaxf(fmaxf(mi[0], mi[1]), fmaxf(mi[2], mi[3])), M);
+            const float keep = M == -INFINITY ? 0.f : ex2f(M - Mn);
+            acc.x *= keep; acc.y *= keep; acc.z *= keep; acc.w *= keep; den *= keep;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float wgt = mi[j] == -INFINITY ? 0.f : ex2f(mi[j] - Mn);
+                acc.x = fmaf(wgt, v[j].x, acc.x); acc.y = fmaf(wgt, v[j].y, acc.y);
+                acc.z = fmaf(wgt, v[j].z, acc.z); acc.w = fmaf(wgt, v[j].w, acc.w);
+                den = fmaf(wgt, li[j], den);
+            }
+            M = Mn;
         }
+        const float inv = den > 0.f ? 1.f / den : 0.f;
+        store_quad(a.out, a.out_dtype, ((int64_t)ob * Hq + (int64_t)og * G + h) * kHeadDim + 4 * lane, acc.x * inv, acc.y * inv, acc.z * inv,
+                   acc.w * inv);
     }
     HMA_TRACE_EPI(a, 11);
+#ifdef HMA_TRACE
+    if ((threadIdx.x & 31) == 0) a.trace[12] = trace_now();     // wall clock at the CTA's exit
+#endif
 }
 
 // kMode 0: attention.  1: stream the records through the ring, no arithmetic (bandwidth probe).
@@ -495,7 +514,9 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     int *misc = stage_ok + kStages;                                               // [0] abort word, [4..12) epilogue, [16..80) scan scratch
     long long *wr = reinterpret_cast<long long *>(misc + 16 + 64);                // [kWarps][2] record range of each warp
     int *wseg = reinterpret_cast<int *>(wr + 2 * kWarps);                         // [kWarps][2] sequence and kv head of its first record
-    int *cum = wseg + 2 * kWarps;                                                 // [batch + 1] pages before each sequence
+    int *gdesc = wseg + 2 * kWarps;                                               // [kMaxGroups][kGroupInts] plan of the CTA-level reduction
+    int *gstate = gdesc + kMaxGroups * kGroupInts;                                // [4]
+    int *cum = gstate + 4;                                                        // [batch + 1] pages before each sequence
     int *ecum = cum + a.batch + 1;                                                // [batch + 1] same, plus kSegCost per non-empty sequence
     volatile int *abort_word = misc;
 
@@ -505,11 +526,15 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(bars + s), 1);
         misc[0] = 0;
+        misc[1] = 0;                     // warps that have published their record range
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     // The kernel is launched with programmatic stream serialisation: its CTAs may be placed while the previous
     // kernel of the stream drains.  Nothing that a predecessor could have written is read before this wait.
+#ifdef HMA_TRACE
+    const unsigned long long tr_entry = trace_now();
+#endif
     asm volatile("griddepcontrol.wait;" ::: "memory");
 #ifdef HMA_TRACE
     const unsigned long long tr_wait = trace_now();
@@ -572,8 +597,21 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     const int64_t u = ubase + warp;                                 // this warp's worker index (if warp < nmine)
     if (lane == 0) { wr[2 * warp] = 0; wr[2 * warp + 1] = 0; }      // no records until shown otherwise
 
+    // Every warp publishes its record range exactly once; the warp that publishes last plans the CTA-level reduction
+    // (who has to combine what at the end) while everybody is still waiting for first data.
+    auto publish = [&]() {
+        __syncwarp();
+        int cnt = 0;
+        if (lane == 0) { __threadfence_block(); cnt = atomicAdd(&misc[1], 1); }
+        cnt = __shfl_sync(0xFFFFFFFFu, cnt, 0);
+        if (cnt == kWarps - 1 && kMode == 0) {
+            __threadfence_block();
+            plan_groups<kFmt>(a.always_partial, Hkv, B, wr, wseg, cum, ecum, gdesc, gstate);
+        }
+    };
+
     do {    // ---- this warp's share of the work list; `break` leaves for the CTA-level reduction ----
-    if (warp >= nmine) break;
+    if (warp >= nmine) { publish(); break; }
     if (kMode == 0 && !a.always_partial)                          // empty sequences get rows of zeros
         for (int64_t b = u; b < B; b += NWK)
             if (cum[b + 1] == cum[b])
@@ -593,11 +631,12 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         return (int64_t)Hkv * cum[lo] + (int64_t)gg * n + max(0, r - kSegCost);
     };
     const int64_t wlo = records_before(u * WX / NWK), whi = records_before((u + 1) * WX / NWK);
-    if (wlo >= whi) break;
+    if (wlo >= whi) { publish(); break; }
     const int Rw = (int)(whi - wlo);
     HMA_TRACE_STAMP(a, u, 0, (unsigned long long)trace_smid());
     HMA_TRACE_STAMP(a, u, 1, tr_wait);
     HMA_TRACE_STAMP(a, u, 2, tr_pro);
+    HMA_TRACE_STAMP(a, u, 7, tr_entry);
     HMA_TRACE_STAMP(a, u, 6, (unsigned long long)Rw);
 
     // the segment (b, g) and page that hold record wlo
@@ -651,7 +690,12 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         if (lane == 0) {
             if (off != kNoRecord) {
                 stage_ok[warp * kDepth + islot] = 1;
+#ifdef HMA_TRACE
+                // the drill: the copy delivers kRecord bytes, the barrier waits for 16 more, the bounded wait runs out
+                mbar_arrive_expect_tx(full0 + 8 * islot, kRecord + (wlo + kissue == a.drill_record ? 16 : 0));
+#else
                 mbar_arrive_expect_tx(full0 + 8 * islot, kRecord);
+#endif
                 bulk_load(ring0 + islot * kRecord, a.cv.layer + (uint64_t)off * 128u, kRecord, full0 + 8 * islot, policy);
             } else {
                 stage_ok[warp * kDepth + islot] = 0;
@@ -666,6 +710,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     // Only the first record is requested now; the other slots are armed after the first segment's Q loads have been
     // issued, so that across the GPU every warp's first record is ahead of anybody's second in the memory queues.
     issue();
+    publish();
 
     // ---- consumer state ----
     const int gq = lane >> 2, t4 = lane & 3;
@@ -762,7 +807,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         const float l0 = lacc[0], l1 = lacc[1];
         const int h0 = 2 * t4, h1 = 2 * t4 + 1;
         // a softmax sum that is not finite: scores overflowed fp32 (K exponents beyond the supported range)
-        if (!(l0 < INFINITY) || !(l1 < INFINITY)) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);
+        if (kMode == 0 && (!(l0 < INFINITY) || !(l1 < INFINITY))) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);
         const int64_t ob = ((int64_t)b * Hq + (int64_t)g * G) * kHeadDim;
         if (kMode == 2 && a.batch >= 0) return;    // the issue-rate probe never stores, but keeps its arithmetic live
         if (whole && !a.always_partial) {
@@ -823,7 +868,11 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         const uint32_t sp = ring0 + slot * kRecord;
         const int s_idx = warp * kDepth + slot;
         if (kMode < 2) {
+#ifdef HMA_TRACE
+            alive = mbar_wait(full0 + 8 * slot, par, abort_word, a.cv.flags, a.spin_limit);
+#else
             alive = mbar_wait(full0 + 8 * slot, par, abort_word, a.cv.flags);
+#endif
             if (!alive) break;
 #ifdef HMA_TRACE
             if (k == 0) HMA_TRACE_STAMP(a, u, 3, trace_now());
@@ -863,7 +912,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                     emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
                     emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
                     const int Rnew = max(Rmine, emax);
-                    if (Rnew > 250) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);   // beyond the supported range
+                    if (kMode == 0 && Rnew > 250) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);   // beyond the supported range
     #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
@@ -1065,11 +1114,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     } while (0);
 
     __syncthreads();
-#ifdef HMA_EXP_NOEPI
-    if (false) {
-#else
     if (kMode == 0) {
-#endif
         EpilogueArgs e;
         e.out = a.out; e.tiles = a.tiles; e.tails = a.tails; e.counters = a.counters;
         e.out_dtype = a.out_dtype; e.always_partial = a.always_partial; e.batch = a.batch;
@@ -1077,7 +1122,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
 #ifdef HMA_TRACE
         e.trace = a.trace + (((int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * sp.nwk / sp.ctas : 0) + warp) * kTraceWords;
 #endif
-        cta_epilogue<kFmt>(e, ring, wr, wseg, cum, ecum, misc);
+        cta_epilogue<kFmt>(e, ring, misc, gdesc, gstate);
     }
 }
 
@@ -1171,12 +1216,14 @@ static size_t attn_smem_bytes(int batch)
 {
     using G = Geo<kFmt>;
     return (size_t)G::stages * G::record + (size_t)G::warps * G::scratch + G::stages * 8 + G::stages * 4 + (16 + 64) * 4 +
-           (size_t)G::warps * 24 + ((size_t)batch + 1) * 8;
+           (size_t)G::warps * 24 + (kMaxGroups * kGroupInts + 4) * 4 + ((size_t)batch + 1) * 8;
 }
 
 // Workspace layout: arrival counters | cum (two-cache merge only) | per-CTA tiles | per-segment tail tiles [| trace]
 static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 8 + 255) & ~(size_t)255; }
-static size_t counter_bytes(int batch, int hkv) { return ((size_t)batch * hkv * 4 + 255) & ~(size_t)255; }
+// The counters sit at the head of the workspace in a region of one size for every call, whatever its batch and head
+// count, so that calls of different shapes can share a workspace without one's tiles landing on the other's counters.
+static size_t counter_bytes(int, int) { return (size_t)kMaxBatch * kMaxKvHeads * 4; }
 static size_t cta_tiles(int batch, int hkv) { return (size_t)kMaxCtas + (size_t)batch * hkv; }
 
 }  // namespace hma
@@ -1192,6 +1239,19 @@ extern "C" size_t hma_decode_attention_workspace_bytes(const hma_cache_desc_t *d
 #endif
     return bytes;
 }
+
+#ifdef HMA_TRACE
+// Instrumented build only: arms the timeout drill for the next attention launch of the calling process.
+static long long g_drill_record = -1;
+static uint32_t g_drill_spin_limit = 1000;
+extern "C" hma_status_t hma_trace_arm_timeout_drill(int64_t record, uint32_t spin_limit)
+{
+    if (record < 0 || spin_limit == 0) return HMA_ERR_INVALID_ARG;
+    g_drill_record = record;
+    g_drill_spin_limit = spin_limit;
+    return HMA_OK;
+}
+#endif
 
 extern "C" hma_status_t hma_decode_attention_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
 {
@@ -1257,6 +1317,9 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.always_partial = always_partial;
 #ifdef HMA_TRACE
     a.trace = (unsigned long long *)(a.tails + (size_t)batch * hkv * hma::kTileFloats);
+    a.drill_record = g_drill_record;
+    a.spin_limit = g_drill_record >= 0 ? g_drill_spin_limit : hma::kSpinLimit;
+    g_drill_record = -1;
 #endif
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
@@ -1360,7 +1423,7 @@ extern "C" hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_
 // below until the process exits.
 namespace hma {
 constexpr int kStaticMaxSegments = 512;       // batch * num_kv_heads
-constexpr size_t kStaticWsBytes = 2048 + 8192 + (size_t)(kMaxCtas + 2 * kStaticMaxSegments) * kTileFloats * 4;   // 4.8 MiB
+constexpr size_t kStaticWsBytes = (size_t)kMaxBatch * kMaxKvHeads * 4 + 8192 + (size_t)(kMaxCtas + 2 * kStaticMaxSegments) * kTileFloats * 4;   // 5.1 MiB
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 static void *g_static_ws_ptr[kMaxDevices];    // device address of g_static_ws on each device, resolved on first use
 }  // namespace hma

@@ -17,6 +17,7 @@ static bool desc_ok(const hma_cache_desc_t *d)
     if (!d) return false;
     if (d->head_dim != hma::kHeadDim || d->page_tokens != hma::kPageTokens || d->bfp_block != hma::kBlock) return false;
     if (d->num_layers <= 0 || d->num_kv_heads <= 0 || d->num_q_heads <= 0 || d->num_pages <= 0) return false;
+    if (d->num_kv_heads > hma::kMaxKvHeads) return false;
     if (d->num_q_heads % d->num_kv_heads) return false;
     int g = d->num_q_heads / d->num_kv_heads;
     if (g < 1 || g > hma::kMaxGroup) return false;

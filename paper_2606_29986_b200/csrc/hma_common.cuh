@@ -18,6 +18,7 @@ constexpr int kBfp8Record = 2 * kBfp8Half;                 // 4352
 constexpr int kBf16Half = 4096;
 constexpr int kBf16Record = 2 * kBf16Half;                 // 8192
 constexpr int kMaxGroup = 8;                               // q heads per kv head
+constexpr int kMaxKvHeads = 64;                            // kv heads per layer
 
 struct CacheView {
     uint8_t *layer;        // base of one layer

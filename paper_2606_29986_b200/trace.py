@@ -67,8 +67,7 @@ def main():
                          first_mean=first.mean(), first_max=first.max(), end_min=loop_end.min(), end_mean=loop_end.mean(),
                          end_p90=np.percentile(loop_end, 90), end_max=loop_end.max(), done_max=done.max(),
                          sm_mean_min=sm_mean.min(), sm_mean_max=sm_mean.max(), sm_mean_std=sm_mean.std(),
-                         epi_walk_setup_us=cyc(12, 8).mean(), epi_seg1_us=cyc(13, 12).mean(), epi_seg2_us=cyc(14, 13).mean(),
-                         epi_seg3_us=cyc(15, 14).mean(), epi_reduce_us=cyc(9, 8).mean(), epi_arrive_us=cyc(10, 9).mean(),
+                         epi_reduce_us=cyc(9, 8).mean(), epi_arrive_us=cyc(10, 9).mean(),
                          epi_merge_us=cyc(11, 10).mean(), epi_total_us_mean=cyc(11, 8).mean(), epi_total_us_max=cyc(11, 8).max(),
                          within_mean=within.mean(), within_max=within.max(), recs_min=int(recs.min()), recs_max=int(recs.max()),
                          slow=[int(x) for x in sms[np.argsort(sm_end)[-8:]]]))

@@ -83,9 +83,10 @@ def parity_metrics(got, ref64):
 def check_attention(out_f32, out_bf16, ref64):
     """The parity bar.  F32 output: max-abs <= 1e-2 and rel-L2 <= 2e-3 against the fp64 oracle, literally.
     BF16 output: bit-for-bit the round-to-nearest-even of that F32 output (so the only extra error is the output
-    format's own rounding), and |err| <= 1e-2 + 2^-8 |ref| everywhere.  A literal rel-L2 bar on the BF16 output is not
-    meaningful: the oracle's own result rounded to BF16 already shows rel-L2 1.3e-3 .. 2.4e-3 on these workloads
-    (BF16 keeps 8 significant bits), which is reported next to the kernel's numbers instead."""
+    format's own rounding), |err| <= 1e-2 + 2^-8 |ref| everywhere, max-abs <= 1e-2 literally on the elements small
+    enough for BF16 to resolve that (|ref| < 2), and rel-L2 <= 2e-3 literally wherever the oracle's own result
+    rounded to BF16 meets that bar, else within 5 % of that rounding floor (BF16 keeps 8 significant bits: on long
+    contexts with outlier channels the floor alone is 1.3e-3 .. 2.4e-3)."""
     ma, rl = parity_metrics(out_f32, ref64)
     assert ma <= 1e-2 and rl <= 2e-3, ("f32 output", ma, rl)
     want16 = torch.from_numpy(np.ascontiguousarray(out_f32, np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
@@ -94,6 +95,11 @@ def check_attention(out_f32, out_bf16, ref64):
     err = np.abs(got - ref64)
     mb, rb = parity_metrics(got, ref64)
     assert (err <= 1e-2 + 2.0 ** -8 * np.abs(ref64)).all(), ("bf16 output bound", (err - 2.0 ** -8 * np.abs(ref64)).max())
+    small = np.abs(ref64) < 2.0
+    assert not small.any() or err[small].max() <= 1e-2, ("bf16 max-abs where BF16 resolves it", err[small].max())
+    floor16 = torch.from_numpy(np.ascontiguousarray(ref64)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    _, floor = parity_metrics(bf16_bits_to_f64(floor16), ref64)
+    assert rb <= (2e-3 if floor <= 1.9e-3 else 1.05 * floor), ("bf16 rel-L2", rb, "rounding floor", floor)
     return ma, rl, mb, rb
 
 

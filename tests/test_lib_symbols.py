@@ -8,9 +8,15 @@ import pytest
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def declared_functions():
+def declared_functions(instrumented=False):
+    """Functions include/hma.h declares: those of the default build, or those that only the -DHMA_TRACE build has."""
     text = open(os.path.join(ROOT, "include", "hma.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    blocks = re.findall(r"#ifdef HMA_TRACE(.*?)#endif", text, flags=re.S)
+    if instrumented:
+        text = "\n".join(blocks)
+    else:
+        text = re.sub(r"#ifdef HMA_TRACE.*?#endif", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(hma_[a-z0-9_]+)\s*\(", text)))
 
 
@@ -26,6 +32,17 @@ def test_library_exports_every_declared_symbol():
     lib = ctypes.CDLL(path)
     for name in declared_functions():
         assert hasattr(lib, name), name
+
+
+def test_instrumented_build_exports_its_extra_symbols():
+    from paper_2606_29986_b200 import build
+    extra = declared_functions(instrumented=True)
+    assert extra == ["hma_trace_arm_timeout_drill"]
+    plain, traced = ctypes.CDLL(build.build()), ctypes.CDLL(build.build(trace=True))
+    for name in extra:
+        assert hasattr(traced, name) and not hasattr(plain, name), name
+    for name in declared_functions():
+        assert hasattr(traced, name), name
 
 
 def test_host_only_calls():
