@@ -119,13 +119,10 @@ class Workload:
                     self.sample_wires[(l, b)] = (kw.cpu().numpy(), vw.cpu().numpy())
             torch.cuda.synchronize(device)
         # the arriving request: TILE32 wire, 4 shards x (hkv/4) heads, every layer, K and V
-        # decode runs on a high-priority stream, the arriving request's ingest on a low-priority one
-        try:
-            lo_pri, hi_pri = torch.cuda.Stream.priority_range()
-        except Exception:
-            lo_pri, hi_pri = 0, -1
-        self.side = torch.cuda.Stream(device, priority=lo_pri)
-        self.main = torch.cuda.Stream(device, priority=hi_pri)
+        # decode and the arriving request's ingest run on two streams of equal priority (measured: giving either one
+        # a higher priority makes the step slower, because the favoured kernel's CTAs then sit on freed SMs waiting)
+        self.side = torch.cuda.Stream(device)
+        self.main = torch.cuda.Stream(device)
         if self.ingest_tokens:
             hs = self.hkv // 4
             one = synth.rowmajor_to_tile32(synth.make_kv_wire(hs, self.ingest_tokens, 4242, device)).reshape(-1)

@@ -135,6 +135,164 @@ __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int wh
     }
 }
 
+// ---------------------------------------------------------------- the streaming rebuild of BFP8 pages
+// A few long-lived CTAs per SM walk all (layer, page, kv head) records of the request: each 4352-byte record arrives by
+// one bulk async copy into a four-deep ring; 256 threads rebuild it (K: one thread = 8 channels of a token, one 16-byte
+// store; V: a word of the record holds four tokens of one channel, so one thread takes four channels of two tokens,
+// transposes the bytes in registers and writes two 8-byte pieces); every store instruction of a warp covers whole
+// 256-byte output rows.  Bit-exact like the kernel above (same dequant4).
+constexpr int kRebuildStages = 4;
+constexpr int kRebuildThreads = 256;
+constexpr uint32_t kRebuildSpin = 1u << 22;
+
+struct RebuildArgs {
+    void *const *layers;          // device array of layer pointers (NULL: cv.layer is the only layer)
+    const int32_t *page_ids;
+    int64_t token_begin, n_tokens;
+    uint16_t *out_k, *out_v;      // rows [n_tokens][Hkv][128] of layer 0 (NULL: tensor not wanted)
+    int64_t layer_stride;         // elements between consecutive layers of one tensor
+    int32_t n_layers, n_pages;
+};
+
+__device__ __forceinline__ uint32_t rb_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool rb_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 1000;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+__global__ void __launch_bounds__(kRebuildThreads) rebuild_stream_kernel(CacheView cv, RebuildArgs a)
+{
+    __shared__ __align__(128) uint8_t ring[kRebuildStages][kBfp8Record];
+    __shared__ __align__(8) uint64_t bars[kRebuildStages];
+    __shared__ int ok_stage[kRebuildStages];
+    const int tid = threadIdx.x, Hkv = cv.num_kv_heads;
+    const int64_t n_items = (int64_t)a.n_layers * a.n_pages * Hkv;      // item = (layer, page, head), head fastest
+    if (tid == 0) {
+        for (int s = 0; s < kRebuildStages; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(rb_smem_u32(bars + s)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    auto load = [&](int64_t item, int stage) {      // thread 0 only
+        const int h = (int)(item % Hkv);
+        const int64_t lp = item / Hkv;
+        const int pg = (int)(lp % a.n_pages), l = (int)(lp / a.n_pages);
+        const int32_t pid = a.page_ids[pg];
+        const uint32_t bar = rb_smem_u32(bars + stage);
+        if (pid < 0 || pid >= cv.num_pages) {
+            ok_stage[stage] = 0;
+            atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_DEQUANT);
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+            return;
+        }
+        ok_stage[stage] = 1;
+        const uint8_t *base = a.layers ? (const uint8_t *)a.layers[l] : cv.layer;
+        // the whole record, or only the half that is wanted
+        const int off = a.out_k ? 0 : kBfp8Half, bytes = (a.out_k && a.out_v) ? kBfp8Record : kBfp8Half;
+        const uint8_t *src = base + ((int64_t)pid * Hkv + h) * (int64_t)kBfp8Record + off;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(rb_smem_u32(ring[stage]) + off),
+                     "l"(src), "r"(bytes), "r"(bar)
+                     : "memory");
+    };
+    if (tid == 0)
+        for (int s = 0; s < kRebuildStages; ++s) {
+            const int64_t item = blockIdx.x + (int64_t)s * gridDim.x;
+            if (item < n_items) load(item, s);
+        }
+    const bool relayout = cv.key_layout == HMA_KEYS_INTERLEAVED;
+    const int64_t first_page = a.token_begin / kPageTokens;
+    int n = 0;
+    bool gave_up = false;
+    for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+        const int stage = n % kRebuildStages;
+        {
+            const uint32_t bar = rb_smem_u32(bars + stage), parity = (n / kRebuildStages) & 1;
+            uint32_t it = 0;
+            bool here = rb_try_wait(bar, parity);
+            while (!here && ++it < kRebuildSpin) here = rb_try_wait(bar, parity);
+            gave_up = __syncthreads_or(!here);
+        }
+        if (gave_up) break;
+        const int h = (int)(item % Hkv);
+        const int64_t lp = item / Hkv;
+        const int pg = (int)(lp % a.n_pages), l = (int)(lp / a.n_pages);
+        const bool ok = ok_stage[stage] != 0;
+        const uint8_t *rec = ring[stage];
+        const int64_t page_tok0 = (first_page + pg) * kPageTokens;            // request token of the page's first slot
+        if (a.out_k) {
+            // K: lane = 8-channel group + 16 * (token & 1), warp = token >> 1: a warp's store covers two whole rows
+            const int tok = 2 * (tid >> 5) + ((tid >> 4) & 1), c0 = (tid & 15) * 8;
+            const int64_t gt = page_tok0 + tok;
+            if (gt >= a.token_begin && gt < a.token_begin + a.n_tokens) {
+                uint2 lo = make_uint2(0u, 0u), hi = lo;
+                if (ok) {
+                    const uint32_t E = rec[bfp8_k_exp_off(tok, c0 >> 4)];
+                    const uint8_t *p = rec + bfp8_k_el_off(tok, c0);
+                    lo = dequant4(*reinterpret_cast<const uint32_t *>(p), E);
+                    hi = dequant4(*reinterpret_cast<const uint32_t *>(p + 16), E);
+                }
+                uint16_t *row = a.out_k + (int64_t)l * a.layer_stride + ((gt - a.token_begin) * Hkv + h) * kHeadDim;
+                if (relayout) {
+                    // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout)
+                    __stcs(reinterpret_cast<uint2 *>(row + (c0 >> 1)), make_uint2((lo.x & 0xFFFFu) | (lo.y << 16), (hi.x & 0xFFFFu) | (hi.y << 16)));
+                    __stcs(reinterpret_cast<uint2 *>(row + 64 + (c0 >> 1)), make_uint2((lo.x >> 16) | (lo.y & 0xFFFF0000u), (hi.x >> 16) | (hi.y & 0xFFFF0000u)));
+                } else {
+                    __stcs(reinterpret_cast<uint4 *>(row + c0), make_uint4(lo.x, lo.y, hi.x, hi.y));      // streaming: written once, read by somebody else
+                }
+            }
+        }
+        if (a.out_v) {
+            // V: a thread takes channels ch0 .. ch0+3 of tokens 2tq + 8*th and 2tq + 8*th + 1.  Lanes differ in tq and in
+            // which quad of a 32-channel span they hold (two-way bank conflicts at most; every store covers whole
+            // 64-byte pieces of output rows); warps differ in the span and in th.
+            const int lane = tid & 31, tq = lane & 3, th = tid >> 7;
+            const int j = 2 * ((tid >> 5) & 3) + ((lane >> 2) & 1), cb0 = 8 * ((lane >> 3) & 1) + 4 * (lane >> 4), ch0 = 16 * j + cb0;
+            const uint8_t *vb = rec + kBfp8Half;
+            uint32_t w[4] = {0u, 0u, 0u, 0u}, e2 = 0u;
+            if (ok) {
+                const uint8_t *p = vb + 128 + (j >> 1) * 512 + ((cb0 & 7) * 4 + tq) * 16 + ((j & 1) * 2 + (cb0 >> 3)) * 4;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) w[i] = *reinterpret_cast<const uint32_t *>(p + 64 * i);       // channel ch0 + i, four tokens
+                e2 = *reinterpret_cast<const uint32_t *>(vb + tq * 32 + j * 4);                           // exponents of the four tokens, block j
+            }
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int k = 2 * th + t, tok = 2 * tq + t + 8 * th;
+                const int64_t gt = page_tok0 + tok;
+                if (gt < a.token_begin || gt >= a.token_begin + a.n_tokens) continue;
+                // byte k of the four words = channels ch0 .. ch0+3 of this token
+                const uint32_t sel = (uint32_t)k | ((uint32_t)(4 + k) << 4);
+                const uint32_t word = __byte_perm(__byte_perm(w[0], w[1], sel), __byte_perm(w[2], w[3], sel), 0x5410u);
+                const uint2 r = ok ? dequant4(word, (e2 >> (8 * k)) & 0xFFu) : make_uint2(0u, 0u);
+                uint16_t *row = a.out_v + (int64_t)l * a.layer_stride + ((gt - a.token_begin) * Hkv + h) * kHeadDim;
+                __stcs(reinterpret_cast<uint2 *>(row + ch0), r);
+            }
+        }
+        __syncthreads();                               // everybody is done with the slot
+        if (tid == 0) {
+            const int64_t next = item + (int64_t)kRebuildStages * gridDim.x;
+            if (next < n_items) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                load(next, stage);
+            }
+        }
+    }
+    if (tid == 0 && gave_up) {
+        atomicOr(cv.flags, HMA_FLAG_WAIT_TIMEOUT);
+        for (int s = 0; s < kRebuildStages; ++s)
+            for (uint32_t it = 0; it < (1u << 16) && !rb_try_wait(rb_smem_u32(bars + s), 0) && !rb_try_wait(rb_smem_u32(bars + s), 1); ++it) {}
+    }
+}
+
 // The elementwise strawman of section 3.3: one thread per output element, byte
 // loads straight from the cache, integer bit assembly, two-byte stores.  Kept only as the comparison point.
 __global__ void __launch_bounds__(256) dequant_naive_kernel(CacheView cv, int which, const int32_t *__restrict__ page_ids,
@@ -162,6 +320,23 @@ __global__ void __launch_bounds__(256) dequant_naive_kernel(CacheView cv, int wh
 }
 
 }  // namespace hma
+
+static hma_status_t launch_rebuild(const hma::CacheView &cv, const hma::RebuildArgs &a, void *stream)
+{
+    int dev = 0, n_sm = 0;
+    HMA_CUDA_OK(cudaGetDevice(&dev));
+    HMA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    const int64_t items = (int64_t)a.n_layers * a.n_pages * cv.num_kv_heads;
+    // one wave of CTAs: as many as are resident at once, each walking its share of the records
+    int per_sm = 0;
+    HMA_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, hma::rebuild_stream_kernel, hma::kRebuildThreads, 0));
+    if (per_sm < 1) per_sm = 1;
+    const int64_t cap = (int64_t)n_sm * per_sm;
+    hma::rebuild_stream_kernel<<<(unsigned)(items < cap ? items : cap), hma::kRebuildThreads, 0, (cudaStream_t)stream>>>(cv, a);
+    hma::count_launch();
+    HMA_CUDA_OK(cudaGetLastError());
+    return HMA_OK;
+}
 
 extern "C" hma_status_t hma_bfp8_dequant_blocks_bf16(const uint8_t *exps, const uint8_t *mants, int64_t n_blocks,
                                                      void *out_bf16, void *stream)
@@ -194,6 +369,11 @@ extern "C" hma_status_t hma_bfp8_dequant_bf16(const hma_cache_t *cache, int32_t 
     if (n_pages > 0x7FFFFFFF) return HMA_ERR_INVALID_ARG;
     hma::CacheView cv{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
                       cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
+    if (cache->desc.format == HMA_KV_BFP8) {
+        hma::RebuildArgs a{nullptr, page_ids, token_begin, n_tokens, which == 0 ? (uint16_t *)out_bf16 : nullptr,
+                           which == 1 ? (uint16_t *)out_bf16 : nullptr, 0, 1, (int32_t)n_pages};
+        return launch_rebuild(cv, a, stream);
+    }
     dim3 grid((unsigned)n_pages, (unsigned)cache->desc.num_kv_heads);
     hma::dequant_paged_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, which, page_ids, token_begin, n_tokens,
                                                                       (uint16_t *)out_bf16, nullptr);
@@ -216,6 +396,12 @@ extern "C" hma_status_t hma_bfp8_rebuild_request(const hma_cache_t *cache, const
     if (n_pages > 0x7FFFFFFF || cache->desc.num_layers > 32767) return HMA_ERR_INVALID_ARG;
     hma::CacheView cv{(uint8_t *)cache->layers[0], cache->desc.num_pages, cache->desc.num_kv_heads,
                       cache->desc.num_q_heads, cache->desc.format, cache->flags, cache->desc.key_layout};
+    if (cache->desc.format == HMA_KV_BFP8) {
+        const int64_t tensor = n_tokens * cache->desc.num_kv_heads * hma::kHeadDim;      // elements of one tensor of one layer
+        hma::RebuildArgs a{cache->d_layers, page_ids, token_begin, n_tokens, (uint16_t *)out_bf16, (uint16_t *)out_bf16 + tensor,
+                           2 * tensor, cache->desc.num_layers, (int32_t)n_pages};
+        return launch_rebuild(cv, a, stream);
+    }
     dim3 grid((unsigned)n_pages, (unsigned)cache->desc.num_kv_heads, (unsigned)(2 * cache->desc.num_layers));
     hma::dequant_paged_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, 0, page_ids, token_begin, n_tokens,
                                                                       (uint16_t *)out_bf16, cache->d_layers);

@@ -2,6 +2,8 @@
 // (sections 3.2 / 3.3: host-to-device copy done by the caller or by mapped reads here, then the
 // tiled -> paged re-layout that merges per-chip shards).  Byte values are never changed on a BFP8
 // cache; on a BF16 cache each element is decoded while it is scattered.
+#include <mutex>
+
 #include "hma_common.cuh"
 
 namespace hma {
@@ -12,7 +14,8 @@ struct IngestArgs {
     int32_t head_begin[kMaxShards], head_count[kMaxShards];
     int32_t n_shards;
     const int32_t *page_ids;
-    int64_t token_begin, n_tokens;
+    int64_t token_begin, n_tokens;      // range of the request's tokens that this launch writes
+    int64_t wire_begin, wire_tokens;    // request token that is wire token 0, and the number of tokens the wire was laid out for
     int32_t layout;
 };
 
@@ -54,13 +57,13 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
     if (lp * kPageTokens < a.token_begin) lo = (int)(a.token_begin - lp * kPageTokens);
     if ((lp + 1) * kPageTokens > a.token_begin + a.n_tokens) hi = (int)(a.token_begin + a.n_tokens - lp * kPageTokens);
     const bool row16 = a.layout == HMA_WIRE_TILE32;   // tile faces are 16-byte aligned; 136-byte rows only 8
-    const bool exp_fast = lo == 0 && hi == kPageTokens && (a.token_begin & 15) == 0;
+    const bool exp_fast = lo == 0 && hi == kPageTokens && (a.wire_begin & 15) == 0;
     for (int item = threadIdx.x; item < 2 * kPageTokens * kBlocksPerRow; item += blockDim.x) {
         const int t = item >> 7 & 1, tok = (item >> 3) & 15, j = item & 7;
         if (tok < lo || tok >= hi) continue;
         const uint8_t *w = t ? a.v_wire[shard] : a.k_wire[shard];
         int64_t eo;
-        const int64_t mo = wire_block_off(a.layout, a.n_tokens, hs, lp * kPageTokens + tok - a.token_begin, j, &eo);
+        const int64_t mo = wire_block_off(a.layout, a.wire_tokens, hs, lp * kPageTokens + tok - a.wire_begin, j, &eo);
         uint8_t *dst = &rows[t][tok][8 + 8 + j * kBlock];                    // elements start at byte 16 of the padded row
         if (row16) {
             *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(w + mo);
@@ -72,12 +75,12 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
     }
     if (exp_fast) {
         // whole page, page-aligned in the wire: the exponents come in 16-byte (tile face) or 8-byte (row) pieces
-        const int64_t wt0 = lp * kPageTokens - a.token_begin;
+        const int64_t wt0 = lp * kPageTokens - a.wire_begin;
         if (row16 && threadIdx.x < 16) {
             const int t = threadIdx.x >> 3, j = threadIdx.x & 7;
             const uint8_t *w = t ? a.v_wire[shard] : a.k_wire[shard];
             int64_t eo;
-            (void)wire_block_off(a.layout, a.n_tokens, hs, wt0, j, &eo);
+            (void)wire_block_off(a.layout, a.wire_tokens, hs, wt0, j, &eo);
             const uint4 e = *reinterpret_cast<const uint4 *>(w + eo);
             const uint32_t ew[4] = {e.x, e.y, e.z, e.w};
 #pragma unroll
@@ -86,7 +89,7 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
             const int t = threadIdx.x >> 4, tok = threadIdx.x & 15;
             const uint8_t *w = t ? a.v_wire[shard] : a.k_wire[shard];
             *reinterpret_cast<uint2 *>(&rows[t][tok][0]) =
-                *reinterpret_cast<const uint2 *>(w + ((int64_t)hs * a.n_tokens + wt0 + tok) * kRowBytes);
+                *reinterpret_cast<const uint2 *>(w + ((int64_t)hs * a.wire_tokens + wt0 + tok) * kRowBytes);
         }
     }
     __syncthreads();
@@ -164,6 +167,181 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
     }
 }
 
+// ---------------------------------------------------------------- the streaming path: 32x32 tiles -> BFP8 records
+// Whole pages of a tiled wire going into a BFP8 cache (the case of sections 3.2 / 3.3: every layer of an arriving
+// request) take this kernel.  A work item is one tile row of one head: 32 tokens = two pages.  Its K bytes and its V
+// bytes are each one contiguous 4352-byte piece of the wire (four 1088-byte tiles), fetched by one bulk async copy each
+// into a four-deep ring; the CTA's 256 threads permute them into the two page records in shared memory (16-byte loads
+// and stores for K, 4x4 byte transposes in registers for V), and each finished 4352-byte record leaves by one bulk
+// async store.  A few hundred long-lived CTAs walk all items, so that a layer costs the GPU a few microseconds
+// instead of thousands of small CTAs each waiting for a free SM beside the persistent attention kernel.
+constexpr int kIngestStages = 4;            // tile rows in flight per CTA
+constexpr int kIngestOut = 3;               // record pairs being written back
+constexpr int kIngestThreads = 256;
+constexpr int kTileRowBytes = 4 * kTileBytes;      // 4352: one tensor of one (head, 32 tokens)
+constexpr uint32_t kIngestSpin = 1u << 22;
+
+__device__ __forceinline__ uint32_t ing_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool ing_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 1000;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+__global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView cv, IngestArgs a, int tile_rows, int full_pages)
+{
+    extern __shared__ __align__(128) uint8_t ing_smem[];
+    uint8_t *in = ing_smem;                                              // [stages][2 tensors][4352]
+    uint8_t *out = in + kIngestStages * 2 * kTileRowBytes;              // [kIngestOut][2 pages][4352]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(out + kIngestOut * 2 * kBfp8Record);
+    const int tid = threadIdx.x;
+    int heads = 0;
+    for (int s = 0; s < a.n_shards; ++s) heads += a.head_count[s];
+    const int n_items = heads * tile_rows;
+    if (tid == 0) {
+        for (int s = 0; s < kIngestStages; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(ing_smem_u32(bars + s)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    // launched with programmatic stream serialisation: nothing a predecessor may have written is read before this
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // item -> (shard, head inside the shard, tile row)
+    auto locate = [&](int item, int *shard, int *hs, int *tr) {
+        int hi = item / tile_rows;
+        *tr = item - hi * tile_rows;
+        int sh = 0;
+        while (sh + 1 < a.n_shards && hi >= a.head_count[sh]) hi -= a.head_count[sh++];
+        *shard = sh;
+        *hs = hi;
+    };
+    auto load = [&](int item, int stage) {      // thread 0 only
+        int shard, hs, tr;
+        locate(item, &shard, &hs, &tr);
+        const int64_t off = ((int64_t)hs * tile_rows + tr) * kTileRowBytes;
+        const uint32_t bar = ing_smem_u32(bars + stage), dst = ing_smem_u32(in + stage * 2 * kTileRowBytes);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * kTileRowBytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                     "l"(a.k_wire[shard] + off), "r"(kTileRowBytes), "r"(bar)
+                     : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst + kTileRowBytes),
+                     "l"(a.v_wire[shard] + off), "r"(kTileRowBytes), "r"(bar)
+                     : "memory");
+    };
+    if (tid == 0)
+        for (int s = 0; s < kIngestStages; ++s) {
+            const int item = blockIdx.x + s * gridDim.x;
+            if (item < n_items) load(item, s);
+        }
+    const int p = tid >> 7, x = tid & 127;      // this thread's page of the item and its slot inside the page
+    int n = 0;
+    bool gave_up = false;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+        const int stage = n % kIngestStages;
+        const uint32_t parity = (n / kIngestStages) & 1;
+        {   // bounded wait for the tile row; the CTA decides together whether it arrived
+            const uint32_t bar = ing_smem_u32(bars + stage);
+            uint32_t it = 0;
+            bool here = ing_try_wait(bar, parity);
+            while (!here && ++it < kIngestSpin) here = ing_try_wait(bar, parity);
+            gave_up = __syncthreads_or(!here);
+        }
+        if (gave_up) break;
+        int shard, hs, tr;
+        locate(item, &shard, &hs, &tr);
+        const int h = a.head_begin[shard] + hs;
+        const int lp = 2 * tr + p;                                       // logical page of the request (from token_begin)
+        const bool page_ok = lp < full_pages;
+        const uint8_t *src = in + stage * 2 * kTileRowBytes;
+        uint8_t *rec = out + ((n % kIngestOut) * 2 + p) * kBfp8Record;
+        if (page_ok) {
+            const uint8_t *kt = src, *vt = src + kTileRowBytes;
+            // K elements: destination 16-byte piece x = blocks 4*(c>>1) .. +3 of token tok, channels 4q .. 4q+3
+            {
+                const int c = x >> 5, lane = x & 31, tok = (lane >> 2) + 8 * (c & 1), q = lane & 3;
+                uint32_t w[4];
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = 4 * (c >> 1) + jj;
+                    w[jj] = *reinterpret_cast<const uint32_t *>(kt + (j >> 1) * kTileBytes + 64 + (2 * p + (j & 1)) * 256 + tok * 16 + q * 4);
+                }
+                *reinterpret_cast<uint4 *>(rec + 128 + c * 512 + lane * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            // V elements: four tokens x four channels, transposed in registers.  The lanes of a warp differ in the token
+            // quad, the parity of the block and the channel quad, which keeps loads and stores to two-way bank conflicts.
+            {
+                const int lane = x & 31, tq = lane & 3, j = 2 * (x >> 5) + ((lane >> 2) & 1), cb0 = 4 * (2 * ((lane >> 3) & 1) + (lane >> 4));
+                const uint8_t *base = vt + (j >> 1) * kTileBytes + 64 + (2 * p + (j & 1)) * 256 + cb0;
+                const uint32_t w0 = *reinterpret_cast<const uint32_t *>(base + (2 * tq) * 16);
+                const uint32_t w1 = *reinterpret_cast<const uint32_t *>(base + (2 * tq + 1) * 16);
+                const uint32_t w2 = *reinterpret_cast<const uint32_t *>(base + (2 * tq + 8) * 16);
+                const uint32_t w3 = *reinterpret_cast<const uint32_t *>(base + (2 * tq + 9) * 16);
+                const uint32_t a01 = __byte_perm(w0, w1, 0x5140), b01 = __byte_perm(w0, w1, 0x7362);
+                const uint32_t a23 = __byte_perm(w2, w3, 0x5140), b23 = __byte_perm(w2, w3, 0x7362);
+                uint32_t *rv = reinterpret_cast<uint32_t *>(rec + kBfp8Half) + 32 + (j >> 1) * 128 + ((cb0 & 7) * 4 + tq) * 4 + (j & 1) * 2 + (cb0 >> 3);
+                rv[0] = __byte_perm(a01, a23, 0x5410);
+                rv[16] = __byte_perm(a01, a23, 0x7632);
+                rv[32] = __byte_perm(b01, b23, 0x5410);
+                rv[48] = __byte_perm(b01, b23, 0x7632);
+            }
+            // exponents: 32 words of K, 32 of V per page
+            if (x < 32) {
+                const int tok = (x >> 2) + 8 * ((x >> 1) & 1);
+                uint32_t val = 0;
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = 4 * (x & 1) + jj;
+                    val |= (uint32_t)kt[(j >> 1) * kTileBytes + (2 * p + (j & 1)) * 16 + tok] << (8 * jj);
+                }
+                reinterpret_cast<uint32_t *>(rec)[x] = val;
+            } else if (x < 64) {
+                const int w = x - 32, tq = w >> 3, j = w & 7;
+                const uint8_t *e = vt + (j >> 1) * kTileBytes + (2 * p + (j & 1)) * 16;
+                reinterpret_cast<uint32_t *>(rec + kBfp8Half)[w] =
+                    e[2 * tq] | (e[2 * tq + 1] << 8) | (e[2 * tq + 8] << 16) | ((uint32_t)e[2 * tq + 9] << 24);
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // this thread's record bytes, before the bulk store reads them
+        __syncthreads();
+        if (tid == 0) {
+            for (int pp = 0; pp < 2; ++pp) {
+                const int lpp = 2 * tr + pp;
+                if (lpp >= full_pages) continue;
+                const int32_t pid = a.page_ids[lpp];
+                if (pid < 0 || pid >= cv.num_pages) { atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_INGEST); continue; }
+                uint8_t *dst = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)kBfp8Record;
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+                             "r"(ing_smem_u32(out + ((n % kIngestOut) * 2 + pp) * kBfp8Record)), "r"(kBfp8Record)
+                             : "memory");
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            // at most one store group still reading shared memory: the buffer two items back is free again
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            const int next = item + kIngestStages * gridDim.x;
+            if (next < n_items) load(next, stage);
+        }
+    }
+    if (tid == 0) {
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");         // every record has landed before the CTA leaves
+        if (gave_up) {
+            // a wait ran out: flag it, and give the copies still in flight a bounded chance to land before the CTA's
+            // shared memory is handed to somebody else
+            atomicOr(cv.flags, HMA_FLAG_WAIT_TIMEOUT);
+            for (int s = 0; s < kIngestStages; ++s)
+                for (uint32_t it = 0; it < (1u << 16) && !ing_try_wait(ing_smem_u32(bars + s), 0) && !ing_try_wait(ing_smem_u32(bars + s), 1); ++it) {}
+        }
+    }
+}
+
 // Plain BF16 rows ([head][token][128], KV made on the decode GPU) into a BF16 cache: one CTA per (page, head).
 // K: two consecutive channels of a token are one word of the record; V: single elements (tokens pair up in a word).
 __global__ void __launch_bounds__(128) ingest_bf16_rows_kernel(CacheView cv, IngestArgs a)
@@ -185,7 +363,7 @@ __global__ void __launch_bounds__(128) ingest_bf16_rows_kernel(CacheView cv, Ing
     for (int i = threadIdx.x; i < kPageTokens * 64; i += blockDim.x) {
         const int tok = i >> 6, ch = (i & 63) * 2;
         if (tok < lo || tok >= hi) continue;
-        const int64_t row = ((int64_t)hs * a.n_tokens + (lp * kPageTokens + tok - a.token_begin)) * kHeadDim;
+        const int64_t row = ((int64_t)hs * a.wire_tokens + (lp * kPageTokens + tok - a.wire_begin)) * kHeadDim;
         *reinterpret_cast<uint32_t *>(rec + bf16_k_el_off(tok, ch)) = *reinterpret_cast<const uint32_t *>(kw + row + ch);
         const uint32_t v2 = *reinterpret_cast<const uint32_t *>(vw + row + ch);
         *reinterpret_cast<uint16_t *>(rec + bf16_v_el_off(tok, ch)) = (uint16_t)v2;
@@ -234,10 +412,63 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
     a.page_ids = page_ids;
     a.token_begin = token_begin;
     a.n_tokens = n_tokens;
+    a.wire_begin = token_begin;
+    a.wire_tokens = n_tokens;
     a.layout = wire_layout;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (wire_layout == HMA_WIRE_TILE32 && cache->desc.format == HMA_KV_BFP8 && (token_begin & 15) == 0 && n_tokens >= hma::kPageTokens &&
+        n_tokens / hma::kPageTokens <= 0x3FFFFFFF) {
+        // whole pages of a tiled wire: the streaming kernel; a ragged last page (if any) follows through the general kernel
+        static std::mutex setup_lock;
+        static int sm_count[64] = {};
+        int dev = 0;
+        HMA_CUDA_OK(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64) return HMA_ERR_UNSUPPORTED_SHAPE;
+        const size_t smem = (size_t)(hma::kIngestStages * 2 * hma::kTileRowBytes + hma::kIngestOut * 2 * hma::kBfp8Record + hma::kIngestStages * 8);
+        {
+            std::lock_guard<std::mutex> guard(setup_lock);
+            if (!sm_count[dev]) {
+                int n = 0;
+                HMA_CUDA_OK(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+                HMA_CUDA_OK(cudaFuncSetAttribute(hma::ingest_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                sm_count[dev] = n;
+            }
+        }
+        const int full_pages = (int)(n_tokens / hma::kPageTokens);
+        const int tile_rows = (int)((n_tokens + 31) / 32);
+        const int64_t items = (int64_t)heads * ((full_pages + 1) / 2);
+        // items are numbered over all tile rows of the wire; a last tile row without a whole page holds no item to do,
+        // but keeping the wire's own row count in the numbering keeps the addressing plain
+        (void)items;
+        const int64_t n_items = (int64_t)heads * tile_rows;
+        const int64_t max_ctas = (int64_t)sm_count[dev] * 3;
+        const unsigned grid_x = (unsigned)(n_items < max_ctas ? n_items : max_ctas);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid_x);
+        cfg.blockDim = dim3(hma::kIngestThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::ingest_tiles_kernel, cv, a, tile_rows, full_pages));
+        hma::count_launch();
+        const int64_t rest = n_tokens - (int64_t)full_pages * hma::kPageTokens;
+        if (rest == 0) return HMA_OK;
+        a.token_begin = token_begin + (int64_t)full_pages * hma::kPageTokens;
+        a.n_tokens = rest;
+        a.page_ids = page_ids + full_pages;
+        dim3 tail_grid(1u, (unsigned)heads);
+        hma::ingest_kernel<<<tail_grid, 128, 0, st>>>(cv, a);
+        hma::count_launch();
+        HMA_CUDA_OK(cudaGetLastError());
+        return HMA_OK;
+    }
     dim3 grid((unsigned)n_pages, (unsigned)heads);
-    if (wire_layout == HMA_WIRE_BF16_ROWS) hma::ingest_bf16_rows_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, a);
-    else hma::ingest_kernel<<<grid, 128, 0, (cudaStream_t)stream>>>(cv, a);
+    if (wire_layout == HMA_WIRE_BF16_ROWS) hma::ingest_bf16_rows_kernel<<<grid, 128, 0, st>>>(cv, a);
+    else hma::ingest_kernel<<<grid, 128, 0, st>>>(cv, a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;
