@@ -312,6 +312,61 @@ void orc_decode_attention_mixed(const uint16_t *q_bf16, const uint8_t *k_wire, c
         }
 }
 
+/* Decode attention with several query tokens per sequence (speculative or chunked decode; the paper's decode loop,
+ * section 1, generates one token per step, this is the widening named in its place).  The cache of sequence b holds
+ * T = ctx_lens[b] tokens, the last q_len of which are the new tokens themselves; query i (0 .. q_len-1) is the i-th
+ * new token and attends causally: to tokens t < T - (q_len - 1 - i).  A query that sees no token gives zeros.
+ *   q_bf16   [B][q_len][Hq][128]
+ *   out      [B][q_len][Hq][128]
+ * Everything else as orc_decode_attention (keys in the queries' head-dim order). */
+void orc_decode_attention_multi(const uint16_t *q_bf16, const uint8_t *k_wire, const uint8_t *v_wire,
+                                const int64_t *wire_off, const int32_t *ctx_lens,
+                                int32_t B, int32_t q_len, int32_t Hq, int32_t Hkv, double sm_scale,
+                                double *out_f64, uint16_t *out_bf16)
+{
+    const int G = Hq / Hkv;
+#pragma omp parallel for collapse(3) schedule(dynamic, 1)
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t i = 0; i < q_len; ++i)
+            for (int32_t h = 0; h < Hq; ++h) {
+                const int64_t T = ctx_lens[b];
+                const int64_t visible = T - (q_len - 1 - i);       /* causal: the later new tokens are masked */
+                const int32_t g = h / G;
+                const int64_t row = ((int64_t)b * q_len + i) * Hq + h;
+                double q[ORC_HEAD_DIM], o[ORC_HEAD_DIM];
+                for (int d = 0; d < ORC_HEAD_DIM; ++d) {
+                    q[d] = orc_bf16_to_f64(q_bf16[row * ORC_HEAD_DIM + d]);
+                    o[d] = 0.0;
+                }
+                if (visible > 0) {
+                    const uint8_t *kr = k_wire + wire_off[b] + (int64_t)g * T * ORC_ROW_BYTES;
+                    const uint8_t *vr = v_wire + wire_off[b] + (int64_t)g * T * ORC_ROW_BYTES;
+                    double *s = (double *)malloc((size_t)T * sizeof(double));
+                    double smax = -INFINITY;
+                    for (int64_t t = 0; t < T; ++t) {
+                        if (t >= visible) { s[t] = -INFINITY; continue; }
+                        const uint8_t *kv = kr + t * ORC_ROW_BYTES;
+                        double acc = 0.0;
+                        for (int d = 0; d < ORC_HEAD_DIM; ++d) acc += q[d] * bfp8_value(kv[d / ORC_BLOCK], kv[ORC_BLOCKS_PER_ROW + d]);
+                        s[t] = sm_scale * acc;
+                        if (s[t] > smax) smax = s[t];
+                    }
+                    double denom = 0.0;
+                    for (int64_t t = 0; t < T; ++t) { s[t] = exp(s[t] - smax); denom += s[t]; }      /* exp(-inf) = 0 for masked tokens */
+                    for (int64_t t = 0; t < T; ++t) {
+                        const uint8_t *vv = vr + t * ORC_ROW_BYTES;
+                        double p = s[t] / denom;
+                        for (int d = 0; d < ORC_HEAD_DIM; ++d) o[d] += p * bfp8_value(vv[d / ORC_BLOCK], vv[ORC_BLOCKS_PER_ROW + d]);
+                    }
+                    free(s);
+                }
+                for (int d = 0; d < ORC_HEAD_DIM; ++d) {
+                    if (out_f64) out_f64[row * ORC_HEAD_DIM + d] = o[d];
+                    if (out_bf16) out_bf16[row * ORC_HEAD_DIM + d] = orc_f64_to_bf16(o[d]);
+                }
+            }
+}
+
 int orc_num_threads(void)
 {
     int n = 1;

@@ -201,6 +201,29 @@ def decode_attention_mixed(q_bf16, k_wires, v_wires, k_tails, v_tails, num_kv_he
     return out64, out16
 
 
+def decode_attention_multi(q_bf16, k_wires, v_wires, num_kv_heads, sm_scale=None):
+    """fp64 decode attention with q_len query tokens per sequence (the last q_len cached tokens are the new tokens;
+    query i sees tokens t < T - (q_len - 1 - i)).
+
+    q_bf16 : uint16 [B][q_len][Hq][128]; k_wires, v_wires as in decode_attention.
+    returns (out_f64 [B][q_len][Hq][128], out_bf16)."""
+    q_bf16 = np.ascontiguousarray(q_bf16, np.uint16)
+    B, q_len, Hq, D = q_bf16.shape
+    assert D == HEAD_DIM and Hq % num_kv_heads == 0 and len(k_wires) == B == len(v_wires)
+    if sm_scale is None:
+        sm_scale = 1.0 / np.sqrt(HEAD_DIM)
+    lens = np.array([w.shape[1] for w in k_wires], np.int32)
+    offs = np.zeros(B, np.int64)
+    offs[1:] = np.cumsum([num_kv_heads * int(t) * ROW_BYTES for t in lens])[:-1]
+    kcat = np.concatenate([np.ascontiguousarray(w, np.uint8).reshape(-1) for w in k_wires] + [np.zeros(1, np.uint8)])
+    vcat = np.concatenate([np.ascontiguousarray(w, np.uint8).reshape(-1) for w in v_wires] + [np.zeros(1, np.uint8)])
+    out64 = np.empty((B, q_len, Hq, D), np.float64)
+    out16 = np.empty((B, q_len, Hq, D), np.uint16)
+    lib().orc_decode_attention_multi(_p(q_bf16), _p(kcat), _p(vcat), _p(offs), _p(lens), ctypes.c_int32(B), ctypes.c_int32(q_len),
+                                     ctypes.c_int32(Hq), ctypes.c_int32(num_kv_heads), ctypes.c_double(sm_scale), _p(out64), _p(out16))
+    return out64, out16
+
+
 def half_split_index(c):
     """Half-split position of interleaved-order channel c (the key re-layout of section 3.3)."""
     lib().orc_half_split_index.restype = ctypes.c_int32
