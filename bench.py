@@ -292,6 +292,41 @@ class Workload:
         torch.cuda.synchronize(self.device)
         return e0.elapsed_time(e1) / 1e3 / reps / self.L
 
+    def time_pcie(self, reps=3):
+        """Host-to-device copy rate of this machine: the arriving request's pinned wire bytes (or 1 GiB of pinned memory)
+        copied to a device buffer by the copy engine, best of `reps`; GB/s."""
+        src = self.wire_host.view(-1) if self.ingest_tokens else torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+        dst = torch.empty(src.numel(), dtype=torch.uint8, device=self.device)
+        best = 1e30
+        for _ in range(reps + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            dst.copy_(src, non_blocking=True)
+            e1.record()
+            torch.cuda.synchronize(self.device)
+            best = min(best, e0.elapsed_time(e1) / 1e3)
+        return src.numel() / best / 1e9
+
+    def time_multi_query(self, q_len, reps=3):
+        """hma_decode_attention_multi with q_len query tokens per sequence (the last q_len cached tokens): mean seconds per call."""
+        hma = self.hma
+        q = synth.make_q(self.B * q_len, self.hq, 4321, self.device).view(self.B, q_len, self.hq, 128)
+        out = torch.empty_like(q)
+        ws = hma.new_workspace(self.caches["bfp8"].desc, self.B * q_len, self.device)
+
+        def run():
+            for l in range(self.L):
+                hma.hma_decode_attention_multi(self.caches["bfp8"], l, q, out, self.table, self.ctx, self.sm_scale, ws)
+        run()
+        torch.cuda.synchronize(self.device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record()
+        torch.cuda.synchronize(self.device)
+        return e0.elapsed_time(e1) / 1e3 / reps / self.L
+
     def time_rebuild(self, reps=3):
         """One-shot BFP8 -> BF16 rebuild of one whole request (sequence 0: every layer, K and V): seconds, bytes moved."""
         T = int(self.lens[0])
@@ -478,6 +513,15 @@ def main():
                  "tokens_per_s": aggregate_value(wl.B, sec_paced, ws), "slowdown_vs_decode_only": sec_paced / sec_decode_only - 1.0}
     sec_e2e = wl.time_steps(max(2, args.steps // 4), 3, host=True)
     sec_e2e_mapped = wl.time_steps(max(2, args.steps // 4), 3, host=True, staged=False) if wl.ingest_tokens else sec_e2e
+    pcie_gbs = wl.time_pcie()
+    e2e_paced = {}
+    if wl.ingest_tokens:
+        # end to end at the paper's operating point: the request's bytes arrive from the host at the link's rate
+        sec_e2e_paced = wl.time_steps(max(2, args.steps // 4), 3, host=True, ingest_layers=paced["layers_per_step"])
+        e2e_paced = {"layers_per_step": paced["layers_per_step"], "ms_per_step": sec_e2e_paced * 1e3,
+                     "tokens_per_s": aggregate_value(wl.B, sec_e2e_paced, ws),
+                     "h2d_bytes_per_step": wl.L * wl.B * wl.hq * 128 * 2 + paced["layers_per_step"] * 2 * 4 * wl.shard_bytes,
+                     "slowdown_vs_decode_only": sec_e2e_paced / sec_decode_only - 1.0}
     extra = {}
     if "bf16" in wl.caches:
         k = max(5, args.steps // 4)
@@ -501,6 +545,13 @@ def main():
     extra["mixed_prefix_tail"] = {"us_per_call": t_mixed * 1e6, "tail_tokens_per_sequence": 64,
                                   "what": "hma_decode_attention_mixed: BFP8 prefix cache + BF16 cache with 64 decode-side tokens per sequence",
                                   "overhead_vs_prefix_only": t_mixed / call_mean - 1.0}
+    mq = {"what": "hma_decode_attention_multi: q_len query tokens per sequence over the same cache (speculative / chunked decode); "
+                  "tokens/s counts query tokens, attention only, all layers"}
+    base_call = wl.time_multi_query(1)
+    for q_len in (1, 2, 4):
+        t = base_call if q_len == 1 else wl.time_multi_query(q_len)
+        mq["q_len_%d" % q_len] = {"us_per_call": t * 1e6, "tokens_per_s": wl.B * q_len / (t * wl.L), "per_token_speedup": q_len * base_call / t}
+    extra["multi_query"] = mq
     kv_step = wl.kv_bytes_per_layer("bfp8") * wl.L
     value = aggregate_value(wl.B, sec, ws)
     achieved = wl.kv_bytes_per_layer("bfp8") / call_mean / 1e9
@@ -520,7 +571,11 @@ def main():
         "e2e": {"value": aggregate_value(wl.B, sec_e2e, ws), "unit": "tokens/s", "ms_per_step": sec_e2e * 1e3,
                 "h2d_bytes_per_step": q_bytes + wire_bytes, "d2h_bytes_per_step": q_bytes,
                 "ingest_source": "pinned host -> device staging (copy engine) -> hma_kv_ingest_layer",
-                "ms_per_step_mapped_reads": sec_e2e_mapped * 1e3},
+                "ms_per_step_mapped_reads": sec_e2e_mapped * 1e3,
+                "pcie_h2d_gbs_measured": pcie_gbs,
+                "h2d_gbs": (q_bytes + wire_bytes) / sec_e2e / 1e9,
+                "frac_of_pcie": (q_bytes + wire_bytes) / sec_e2e / 1e9 / pcie_gbs,
+                "at_link_rate": e2e_paced},
         "gpu_launches": int(launches * args.steps),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": "of " + peak_kind, "frac_of_8000": achieved / 8000.0,
@@ -550,6 +605,18 @@ def main():
                                 "kv_gbs": toks * wl.hkv * BFP8_ROW / t / 1e9, "seconds": t,
                                 "sample": "layer 0 of all %d sequences (%d tokens x %d q heads); tokens/s = %d / (t x %d layers)"
                                 % (n_seq, toks, wl.hq, n_seq, wl.L)}
+    if rank == 0 and ws == 1 and not args.no_cpu:
+        # the oracle's BFP8 -> BF16 decode beside the library's rebuild (elements per second)
+        from oracle import oracle as orc
+        wire = synth.make_kv_wire(wl.hkv, 8192, 99).numpy()
+        orc.decode_rowmajor_bf16(wire[:, :64])
+        t0 = time.perf_counter()
+        orc.decode_rowmajor_bf16(wire)
+        t_dec = time.perf_counter() - t0
+        rb = extra["rebuild_request"]
+        line["cpu_baseline"]["dequant"] = {"oracle_elements_per_s": wire.shape[0] * wire.shape[1] * 128 / t_dec, "oracle_threads": 1,
+                                           "oracle_sample": "one tensor of one layer of one 8192-token request (%d elements)" % (wire.shape[0] * wire.shape[1] * 128),
+                                           "gpu_elements_per_s": rb_elems / (rb["ms"] / 1e3), "gpu_call": "hma_bfp8_rebuild_request"}
     if rank == 0:
         print(json.dumps(line))
     if ws > 1:

@@ -183,6 +183,22 @@ hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,
                                   void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Decode attention with q_len query tokens per sequence (speculative or chunked decode; section 1 describes decode as
+ * one token per step, this is the widening of it).  The cache of sequence b already holds all context_lens[b] tokens,
+ * the last q_len of which are the new tokens themselves; query i (0 .. q_len-1) attends causally, to tokens
+ * t < context_lens[b] - (q_len - 1 - i).  A query that sees no token gives a row of zeros.
+ *   q, out       [batch][q_len][num_q_heads][128]
+ *   workspace    >= hma_decode_attention_workspace_bytes(desc, batch * q_len); batch * q_len <= 1024
+ * Everything else as hma_decode_attention, of which this is the q_len = 1 case.  The q_len rows of a sequence walk the
+ * same pages at the same time, so HBM is read about once and the L2 serves the rest; the arithmetic is not shared.
+ */
+hma_status_t hma_decode_attention_multi(const hma_cache_t *cache, int32_t layer,
+                                        const void *q, void *out, int32_t out_dtype,
+                                        const int32_t *block_table, int32_t max_pages_per_seq,
+                                        const int32_t *context_lens, int32_t batch, int32_t q_len, float sm_scale,
+                                        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * hma_decode_attention for callers that cannot allocate.  (The paper has no counterpart: this exists for
  * the way the library gets embedded, not for the method.)  A decode loop that fixed its memory pool at
  * start-up, or code running where the host framework forbids allocation, has no workspace to pass; here

@@ -61,7 +61,8 @@ struct AttnArgs {
     const int32_t *block_table;
     int max_pages;
     const int32_t *ctx;
-    int batch;
+    int batch;                      // rows of q and out: sequences x query tokens per sequence
+    int q_len;                      // query tokens per sequence; row r is query r % q_len of sequence r / q_len
     float sm_scale;
     int32_t *counters;              // workspace: one arrival counter per (sequence, kv head); zero between calls
     int32_t *cum;                   // workspace: pages before each sequence, then pages + segment costs before each
@@ -234,13 +235,17 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float r)
     return (uint16_t)(u >> 16);
 }
 
-// pages of sequence b (context clamped to what the block table can address)
-__device__ __forceinline__ int pages_of(const AttnArgs &a, int b)
+// Tokens that row b of the batch attends to.  With one query token per sequence that is the sequence's context (clamped
+// to what the block table can address).  With q_len query tokens the cache already holds all of them: query i sees the
+// context less the q_len - 1 - i newer tokens (causal inside the new tokens), and the q_len rows of a sequence share its
+// block table row.
+__device__ __forceinline__ int context_of(const AttnArgs &a, int b)
 {
-    int T = a.ctx[b];
-    T = max(0, min(T, a.max_pages * kPageTokens));
-    return (T + kPageTokens - 1) / kPageTokens;
+    const int s = b / a.q_len, i = b - s * a.q_len;
+    const int T = max(0, min(a.ctx[s], a.max_pages * kPageTokens));
+    return max(0, T - (a.q_len - 1 - i));
 }
+__device__ __forceinline__ int pages_of(const AttnArgs &a, int b) { return (context_of(a, b) + kPageTokens - 1) / kPageTokens; }
 
 __device__ __forceinline__ void store_out(const AttnArgs &a, int64_t idx, float v)
 {
@@ -680,7 +685,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
             const int npb = cum[lo + 1] - cum[lo];
             const int off = (int)(wr - (int64_t)Hkv * cum[lo]);
             const int gg = off / npb, pp = off - gg * npb;
-            const int32_t pid = a.block_table[(int64_t)lo * a.max_pages + pp];
+            const int32_t pid = a.block_table[(int64_t)(lo / a.q_len) * a.max_pages + pp];
             if (pid >= 0 && pid < a.cv.num_pages) roff = (uint32_t)(((int64_t)pid * Hkv + gg) * (kRecord / 128));
         }
     };
@@ -729,7 +734,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
 
     auto begin_segment = [&](int k) {
         np = cum[b + 1] - cum[b];
-        T = min(a.ctx[b], a.max_pages * kPageTokens);
+        T = context_of(a, b);
         tail = T - (np - 1) * kPageTokens;
         whole = page == 0 && Rw - k >= np;
         // Q fragments of this (sequence, kv head): FP16, one power-of-two scale per head
@@ -1263,10 +1268,13 @@ extern "C" hma_status_t hma_decode_attention_workspace_init(void *workspace, siz
 
 static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, const void *q, void *out, int32_t out_dtype,
                                      const int32_t *block_table, int32_t max_pages_per_seq, const int32_t *context_lens,
-                                     int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes, void *stream,
-                                     int probe, int always_partial = 0, hma::AttnArgs *args_out = nullptr, int *ctas_out = nullptr)
+                                     int32_t n_seqs, float sm_scale, void *workspace, size_t workspace_bytes, void *stream,
+                                     int probe, int always_partial = 0, hma::AttnArgs *args_out = nullptr, int *ctas_out = nullptr,
+                                     int32_t q_len = 1)
 {
-    if (!cache || layer < 0 || layer >= cache->desc.num_layers || batch < 0 || max_pages_per_seq < 0) return HMA_ERR_INVALID_ARG;
+    if (!cache || layer < 0 || layer >= cache->desc.num_layers || n_seqs < 0 || max_pages_per_seq < 0 || q_len < 1) return HMA_ERR_INVALID_ARG;
+    if ((int64_t)n_seqs * q_len > hma::kMaxBatch) return HMA_ERR_UNSUPPORTED_SHAPE;
+    const int32_t batch = n_seqs * q_len;         // rows of q and out
     if (out_dtype != HMA_OUT_BF16 && out_dtype != HMA_OUT_F32) return HMA_ERR_INVALID_ARG;
     if (batch == 0) return HMA_OK;
     if (!block_table || !context_lens || !workspace || (!probe && (!q || !out))) return HMA_ERR_INVALID_ARG;
@@ -1308,6 +1316,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.max_pages = max_pages_per_seq;
     a.ctx = context_lens;
     a.batch = batch;
+    a.q_len = q_len;
     a.sm_scale = sm_scale;
     const int hkv = cache->desc.num_kv_heads;
     a.counters = (int32_t *)workspace;
@@ -1354,6 +1363,15 @@ extern "C" hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t l
 {
     return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
                             workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" hma_status_t hma_decode_attention_multi(const hma_cache_t *cache, int32_t layer, const void *q, void *out,
+                                                   int32_t out_dtype, const int32_t *block_table, int32_t max_pages_per_seq,
+                                                   const int32_t *context_lens, int32_t batch, int32_t q_len, float sm_scale,
+                                                   void *workspace, size_t workspace_bytes, void *stream)
+{
+    return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
+                            workspace, workspace_bytes, stream, 0, 0, nullptr, nullptr, q_len);
 }
 
 extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,

@@ -69,6 +69,8 @@ def lib():
         L.hma_decode_attention_workspace_init.argtypes = [vp, sz, vp]
         L.hma_decode_attention.restype = i32
         L.hma_decode_attention.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp, sz, vp]
+        L.hma_decode_attention_multi.restype = i32
+        L.hma_decode_attention_multi.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, i32, f32, vp, sz, vp]
         L.hma_decode_attention_static.restype = i32
         L.hma_decode_attention_static.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
         L.hma_decode_attention_static_limit_bytes.restype = sz
@@ -209,6 +211,15 @@ def hma_decode_attention(cache, layer, q, out, block_table, context_lens, sm_sca
                                       block_table.shape[1], _ptr(context_lens), q.shape[0], float(sm_scale),
                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "hma_decode_attention")
+
+
+def hma_decode_attention_multi(cache, layer, q, out, block_table, context_lens, sm_scale, workspace, stream=None):
+    """q, out: [batch][q_len][Hq][128]; the last q_len cached tokens of each sequence are the query tokens (causal)."""
+    out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
+    _check(lib().hma_decode_attention_multi(cache.handle, layer, _ptr(q), _ptr(out), out_dtype, _ptr(block_table),
+                                            block_table.shape[1], _ptr(context_lens), q.shape[0], q.shape[1], float(sm_scale),
+                                            _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "hma_decode_attention_multi")
 
 
 def hma_decode_attention_static(cache, layer, q, out, block_table, context_lens, sm_scale, stream=None):
