@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(128) ingest_kernel(CacheView cv, IngestArgs a)
 // async store.  A few hundred long-lived CTAs walk all items, so that a layer costs the GPU a few microseconds
 // instead of thousands of small CTAs each waiting for a free SM beside the persistent attention kernel.
 constexpr int kIngestStages = 4;            // tile rows in flight per CTA
-constexpr int kIngestOut = 3;               // record pairs being written back
+constexpr int kIngestOut = 2;               // record pairs being written back
 constexpr int kIngestThreads = 256;
 constexpr int kTileRowBytes = 4 * kTileBytes;      // 4352: one tensor of one (head, 32 tokens)
 constexpr uint32_t kIngestSpin = 1u << 22;
@@ -248,6 +248,13 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
         const int stage = n % kIngestStages;
         const uint32_t parity = (n / kIngestStages) & 1;
+        // the physical pages of this item are asked for now, so that the table read is over when the records are ready to leave
+        int32_t pid2[2] = {-1, -1};
+        if (tid == 0) {
+            const int tr0 = item % tile_rows;
+            if (2 * tr0 < full_pages) pid2[0] = a.page_ids[2 * tr0];
+            if (2 * tr0 + 1 < full_pages) pid2[1] = a.page_ids[2 * tr0 + 1];
+        }
         {   // bounded wait for the tile row; the CTA decides together whether it arrived
             const uint32_t bar = ing_smem_u32(bars + stage);
             uint32_t it = 0;
@@ -311,12 +318,15 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
             }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // this thread's record bytes, before the bulk store reads them
+        // the store issued two items ago read the buffer that the next item will fill: it must be through before anybody
+        // passes the barrier below (at most the previous item's store is still pending here)
+        if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncthreads();
         if (tid == 0) {
             for (int pp = 0; pp < 2; ++pp) {
                 const int lpp = 2 * tr + pp;
                 if (lpp >= full_pages) continue;
-                const int32_t pid = a.page_ids[lpp];
+                const int32_t pid = pid2[pp];
                 if (pid < 0 || pid >= cv.num_pages) { atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_INGEST); continue; }
                 uint8_t *dst = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)kBfp8Record;
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
@@ -324,8 +334,6 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
                              : "memory");
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            // at most one store group still reading shared memory: the buffer two items back is free again
-            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
             const int next = item + kIngestStages * gridDim.x;
             if (next < n_items) load(next, stage);
         }
@@ -441,7 +449,7 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
         // but keeping the wire's own row count in the numbering keeps the addressing plain
         (void)items;
         const int64_t n_items = (int64_t)heads * tile_rows;
-        const int64_t max_ctas = (int64_t)sm_count[dev] * 3;
+        const int64_t max_ctas = (int64_t)sm_count[dev] * 4;
         const unsigned grid_x = (unsigned)(n_items < max_ctas ? n_items : max_ctas);
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
