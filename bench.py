@@ -609,7 +609,7 @@ def main():
                                   "attention_us": [inter_mean * 1e6, inter_med * 1e6, inter_min * 1e6],
                                   "kv_read_probe_us": [probe_mean * 1e6, probe_med * 1e6, probe_min * 1e6],
                                   "hbm_read_us": [hbm_mean * 1e6, hbm_med * 1e6, hbm_min * 1e6]},
-                     "kernel": "hma_decode_attention (attn_kernel<0,0> + attn_merge_kernel)",
+                     "kernel": "hma_decode_attention (attn_kernel<0,0>: attention and cross-split reduction in one launch)",
                      "bytes_per_launch": wl.kv_bytes_per_layer("bfp8"), "us_per_launch_mean": call_mean * 1e6,
                      "us_per_launch_median": call_med * 1e6, "us_per_launch_min": call_min * 1e6},
         "decode_only": {"tokens_per_s": aggregate_value(wl.B, sec_decode_only, ws), "ms_per_step": sec_decode_only * 1e3,

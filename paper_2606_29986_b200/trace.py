@@ -4,7 +4,8 @@
 
 Builds libhma_trace.so if needed, runs hma_decode_attention on a benchmark workload with that image, reads the
 time stamps every worker (warp) left behind its partial tiles, and prints a summary: when warps start, when their
-first record lands, when they leave the record loop, how that spreads inside an SM and between SMs.  The default
+first record lands, when they leave the record loop, how that spreads inside an SM and between SMs, what the CTA-level
+reduction costs, and how three consecutive calls hand over to one another.  The default
 library carries none of the instrumentation; the numbers printed here are about where time goes, not bench values.
 """
 import argparse
@@ -71,6 +72,27 @@ def main():
                          epi_merge_us=cyc(11, 10).mean(), epi_total_us_mean=cyc(11, 8).mean(), epi_total_us_max=cyc(11, 8).max(),
                          within_mean=within.mean(), within_max=within.max(), recs_min=int(recs.min()), recs_max=int(recs.max()),
                          slow=[int(x) for x in sms[np.argsort(sm_end)[-8:]]]))
+    # three consecutive calls, each with a workspace of its own so that all three traces survive: where one kernel ends
+    # and the next begins on the same clock (the hand-off under programmatic stream serialisation)
+    wss = [hma.new_workspace(wl.caches["bfp8"].desc, wl.B, dev) for _ in range(3)]
+    for i in range(24):
+        l = i % wl.L
+        hma.hma_decode_attention(wl.caches["bfp8"], l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wss[i % 3])
+    torch.cuda.synchronize()
+    chain = []
+    for ws in wss:
+        tr = ws[trace_off:ws_bytes].view(torch.int64).cpu().numpy().reshape(-1, TRACE_WORDS)
+        chain.append(tr[tr[:, 1] > 0])
+    c0 = chain[0][:, 1].min()
+    print("three consecutive calls in one stream (calls 22, 23, 24 of 24), us after the first warp of the first passed its wait:")
+    print("| call | CTAs enter (min .. max) | wait passed (min .. max) | first record lands (mean) | record loop ends (mean, max) | CTA leaves (min, mean, max) |")
+    print("|---|---|---|---|---|---|")
+    for i, T in enumerate(chain):
+        f = lambda x: (x - c0) / 1e3
+        ex = T[:, 12][T[:, 12] > 0]
+        print("| %d | %.1f .. %.1f | %.1f .. %.1f | %.1f | %.1f, %.1f | %.1f, %.1f, %.1f |" % (
+            i, f(T[:, 7].min()), f(T[:, 7].max()), f(T[:, 1].min()), f(T[:, 1].max()), f(T[:, 3].mean()), f(T[:, 4].mean()), f(T[:, 4].max()),
+            f(ex.min()), f(ex.mean()), f(ex.max())))
     keys = [k for k in rows[0] if k != "slow"]
     print("workload %s, %d layers built, %d traced calls (all times in us after the first warp passed the grid-dependency wait)" %
           (args.workload, wl.L, len(rows)))
