@@ -33,11 +33,14 @@ constexpr int kDepth = 3;                         // ring slots per warp
 constexpr int kScratch = 768;                     // per warp: 512 B of fp32 K scales + 256 B of FP16 V scales
 // Per cache format: a BF16 record is 8192 B, so only 8 warps x 3 slots fit in shared memory; its arithmetic is
 // light enough (no unpack) for 8 warps.
-template <int kFmt>
+// kQ: query tokens a warp works on at once (one MMA n-tile of up to 8 heads each).  Two tiles need about 56 more
+// registers per thread, so that variant runs 8 warps of 256 registers, each with a ring twice as deep.
+template <int kFmt, int kQ = 1>
 struct Geo {
-    static constexpr int warps = kFmt == HMA_KV_BFP8 ? kWarps : 8;
+    static constexpr int warps = kFmt == HMA_KV_BFP8 ? kWarps / kQ : 8;
+    static constexpr int depth = kFmt == HMA_KV_BFP8 ? kDepth * kQ : kDepth;      // ring slots per warp
     static constexpr int threads = warps * 32;
-    static constexpr int stages = warps * kDepth;
+    static constexpr int stages = warps * depth;
     static constexpr int record = kFmt == HMA_KV_BFP8 ? kBfp8Record : kBf16Record;
     static constexpr int scratch = kFmt == HMA_KV_BFP8 ? kScratch : 0;
 };
@@ -62,7 +65,9 @@ struct AttnArgs {
     int max_pages;
     const int32_t *ctx;
     int batch;                      // rows of q and out: sequences x query tokens per sequence
-    int q_len;                      // query tokens per sequence; row r is query r % q_len of sequence r / q_len
+    int q_len;                      // query tokens per sequence
+    int rows_per_seq;               // rows of the work list per sequence: q_len / (query tokens per warp); row r belongs
+                                    // to sequence r / rows_per_seq and holds its queries (r % rows_per_seq) * kQ ..
     float sm_scale;
     int32_t *counters;              // workspace: one arrival counter per (sequence, kv head); zero between calls
     int32_t *cum;                   // workspace: pages before each sequence, then pages + segment costs before each
@@ -235,17 +240,26 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float r)
     return (uint16_t)(u >> 16);
 }
 
-// Tokens that row b of the batch attends to.  With one query token per sequence that is the sequence's context (clamped
-// to what the block table can address).  With q_len query tokens the cache already holds all of them: query i sees the
-// context less the q_len - 1 - i newer tokens (causal inside the new tokens), and the q_len rows of a sequence share its
-// block table row.
+// Tokens that row b of the work list attends to.  With one query token per sequence that is the sequence's context
+// (clamped to what the block table can address).  With q_len query tokens the cache already holds all of them: query i
+// sees the context less the q_len - 1 - i newer tokens (causal inside the new tokens), and the rows of a sequence share
+// its block table row.
+// A row of kQ queries walks the pages its newest query sees; its older queries see one token fewer each.
+template <int kQ>
 __device__ __forceinline__ int context_of(const AttnArgs &a, int b)
 {
-    const int s = b / a.q_len, i = b - s * a.q_len;
+    const int s = b / a.rows_per_seq, i = (b - s * a.rows_per_seq) * kQ + kQ - 1;      // the row's newest query
     const int T = max(0, min(a.ctx[s], a.max_pages * kPageTokens));
     return max(0, T - (a.q_len - 1 - i));
 }
-__device__ __forceinline__ int pages_of(const AttnArgs &a, int b) { return (context_of(a, b) + kPageTokens - 1) / kPageTokens; }
+template <int kQ>
+__device__ __forceinline__ int pages_of(const AttnArgs &a, int b) { return (context_of<kQ>(a, b) + kPageTokens - 1) / kPageTokens; }
+// row of q and out that holds query t of work-list row b
+__device__ __forceinline__ int64_t query_row(int q_len, int rows_per_seq, int kq, int b, int t)
+{
+    const int s = b / rows_per_seq;
+    return (int64_t)s * q_len + (int64_t)(b - s * rows_per_seq) * kq + t;
+}
 
 __device__ __forceinline__ void store_out(const AttnArgs &a, int64_t idx, float v)
 {
@@ -285,7 +299,7 @@ struct EpilogueArgs {       // what the reduction needs of AttnArgs, by value (r
     void *out;
     float *tiles, *tails;
     int32_t *counters;
-    int out_dtype, always_partial, batch;
+    int out_dtype, always_partial, batch, q_len, rows_per_seq;
     struct { int num_kv_heads, num_q_heads; } cv;
 #ifdef HMA_TRACE
     unsigned long long *trace;      // this warp's trace words
@@ -305,11 +319,11 @@ constexpr int kGroupInts = 6;        // sequence, kv head, member mask, flags (1
 // entirely: `members` are the warps whose last partial (ring slot 0) belongs to it; a warp that held the segment's end
 // and went on contributes its tail tile (ring slot 1) after them.  If the CTA holds only part of the segment,
 // parts = number of CTAs that share it, first CTA = the lowest.  gstate[0] = number of groups.
-template <int kFmt>
+template <int kFmt, int kQ>
 __device__ __noinline__ void plan_groups(int always_partial, int Hkv, int B, const long long *wr, const int *wseg, const int *cum,
                                          const int *ecum, int *gdesc, int *gstate)
 {
-    constexpr int kWarps = Geo<kFmt>::warps;
+    constexpr int kWarps = Geo<kFmt, kQ>::warps;
     const int lane = threadIdx.x & 31;
     const long long my_lo = lane < kWarps ? wr[2 * lane] : 0, my_hi = lane < kWarps ? wr[2 * lane + 1] : 0;   // lane i: range of warp i
     const unsigned have = __ballot_sync(0xFFFFFFFFu, my_lo < my_hi);
@@ -374,12 +388,13 @@ __device__ __forceinline__ float4 lds_f4(uint32_t addr)
 // Runs once per CTA after all of its warps have parked their last partial (a function of its own so that its
 // registers do not weigh on the record loop).  Work items are (group, q head): one warp each, four channels per
 // lane; lane i weighs the partial of warp i (lane kWarps: the tail tile), so the weights of a group cost one round of
-// loads and two shuffle reductions, and the 128-vectors are then summed in warp order, four loads in flight.
-template <int kFmt>
+// loads and two shuffle reductions, and the 128-vectors are then summed in warp order, all loads in flight.  With two
+// query tiles per warp every (segment, q head) item exists once per tile.
+template <int kFmt, int kQ>
 __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *ring,
                                           int *misc, const int *gdesc, const int *gstate)
 {
-    constexpr int kWarps = Geo<kFmt>::warps, kRecord = Geo<kFmt>::record;
+    constexpr int kWarps = Geo<kFmt, kQ>::warps, kRecord = Geo<kFmt, kQ>::record, kDepth = Geo<kFmt, kQ>::depth;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
     const bool aborted = misc[0] != 0;            // outputs of this CTA are void (and flagged); arrivals still happen
@@ -389,17 +404,17 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
     {
         const int n = gstate[0];
         if (!aborted)
-            for (int item = warp; item < n * 8; item += kWarps) {
-                const int h = item & 7;
+            for (int item = warp; item < n * kQ * 8; item += kWarps) {
+                const int h = item & 7, t = (item >> 3) % kQ;
                 if (h >= G) continue;
-                const int *d = gdesc + (item >> 3) * kGroupInts;
+                const int *d = gdesc + (item >> 3) / kQ * kGroupInts;
                 const int sb = d[0], sg = d[1];
                 const unsigned mem = (unsigned)d[2];
                 const bool whole_seg = d[3] & 1, has_tail = d[3] & 2;
-                const uint32_t gtail = ring_s + ((d[3] >> 8) * kDepth + 1) * kRecord;      // dense tile layout
+                const uint32_t gtail = ring_s + ((d[3] >> 8) * kDepth + kQ + t) * kRecord;      // dense tile layout
                 float mine_m = -INFINITY, mine_l = 0.f;
                 if (lane < kWarps && (mem >> lane & 1u)) {
-                    const uint32_t pc = ring_s + lane * kDepth * kRecord + (8 * kPieceStride + h) * 4;
+                    const uint32_t pc = ring_s + (lane * kDepth + t) * kRecord + (8 * kPieceStride + h) * 4;
                     mine_m = __uint_as_float(lds32(pc)); mine_l = __uint_as_float(lds32(pc + 32));
                 } else if (lane == kWarps && has_tail) {
                     mine_m = __uint_as_float(lds32(gtail + (8 * kHeadDim + h) * 4)); mine_l = __uint_as_float(lds32(gtail + (8 * kHeadDim + 8 + h) * 4));
@@ -409,7 +424,7 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
 #pragma unroll
                 for (int i = 0; i < kWarps; ++i) {
                     v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (mem >> i & 1u) v[i] = lds_f4(ring_s + i * kDepth * kRecord + (h * kPieceStride + 4 * lane) * 4);
+                    if (mem >> i & 1u) v[i] = lds_f4(ring_s + (i * kDepth + t) * kRecord + (h * kPieceStride + 4 * lane) * 4);
                 }
                 v[kWarps] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (has_tail) v[kWarps] = lds_f4(gtail + (h * kHeadDim + 4 * lane) * 4);
@@ -429,10 +444,10 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
                 }
                 if (whole_seg && !a.always_partial) {
                     const float inv = den > 0.f ? 1.f / den : 0.f;
-                    store_quad(a.out, a.out_dtype, ((int64_t)sb * Hq + (int64_t)sg * G + h) * kHeadDim + 4 * lane, acc.x * inv, acc.y * inv,
-                               acc.z * inv, acc.w * inv);
+                    store_quad(a.out, a.out_dtype, (query_row(a.q_len, a.rows_per_seq, kQ, sb, t) * Hq + (int64_t)sg * G + h) * kHeadDim + 4 * lane,
+                               acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
                 } else {
-                    float *tp = a.tiles + ((int64_t)blockIdx.x + (int64_t)sb * Hkv + sg) * kTileFloats;
+                    float *tp = a.tiles + (((int64_t)blockIdx.x + (int64_t)sb * Hkv + sg) * kQ + t) * kTileFloats;
                     *reinterpret_cast<float4 *>(tp + h * kHeadDim + 4 * lane) = acc;
                     if (lane == 0) { tp[8 * kHeadDim + h] = M; tp[8 * kHeadDim + 8 + h] = den; }
                 }
@@ -460,12 +475,12 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
     }
     __syncthreads();
     HMA_TRACE_EPI(a, 10);
-    for (int item = warp; item < n_open * 8; item += kWarps) {
-        const int k = item >> 3, h = item & 7;
+    for (int item = warp; item < n_open * kQ * 8; item += kWarps) {
+        const int k = (item >> 3) / kQ, t = (item >> 3) % kQ, h = item & 7;
         const int parts = misc[4 + 4 * k];
         if (parts == 0 || h >= G) continue;       // another CTA will arrive later and finish this segment
         const int ob = misc[6 + 4 * k], og = misc[7 + 4 * k];
-        const float *t0 = a.tiles + ((int64_t)misc[5 + 4 * k] + (int64_t)ob * Hkv + og) * kTileFloats;       // part i is at t0 + i * kTileFloats
+        const float *t0 = a.tiles + (((int64_t)misc[5 + 4 * k] + (int64_t)ob * Hkv + og) * kQ + t) * kTileFloats;      // part i is at t0 + i * kQ * kTileFloats
         // parts in CTA order, four at a time (one trip to L2 for the usual two to four parts), running maximum
         float M = -INFINITY, den = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -474,7 +489,7 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
             float4 v[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float *tp = t0 + (int64_t)(p0 + j) * kTileFloats;
+                const float *tp = t0 + (int64_t)(p0 + j) * kQ * kTileFloats;
                 const bool ok = p0 + j < parts;
                 mi[j] = ok ? __ldcg(tp + 8 * kHeadDim + h) : -INFINITY;
                 li[j] = ok ? __ldcg(tp + 8 * kHeadDim + 8 + h) : 0.f;
@@ -493,8 +508,8 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
             M = Mn;
         }
         const float inv = den > 0.f ? 1.f / den : 0.f;
-        store_quad(a.out, a.out_dtype, ((int64_t)ob * Hq + (int64_t)og * G + h) * kHeadDim + 4 * lane, acc.x * inv, acc.y * inv, acc.z * inv,
-                   acc.w * inv);
+        store_quad(a.out, a.out_dtype, (query_row(a.q_len, a.rows_per_seq, kQ, ob, t) * Hq + (int64_t)og * G + h) * kHeadDim + 4 * lane,
+                   acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
     }
     HMA_TRACE_EPI(a, 11);
 #ifdef HMA_TRACE
@@ -506,15 +521,16 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
 // 2: the arithmetic of every record on whatever the ring holds, nothing loaded or written (issue-rate probe).
 extern __shared__ __align__(128) uint8_t smem_raw[];
 
-template <int kMode, int kFmt>
-__global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnArgs a)
+template <int kMode, int kFmt, int kQ>
+__global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const AttnArgs a)
 {
-    constexpr int kWarps = Geo<kFmt>::warps, kThreads = Geo<kFmt>::threads, kStages = Geo<kFmt>::stages;
-    constexpr int kRecord = Geo<kFmt>::record;
+    constexpr int kWarps = Geo<kFmt, kQ>::warps, kThreads = Geo<kFmt, kQ>::threads, kStages = Geo<kFmt, kQ>::stages;
+    constexpr int kRecord = Geo<kFmt, kQ>::record, kDepth = Geo<kFmt, kQ>::depth;
+    static_assert(kQ == 1 || kFmt == HMA_KV_BFP8, "two query tiles per warp exist for BFP8 caches only");
     constexpr bool kBfp8 = kFmt == HMA_KV_BFP8;
     uint8_t *ring = smem_raw;                                                     // kStages records
     uint8_t *scratch = ring + kStages * kRecord;                                  // kWarps x kScratch (BFP8 only)
-    uint64_t *bars = reinterpret_cast<uint64_t *>(scratch + kWarps * Geo<kFmt>::scratch);   // full[kStages]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(scratch + kWarps * Geo<kFmt, kQ>::scratch);   // full[kStages]
     int *stage_ok = reinterpret_cast<int *>(bars + kStages);                      // [kStages]
     int *misc = stage_ok + kStages;                                               // [0] abort word, [4..12) epilogue, [16..80) scan scratch
     long long *wr = reinterpret_cast<long long *>(misc + 16 + 64);                // [kWarps][2] record range of each warp
@@ -550,7 +566,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         const int per = (B + kThreads - 1) / kThreads;
         const int b0 = min(B, tid * per), b1 = min(B, b0 + per);
         int mine = 0, emine = 0;
-        for (int b = b0; b < b1; ++b) { const int n = pages_of(a, b); mine += n; emine += n ? n + kSegCost : 0; }
+        for (int b = b0; b < b1; ++b) { const int n = pages_of<kQ>(a, b); mine += n; emine += n ? n + kSegCost : 0; }
         int incl = mine, eincl = emine;                    // inclusive scans inside the warp
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -573,7 +589,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         __syncthreads();
         int run = misc[16 + warp] + incl - mine, erun = misc[16 + 32 + warp] + eincl - emine;
         for (int b = b0; b < b1; ++b) {
-            const int n = pages_of(a, b);
+            const int n = pages_of<kQ>(a, b);
             cum[b] = run; ecum[b] = erun;
             run += n; erun += n ? n + kSegCost : 0;
         }
@@ -611,7 +627,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         cnt = __shfl_sync(0xFFFFFFFFu, cnt, 0);
         if (cnt == kWarps - 1 && kMode == 0) {
             __threadfence_block();
-            plan_groups<kFmt>(a.always_partial, Hkv, B, wr, wseg, cum, ecum, gdesc, gstate);
+            plan_groups<kFmt, kQ>(a.always_partial, Hkv, B, wr, wseg, cum, ecum, gdesc, gstate);
         }
     };
 
@@ -620,7 +636,8 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     if (kMode == 0 && !a.always_partial)                          // empty sequences get rows of zeros
         for (int64_t b = u; b < B; b += NWK)
             if (cum[b + 1] == cum[b])
-                for (int i = lane; i < Hq * kHeadDim; i += 32) store_out(a, b * Hq * kHeadDim + i, 0.f);
+                for (int i = lane; i < kQ * Hq * kHeadDim; i += 32)
+                    store_out(a, query_row(a.q_len, a.rows_per_seq, kQ, (int)b, i / (Hq * kHeadDim)) * Hq * kHeadDim + i % (Hq * kHeadDim), 0.f);
 
     // number of records that lie before cost position p
     auto records_before = [&](int64_t p) -> int64_t {
@@ -685,7 +702,7 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
             const int npb = cum[lo + 1] - cum[lo];
             const int off = (int)(wr - (int64_t)Hkv * cum[lo]);
             const int gg = off / npb, pp = off - gg * npb;
-            const int32_t pid = a.block_table[(int64_t)(lo / a.q_len) * a.max_pages + pp];
+            const int32_t pid = a.block_table[(int64_t)(lo / a.rows_per_seq) * a.max_pages + pp];
             if (pid >= 0 && pid < a.cv.num_pages) roff = (uint32_t)(((int64_t)pid * Hkv + gg) * (kRecord / 128));
         }
     };
@@ -720,13 +737,14 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     // ---- consumer state ----
     const int gq = lane >> 2, t4 = lane & 3;
     const float kLog2e = 1.4426950408889634f;
-    const uint32_t scrK = smem_u32(scratch + warp * Geo<kFmt>::scratch);   // fp32 2^(E-127) of every (token, block) of K
+    const uint32_t scrK = smem_u32(scratch + warp * Geo<kFmt, kQ>::scratch);   // fp32 2^(E-127) of every (token, block) of K
     const uint32_t scrV = scrK + 512;                            // FP16 scales of every (token pair, block) of V
-    uint32_t qf[8][2];
-    float cs0 = 0.f, cs1 = 0.f;                    // score multipliers of heads 2*t4, 2*t4+1
-    float m0 = -INFINITY, m1 = -INFINITY;          // running maxima (log2 domain) of heads 2*t4, 2*t4+1
-    float lacc[4] = {0.f, 0.f, 0.f, 0.f};          // running sums, via an all-ones MMA
-    float o[8][4];
+    // per query tile t (one query token of the row, its up to 8 heads on the MMA's N side):
+    uint32_t qf[kQ][8][2];
+    float cs0[kQ], cs1[kQ];                        // score multipliers of heads 2*t4, 2*t4+1
+    float m0[kQ], m1[kQ];                          // running maxima (log2 domain) of heads 2*t4, 2*t4+1
+    float lacc[kQ][4];                             // running sums, via an all-ones MMA
+    float o[kQ][8][4];
     int Rmine = 0;                                 // reference exponent of V channel block (lane & 7)
     int T = 0, tail = kPageTokens;
     bool whole = false;                            // this warp holds every record of the current segment
@@ -734,63 +752,66 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
 
     auto begin_segment = [&](int k) {
         np = cum[b + 1] - cum[b];
-        T = context_of(a, b);
+        T = context_of<kQ>(a, b);
         tail = T - (np - 1) * kPageTokens;
         whole = page == 0 && Rw - k >= np;
-        // Q fragments of this (sequence, kv head): FP16, one power-of-two scale per head
-        float f[8][4];
-        float amax = 0.f;
+        // Q fragments of this (sequence, kv head), per query token: FP16, one power-of-two scale per head
         const bool hv = gq < G && kMode == 0;      // the probes have no Q: nothing is read through a.q
-        const uint16_t *qrow = a.q + ((int64_t)b * Hq + (int64_t)g * G + (hv ? gq : 0)) * kHeadDim;
         const bool inter = a.cv.key_layout == HMA_KEYS_INTERLEAVED;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            // this lane's cached key channels 16j + 4*t4 .. +3 meet the query channels of the same rotary pairs
-            uint2 v = make_uint2(0u, 0u);
-            if (hv && !inter) v = *reinterpret_cast<const uint2 *>(qrow + 16 * j + 4 * t4);
-            if (hv && inter) {
-                const uint32_t lo = *reinterpret_cast<const uint32_t *>(qrow + 8 * j + 2 * t4);        // q[a], q[a+1]
-                const uint32_t hi = *reinterpret_cast<const uint32_t *>(qrow + 8 * j + 2 * t4 + 64);   // q[a+64], q[a+65]
-                v.x = (lo & 0xFFFFu) | (hi << 16);            // key channels 4*t4, 4*t4+1  <- q[a], q[a+64]
-                v.y = (lo >> 16) | (hi & 0xFFFF0000u);        // key channels 4*t4+2, +3    <- q[a+1], q[a+65]
-            }
-            f[j][0] = __uint_as_float(v.x << 16);
-            f[j][1] = __uint_as_float(v.x & 0xFFFF0000u);
-            f[j][2] = __uint_as_float(v.y << 16);
-            f[j][3] = __uint_as_float(v.y & 0xFFFF0000u);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) amax = fmaxf(amax, fabsf(f[j][c]));
-        }
-        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
-        float cs;
-        if (kBfp8) {
-            int shift = 0;
-            if (amax > 0.f && amax < INFINITY) shift = 14 - ((int)((__float_as_uint(amax) >> 23) & 0xFF) - 127);
-            shift = max(-120, min(120, shift));
-            const float up = pow2_field(127 + shift), down = pow2_field(127 - shift);
+        for (int t = 0; t < kQ; ++t) {
+            float f[8][4];
+            float amax = 0.f;
+            const uint16_t *qrow = a.q + ((query_row(a.q_len, a.rows_per_seq, kQ, b, t) * Hq + (int64_t)g * G + (hv ? gq : 0))) * kHeadDim;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                qf[j][0] = pack_half2(f[j][0] * up, f[j][1] * up);
-                qf[j][1] = pack_half2(f[j][2] * up, f[j][3] * up);
-            }
-            // mantissas enter as m * 2^-24 and exponents as 2^(E-127) while values are m * 2^(E-133): 2^18 is owed
-            cs = a.sm_scale * kLog2e * down * 262144.f;
-        } else {
+                // this lane's cached key channels 16j + 4*t4 .. +3 meet the query channels of the same rotary pairs
+                uint2 v = make_uint2(0u, 0u);
+                if (hv && !inter) v = *reinterpret_cast<const uint2 *>(qrow + 16 * j + 4 * t4);
+                if (hv && inter) {
+                    const uint32_t lo = *reinterpret_cast<const uint32_t *>(qrow + 8 * j + 2 * t4);        // q[a], q[a+1]
+                    const uint32_t hi = *reinterpret_cast<const uint32_t *>(qrow + 8 * j + 2 * t4 + 64);   // q[a+64], q[a+65]
+                    v.x = (lo & 0xFFFFu) | (hi << 16);            // key channels 4*t4, 4*t4+1  <- q[a], q[a+64]
+                    v.y = (lo >> 16) | (hi & 0xFFFF0000u);        // key channels 4*t4+2, +3    <- q[a+1], q[a+65]
+                }
+                f[j][0] = __uint_as_float(v.x << 16);
+                f[j][1] = __uint_as_float(v.x & 0xFFFF0000u);
+                f[j][2] = __uint_as_float(v.y << 16);
+                f[j][3] = __uint_as_float(v.y & 0xFFFF0000u);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {       // Q stays BF16: exact repacking of the loaded bits
-                qf[j][0] = (__float_as_uint(f[j][0]) >> 16) | (__float_as_uint(f[j][1]) & 0xFFFF0000u);
-                qf[j][1] = (__float_as_uint(f[j][2]) >> 16) | (__float_as_uint(f[j][3]) & 0xFFFF0000u);
+                for (int c = 0; c < 4; ++c) amax = fmaxf(amax, fabsf(f[j][c]));
             }
-            cs = a.sm_scale * kLog2e;
+            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+            float cs;
+            if (kBfp8) {
+                int shift = 0;
+                if (amax > 0.f && amax < INFINITY) shift = 14 - ((int)((__float_as_uint(amax) >> 23) & 0xFF) - 127);
+                shift = max(-120, min(120, shift));
+                const float up = pow2_field(127 + shift), down = pow2_field(127 - shift);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    qf[t][j][0] = pack_half2(f[j][0] * up, f[j][1] * up);
+                    qf[t][j][1] = pack_half2(f[j][2] * up, f[j][3] * up);
+                }
+                // mantissas enter as m * 2^-24 and exponents as 2^(E-127) while values are m * 2^(E-133): 2^18 is owed
+                cs = a.sm_scale * kLog2e * down * 262144.f;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {       // Q stays BF16: exact repacking of the loaded bits
+                    qf[t][j][0] = (__float_as_uint(f[j][0]) >> 16) | (__float_as_uint(f[j][1]) & 0xFFFF0000u);
+                    qf[t][j][1] = (__float_as_uint(f[j][2]) >> 16) | (__float_as_uint(f[j][3]) & 0xFFFF0000u);
+                }
+                cs = a.sm_scale * kLog2e;
+            }
+            cs0[t] = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4) * 4);
+            cs1[t] = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4 + 1) * 4);
+            m0[t] = -INFINITY;
+            m1[t] = -INFINITY;
+            lacc[t][0] = lacc[t][1] = lacc[t][2] = lacc[t][3] = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) o[t][j][0] = o[t][j][1] = o[t][j][2] = o[t][j][3] = 0.f;
         }
-        cs0 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4) * 4);
-        cs1 = __shfl_sync(0xFFFFFFFFu, cs, (2 * t4 + 1) * 4);
-        m0 = -INFINITY;
-        m1 = -INFINITY;
-        lacc[0] = lacc[1] = lacc[2] = lacc[3] = 0.f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
         Rmine = 0;
     };
 
@@ -798,54 +819,59 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
     // to `out`, or as a partial tile for the two-cache merge).  Otherwise the partial (o, m, l) waits for the CTA-level
     // reduction: in the warp's ring slot 0 if these were the warp's last records (the ring is idle by then), else (the
     // warp goes on into the next segment, so it held the end of this one, and only one warp does) in the segment's
-    // tail tile in global memory, which the warp copies back into its ring slot 1 once its ring is idle.
+    // tail tile in global memory, which the warp copies back into its ring slot kQ + t once its ring is idle (per query
+    // tile t: slots 0 .. kQ-1 hold the last partial, slots kQ .. 2kQ-1 the tail tile).
     auto finish_segment = [&](bool at_end) {
         if (kMode == 1) return;
-        if (kBfp8) {
-            // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float vsc = pow2_field(min(__shfl_sync(0xFFFFFFFFu, Rmine, j) + 3, 254));
-                o[j][0] *= vsc; o[j][1] *= vsc; o[j][2] *= vsc; o[j][3] *= vsc;
-            }
-        }
-        const float l0 = lacc[0], l1 = lacc[1];
         const int h0 = 2 * t4, h1 = 2 * t4 + 1;
-        // a softmax sum that is not finite: scores overflowed fp32 (K exponents beyond the supported range)
-        if (kMode == 0 && (!(l0 < INFINITY) || !(l1 < INFINITY))) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);
-        const int64_t ob = ((int64_t)b * Hq + (int64_t)g * G) * kHeadDim;
-        if (kMode == 2 && a.batch >= 0) return;    // the issue-rate probe never stores, but keeps its arithmetic live
-        if (whole && !a.always_partial) {
-            const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+        const int64_t seg = (int64_t)b * Hkv + g;
+        if (!whole && !at_end) tail_seg = seg;
+#pragma unroll
+        for (int t = 0; t < kQ; ++t) {
+            if (kBfp8) {
+                // to true units: accumulators hold sum p * m * 2^(E - R - 9); values are m * 2^(E-133)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float vsc = pow2_field(min(__shfl_sync(0xFFFFFFFFu, Rmine, j) + 3, 254));
+                    o[t][j][0] *= vsc; o[t][j][1] *= vsc; o[t][j][2] *= vsc; o[t][j][3] *= vsc;
+                }
+            }
+            const float l0 = lacc[t][0], l1 = lacc[t][1];
+            // a softmax sum that is not finite: scores overflowed fp32 (K exponents beyond the supported range)
+            if (kMode == 0 && (!(l0 < INFINITY) || !(l1 < INFINITY))) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);
+            if (kMode == 2 && a.batch >= 0) continue;    // the issue-rate probe never stores, but keeps its arithmetic live
+            if (whole && !a.always_partial) {
+                const int64_t ob = (query_row(a.q_len, a.rows_per_seq, kQ, b, t) * Hq + (int64_t)g * G) * kHeadDim;
+                const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int h = (c & 1) ? h1 : h0;
+                        if (h < G) store_out(a, ob + h * kHeadDim + 16 * j + gq + 8 * (c >> 1), o[t][j][c] * ((c & 1) ? i1 : i0));
+                    }
+                continue;
+            }
+            float *tp;
+            int hs;           // floats between heads
+            if (whole) {      // two-cache attention: nobody else touches this segment, its tile goes straight to global memory
+                tp = a.tiles + (((int64_t)blockIdx.x + seg) * kQ + t) * kTileFloats;
+                hs = kHeadDim;
+            } else if (at_end) {
+                tp = reinterpret_cast<float *>(ring + (warp * kDepth + t) * kRecord);
+                hs = kPieceStride;
+            } else {
+                tp = a.tails + (seg * kQ + t) * kTileFloats;
+                hs = kHeadDim;
+            }
 #pragma unroll
             for (int j = 0; j < 8; ++j)
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int h = (c & 1) ? h1 : h0;
-                    if (h < G) store_out(a, ob + h * kHeadDim + 16 * j + gq + 8 * (c >> 1), o[j][c] * ((c & 1) ? i1 : i0));
-                }
-            return;
-        }
-        float *tp;
-        int hs;           // floats between heads
-        if (whole) {      // two-cache attention: nobody else touches this segment, its tile goes straight to global memory
-            tp = a.tiles + ((int64_t)blockIdx.x + (int64_t)b * Hkv + g) * kTileFloats;
-            hs = kHeadDim;
-        } else if (at_end) {
-            tp = reinterpret_cast<float *>(ring + (warp * kDepth) * kRecord);
-            hs = kPieceStride;
-        } else {
-            tail_seg = (int64_t)b * Hkv + g;
-            tp = a.tails + tail_seg * kTileFloats;
-            hs = kHeadDim;
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tp[((c & 1) ? h1 : h0) * hs + 16 * j + gq + 8 * (c >> 1)] = o[j][c];
-        if (gq == 0) {
-            tp[8 * hs + h0] = m0; tp[8 * hs + h1] = m1;
-            tp[8 * hs + 8 + h0] = l0; tp[8 * hs + 8 + h1] = l1;
+                for (int c = 0; c < 4; ++c) tp[((c & 1) ? h1 : h0) * hs + 16 * j + gq + 8 * (c >> 1)] = o[t][j][c];
+            if (gq == 0) {
+                tp[8 * hs + h0] = m0[t]; tp[8 * hs + h1] = m1[t];
+                tp[8 * hs + 8 + h0] = l0; tp[8 * hs + 8 + h1] = l1;
+            }
         }
     };
 
@@ -885,7 +911,8 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         }
         if (++slot == kDepth) { slot = 0; par ^= 1u; }
         const bool ok = kMode == 2 || stage_ok[s_idx] != 0;
-        const int nvalid = page == np - 1 ? tail : kPageTokens;
+        const bool last_page = page == np - 1;
+        const int nvalid = last_page ? tail : kPageTokens;
         ++page;
         if (kMode == 1 || !ok) {
             __syncwarp();
@@ -922,7 +949,8 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                     for (int j = 0; j < 8; ++j) {
                         const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
                         const float fr = dlt < -126 ? 0.f : pow2_field(127 + dlt);
-                        o[j][0] *= fr; o[j][1] *= fr; o[j][2] *= fr; o[j][3] *= fr;
+    #pragma unroll
+                        for (int t = 0; t < kQ; ++t) { o[t][j][0] *= fr; o[t][j][1] *= fr; o[t][j][2] *= fr; o[t][j][3] *= fr; }
                     }
                     Rmine = Rnew;
                 }
@@ -937,7 +965,9 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
             __syncwarp();
 
             // ================= Q.K^T =================
-            float sc[4] = {0.f, 0.f, 0.f, 0.f};
+            float sc[kQ][4];
+    #pragma unroll
+            for (int t = 0; t < kQ; ++t) sc[t][0] = sc[t][1] = sc[t][2] = sc[t][3] = 0.f;
             {
                 float ks[16];      // 2^(E-127): token gq blocks 0..7, token gq+8 blocks 0..7
     #pragma unroll
@@ -957,12 +987,15 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                     af[1] = prmt(wh, 0u, 0x1100u) & 0x807F807Fu;
                     af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
                     af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
-                    float d[4];
-                    mma_f16(d, af, qf[j][0], qf[j][1], zero4);
-                    sc[0] = fmaf(d[0], ks[j], sc[0]);
-                    sc[1] = fmaf(d[1], ks[j], sc[1]);
-                    sc[2] = fmaf(d[2], ks[8 + j], sc[2]);
-                    sc[3] = fmaf(d[3], ks[8 + j], sc[3]);
+    #pragma unroll
+                    for (int t = 0; t < kQ; ++t) {       // the unpacked keys serve every query tile
+                        float d[4];
+                        mma_f16(d, af, qf[t][j][0], qf[t][j][1], zero4);
+                        sc[t][0] = fmaf(d[0], ks[j], sc[t][0]);
+                        sc[t][1] = fmaf(d[1], ks[j], sc[t][1]);
+                        sc[t][2] = fmaf(d[2], ks[8 + j], sc[t][2]);
+                        sc[t][3] = fmaf(d[3], ks[8 + j], sc[t][3]);
+                    }
                 }
             }
             // the V element words go to registers now, so that the ring slot can be re-armed for the record
@@ -975,34 +1008,42 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                 if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads above, bulk write below
                 issue();
             }
-            float s0 = sc[0] * cs0, s1 = sc[1] * cs1, s2 = sc[2] * cs0, s3 = sc[3] * cs1;
-            if (nvalid < kPageTokens) {
-                if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
-                if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
-            }
-            // ================= online softmax (log2 domain) =================
-            // The warp-wide maximum is only formed when some score exceeds the running maximum.
-            if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
-                float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
+            uint32_t pb0[kQ], pb1[kQ];
     #pragma unroll
-                for (int d = 4; d <= 16; d <<= 1) {
-                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
+            for (int t = 0; t < kQ; ++t) {
+                float s0 = sc[t][0] * cs0[t], s1 = sc[t][1] * cs1[t], s2 = sc[t][2] * cs0[t], s3 = sc[t][3] * cs1[t];
+                // query t of the row sees kQ - 1 - t tokens fewer than the row's newest query: they are the last tokens
+                // of the last page
+                const int nv = kQ == 1 ? nvalid : nvalid - (last_page ? kQ - 1 - t : 0);
+                if (nv < kPageTokens) {
+                    if (gq >= nv) { s0 = -INFINITY; s1 = -INFINITY; }
+                    if (gq + 8 >= nv) { s2 = -INFINITY; s3 = -INFINITY; }
                 }
-                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-                const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
-                m0 = mn0;
-                m1 = mn1;
-                lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
+                // ================= online softmax (log2 domain) =================
+                // The warp-wide maximum is only formed when some score exceeds the running maximum.
+                if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0[t] || fmaxf(s1, s3) > m1[t])) {
+                    float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
     #pragma unroll
-                for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
-            }
-            // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
-            const uint32_t pb0 = movmatrix_trans(pack_half2(ex2f(s0 - m0), ex2f(s1 - m1)));   // tokens 2*t4, 2*t4+1 of head gq
-            const uint32_t pb1 = movmatrix_trans(pack_half2(ex2f(s2 - m0), ex2f(s3 - m1)));   // tokens 2*t4+8, 2*t4+9
-            {
+                    for (int d = 4; d <= 16; d <<= 1) {
+                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
+                    }
+                    const float mn0 = fmaxf(m0[t], mx0), mn1 = fmaxf(m1[t], mx1);
+                    const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0[t] - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1[t] - mn1);
+                    m0[t] = mn0;
+                    m1[t] = mn1;
+                    lacc[t][0] *= a0; lacc[t][1] *= a1; lacc[t][2] *= a0; lacc[t][3] *= a1;
+    #pragma unroll
+                    for (int j = 0; j < 8; ++j) { o[t][j][0] *= a0; o[t][j][1] *= a1; o[t][j][2] *= a0; o[t][j][3] *= a1; }
+                }
+                // With several query tiles a tile may not have seen any token yet (its only token so far is masked): its
+                // maximum is still -inf and every score is -inf; the weights must then be 0, not exp2(-inf + inf).
+                const float r0 = (kQ > 1 && m0[t] == -INFINITY) ? 0.f : m0[t], r1 = (kQ > 1 && m1[t] == -INFINITY) ? 0.f : m1[t];
+                // weights as FP16, transposed from (token, head) accumulator layout to the B-operand layout
+                pb0[t] = movmatrix_trans(pack_half2(ex2f(s0 - r0), ex2f(s1 - r1)));   // tokens 2*t4, 2*t4+1 of head gq
+                pb1[t] = movmatrix_trans(pack_half2(ex2f(s2 - r0), ex2f(s3 - r1)));   // tokens 2*t4+8, 2*t4+9
                 const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
-                mma_f16_acc(lacc, ones, pb0, pb1);
+                mma_f16_acc(lacc[t], ones, pb0[t], pb1[t]);
             }
             // ================= P.V =================
             {
@@ -1019,7 +1060,8 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                     af[2] = prmt(wl, 0u, 0x3322u) & 0x807F807Fu;
                     af[3] = prmt(wh, 0u, 0x3322u) & 0x807F807Fu;
                     const uint32_t f01 = (j & 1) ? vs[j >> 1].z : vs[j >> 1].x, f89 = (j & 1) ? vs[j >> 1].w : vs[j >> 1].y;
-                    mma_f16_acc(o[j], af, hmul2_u32(pb0, f01), hmul2_u32(pb1, f89));
+    #pragma unroll
+                    for (int t = 0; t < kQ; ++t) mma_f16_acc(o[t][j], af, hmul2_u32(pb0[t], f01), hmul2_u32(pb1[t], f89));
                 }
             }
             __syncwarp();      // every lane is done with the scratch tables
@@ -1032,8 +1074,8 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                 const uint4 klo = lds128(sp + (2 * jp) * 512 + lane * 16);       // token gq: blocks 2jp, 2jp+1
                 const uint4 khi = lds128(sp + (2 * jp + 1) * 512 + lane * 16);   // token gq+8
                 const uint32_t a0[4] = {klo.x, khi.x, klo.y, khi.y}, a1[4] = {klo.z, khi.z, klo.w, khi.w};
-                mma_bf16_acc(sca, a0, qf[2 * jp][0], qf[2 * jp][1]);
-                mma_bf16_acc(scb, a1, qf[2 * jp + 1][0], qf[2 * jp + 1][1]);
+                mma_bf16_acc(sca, a0, qf[0][2 * jp][0], qf[0][2 * jp][1]);
+                mma_bf16_acc(scb, a1, qf[0][2 * jp + 1][0], qf[0][2 * jp + 1][1]);
             }
             // the V words go to registers now, so that the ring slot can be re-armed while softmax and P.V run
             uint4 vm[8];
@@ -1051,28 +1093,28 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
                 if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads above, bulk write below
                 issue();
             }
-            float s0 = (sca[0] + scb[0]) * cs0, s1 = (sca[1] + scb[1]) * cs1, s2 = (sca[2] + scb[2]) * cs0, s3 = (sca[3] + scb[3]) * cs1;
+            float s0 = (sca[0] + scb[0]) * cs0[0], s1 = (sca[1] + scb[1]) * cs1[0], s2 = (sca[2] + scb[2]) * cs0[0], s3 = (sca[3] + scb[3]) * cs1[0];
             if (nvalid < kPageTokens) {
                 if (gq >= nvalid) { s0 = -INFINITY; s1 = -INFINITY; }
                 if (gq + 8 >= nvalid) { s2 = -INFINITY; s3 = -INFINITY; }
             }
-            if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0 || fmaxf(s1, s3) > m1)) {
+            if (__any_sync(0xFFFFFFFFu, fmaxf(s0, s2) > m0[0] || fmaxf(s1, s3) > m1[0])) {
                 float mx0 = fmaxf(s0, s2), mx1 = fmaxf(s1, s3);
 #pragma unroll
                 for (int d = 4; d <= 16; d <<= 1) {
                     mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, d));
                     mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, d));
                 }
-                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-                const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0 - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1 - mn1);
-                m0 = mn0;
-                m1 = mn1;
-                lacc[0] *= a0; lacc[1] *= a1; lacc[2] *= a0; lacc[3] *= a1;
+                const float mn0 = fmaxf(m0[0], mx0), mn1 = fmaxf(m1[0], mx1);
+                const float a0 = mn0 == -INFINITY ? 1.f : ex2f(m0[0] - mn0), a1 = mn1 == -INFINITY ? 1.f : ex2f(m1[0] - mn1);
+                m0[0] = mn0;
+                m1[0] = mn1;
+                lacc[0][0] *= a0; lacc[0][1] *= a1; lacc[0][2] *= a0; lacc[0][3] *= a1;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { o[j][0] *= a0; o[j][1] *= a1; o[j][2] *= a0; o[j][3] *= a1; }
+                for (int j = 0; j < 8; ++j) { o[0][j][0] *= a0; o[0][j][1] *= a1; o[0][j][2] *= a0; o[0][j][3] *= a1; }
             }
             // weights as BF16 hi + lo (16 significant bits): BF16-rounded weights alone would cost 1e-3 of relative error
-            const float p0 = ex2f(s0 - m0), p1 = ex2f(s1 - m1), p2 = ex2f(s2 - m0), p3 = ex2f(s3 - m1);
+            const float p0 = ex2f(s0 - m0[0]), p1 = ex2f(s1 - m1[0]), p2 = ex2f(s2 - m0[0]), p3 = ex2f(s3 - m1[0]);
             const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);
             const uint32_t l01 = pack_bf16x2(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xFFFF0000u));
             const uint32_t l23 = pack_bf16x2(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xFFFF0000u));
@@ -1080,15 +1122,15 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
             const uint32_t pl0 = movmatrix_trans(l01), pl1 = movmatrix_trans(l23);
             {
                 const uint32_t ones[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};
-                mma_bf16_acc(lacc, ones, ph0, ph1);
-                mma_bf16_acc(lacc, ones, pl0, pl1);
+                mma_bf16_acc(lacc[0], ones, ph0, ph1);
+                mma_bf16_acc(lacc[0], ones, pl0, pl1);
             }
             // P.V: channels on M, tokens on K; one 16-byte word per lane is one operand fragment
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const uint32_t af[4] = {vm[j].x, vm[j].y, vm[j].z, vm[j].w};
-                mma_bf16_acc(o[j], af, ph0, ph1);
-                mma_bf16_acc(o[j], af, pl0, pl1);
+                mma_bf16_acc(o[0][j], af, ph0, ph1);
+                mma_bf16_acc(o[0][j], af, pl0, pl1);
             }
         }
     }
@@ -1099,15 +1141,18 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
             // the last tail tile this warp wrote (it can only be shared with other warps if it was the warp's first
             // segment, and a warp writes at most one such) comes back from L2 into ring slot 1, same layout
             __syncwarp();
-            const uint4 *src = reinterpret_cast<const uint4 *>(a.tails + tail_seg * kTileFloats);
-            const uint32_t dst = ring0 + kRecord;
-            uint4 v[(kTileFloats * 4 / 16 + 31) / 32];
 #pragma unroll
-            for (int i = 0; i < (kTileFloats * 4 / 16 + 31) / 32; ++i)
-                if (lane + 32 * i < kTileFloats * 4 / 16) v[i] = __ldcg(src + lane + 32 * i);
+            for (int t = 0; t < kQ; ++t) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(a.tails + (tail_seg * kQ + t) * kTileFloats);
+                const uint32_t dst = ring0 + (kQ + t) * kRecord;
+                uint4 v[(kTileFloats * 4 / 16 + 31) / 32];
 #pragma unroll
-            for (int i = 0; i < (kTileFloats * 4 / 16 + 31) / 32; ++i)
-                if (lane + 32 * i < kTileFloats * 4 / 16) sts128(dst + (lane + 32 * i) * 16, v[i].x, v[i].y, v[i].z, v[i].w);
+                for (int i = 0; i < (kTileFloats * 4 / 16 + 31) / 32; ++i)
+                    if (lane + 32 * i < kTileFloats * 4 / 16) v[i] = __ldcg(src + lane + 32 * i);
+#pragma unroll
+                for (int i = 0; i < (kTileFloats * 4 / 16 + 31) / 32; ++i)
+                    if (lane + 32 * i < kTileFloats * 4 / 16) sts128(dst + (lane + 32 * i) * 16, v[i].x, v[i].y, v[i].z, v[i].w);
+            }
         }
     }
     HMA_TRACE_STAMP(a, u, 5, trace_now());
@@ -1123,11 +1168,12 @@ __global__ void __launch_bounds__(Geo<kFmt>::threads, 1) attn_kernel(const AttnA
         EpilogueArgs e;
         e.out = a.out; e.tiles = a.tiles; e.tails = a.tails; e.counters = a.counters;
         e.out_dtype = a.out_dtype; e.always_partial = a.always_partial; e.batch = a.batch;
+        e.q_len = a.q_len; e.rows_per_seq = a.rows_per_seq;
         e.cv.num_kv_heads = a.cv.num_kv_heads; e.cv.num_q_heads = a.cv.num_q_heads;
 #ifdef HMA_TRACE
         e.trace = a.trace + (((int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * sp.nwk / sp.ctas : 0) + warp) * kTraceWords;
 #endif
-        cta_epilogue<kFmt>(e, ring, misc, gdesc, gstate);
+        cta_epilogue<kFmt, kQ>(e, ring, misc, gdesc, gstate);
     }
 }
 
@@ -1216,10 +1262,10 @@ __global__ void __launch_bounds__(256) attn_merge_mixed_kernel(const AttnArgs a,
     }
 }
 
-template <int kFmt>
+template <int kFmt, int kQ = 1>
 static size_t attn_smem_bytes(int batch)
 {
-    using G = Geo<kFmt>;
+    using G = Geo<kFmt, kQ>;
     return (size_t)G::stages * G::record + (size_t)G::warps * G::scratch + G::stages * 8 + G::stages * 4 + (16 + 64) * 4 +
            (size_t)G::warps * 24 + (kMaxGroups * kGroupInts + 4) * 4 + ((size_t)batch + 1) * 8;
 }
@@ -1229,7 +1275,7 @@ static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 8 + 255) & ~(
 // The counters sit at the head of the workspace in a region of one size for every call, whatever its batch and head
 // count, so that calls of different shapes can share a workspace without one's tiles landing on the other's counters.
 static size_t counter_bytes(int, int) { return (size_t)kMaxBatch * kMaxKvHeads * 4; }
-static size_t cta_tiles(int batch, int hkv) { return (size_t)kMaxCtas + (size_t)batch * hkv; }
+static size_t cta_tiles(int batch, int hkv) { return 2 * (size_t)kMaxCtas + (size_t)batch * hkv; }     // enough for two query tiles per row
 
 }  // namespace hma
 
@@ -1283,6 +1329,10 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     if (workspace_bytes < hma_decode_attention_workspace_bytes(&cache->desc, batch)) return HMA_ERR_WORKSPACE_TOO_SMALL;
     const bool bf16 = cache->desc.format != HMA_KV_BFP8;
     if (bf16 && probe == 2) return HMA_ERR_UNSUPPORTED_SHAPE;
+    // Two query tokens per warp (they share the unpacked K and V operands) when the query count is even, on BFP8 caches;
+    // otherwise every query token is a row of its own.
+    const int kq = (!bf16 && probe == 0 && !always_partial && q_len % 2 == 0) ? 2 : 1;
+    const int32_t rows = batch / kq;              // rows of the work list
     // per-device set-up, done by the first call on each device: SM count and the kernels' shared-memory opt-in
     static std::mutex setup_lock;
     static int sm_count[hma::kMaxDevices] = {};
@@ -1295,16 +1345,18 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
         if (!sm_count[dev]) {
             int n = 0;
             HMA_CUDA_OK(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
-            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<2, HMA_KV_BFP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BFP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<2, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             sm_count[dev] = n;
         }
     }
     const int n_sm = sm_count[dev];
-    const size_t smem = bf16 ? hma::attn_smem_bytes<HMA_KV_BF16>(batch) : hma::attn_smem_bytes<HMA_KV_BFP8>(batch);
+    const size_t smem = bf16 ? hma::attn_smem_bytes<HMA_KV_BF16>(rows)
+                             : kq == 2 ? hma::attn_smem_bytes<HMA_KV_BFP8, 2>(rows) : hma::attn_smem_bytes<HMA_KV_BFP8>(rows);
     if (smem > 227 * 1024) return HMA_ERR_UNSUPPORTED_SHAPE;
     hma::AttnArgs a;
     a.cv = hma::CacheView{(uint8_t *)cache->layers[layer], cache->desc.num_pages, cache->desc.num_kv_heads,
@@ -1315,14 +1367,15 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.block_table = block_table;
     a.max_pages = max_pages_per_seq;
     a.ctx = context_lens;
-    a.batch = batch;
+    a.batch = rows;
     a.q_len = q_len;
+    a.rows_per_seq = q_len / kq;
     a.sm_scale = sm_scale;
     const int hkv = cache->desc.num_kv_heads;
     a.counters = (int32_t *)workspace;
     a.cum = (int32_t *)((uint8_t *)workspace + hma::counter_bytes(batch, hkv));
     a.tiles = (float *)((uint8_t *)a.cum + hma::cum_bytes(batch));
-    a.tails = a.tiles + hma::cta_tiles(batch, hkv) * hma::kTileFloats;
+    a.tails = a.tiles + hma::cta_tiles(batch, hkv) * hma::kTileFloats;      // batch = rows x query tiles per row
     a.always_partial = always_partial;
 #ifdef HMA_TRACE
     a.trace = (unsigned long long *)(a.tails + (size_t)batch * hkv * hma::kTileFloats);
@@ -1332,7 +1385,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
 #endif
     const int n_ctas = n_sm < hma::kMaxCtas ? n_sm : hma::kMaxCtas;
     cudaStream_t s = (cudaStream_t)stream;
-    constexpr int tb = hma::Geo<HMA_KV_BFP8>::threads, tf = hma::Geo<HMA_KV_BF16>::threads;
+    const int tb = kq == 2 ? hma::Geo<HMA_KV_BFP8, 2>::threads : hma::Geo<HMA_KV_BFP8>::threads, tf = hma::Geo<HMA_KV_BF16>::threads;
     // The kernel is launched with programmatic stream serialisation: it may be placed on the SMs while its
     // predecessor drains, and it waits on the grid dependency itself before it reads anything.
     cudaLaunchAttribute attr[1];
@@ -1345,11 +1398,12 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (bf16 && probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BF16>, a));
-    else if (bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BF16>, a));
-    else if (probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BFP8>, a));
-    else if (probe == 1) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BFP8>, a));
-    else HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<2, HMA_KV_BFP8>, a));
+    if (bf16 && probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BF16, 1>, a));
+    else if (bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BF16, 1>, a));
+    else if (probe == 0 && kq == 2) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BFP8, 2>, a));
+    else if (probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BFP8, 1>, a));
+    else if (probe == 1) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BFP8, 1>, a));
+    else HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<2, HMA_KV_BFP8, 1>, a));
     hma::count_launch();
     if (args_out) *args_out = a;
     if (ctas_out) *ctas_out = n_ctas;
