@@ -189,8 +189,9 @@ hma_status_t hma_decode_attention(const hma_cache_t *cache, int32_t layer,
  * t < context_lens[b] - (q_len - 1 - i).  A query that sees no token gives a row of zeros.
  *   q, out       [batch][q_len][num_q_heads][128]
  *   workspace    >= hma_decode_attention_workspace_bytes(desc, batch * q_len); batch * q_len <= 1024
- * Everything else as hma_decode_attention, of which this is the q_len = 1 case.  The q_len rows of a sequence walk the
- * same pages at the same time, so HBM is read about once and the L2 serves the rest; the arithmetic is not shared.
+ * Everything else as hma_decode_attention, of which this is the q_len = 1 case.  With an even q_len on a BFP8 cache
+ * two query tokens are handled per warp and share the unpacked K and V operands (about 1.2x per query token); otherwise
+ * every query token costs what a sequence of hma_decode_attention costs.
  */
 hma_status_t hma_decode_attention_multi(const hma_cache_t *cache, int32_t layer,
                                         const void *q, void *out, int32_t out_dtype,
