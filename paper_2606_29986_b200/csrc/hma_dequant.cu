@@ -6,16 +6,26 @@
 namespace hma {
 
 // Four elements of one block -> four BF16 bit patterns, bit-exact for every (E, byte) pair.
-// The byte s<<7|m is first spread to the FP16 pattern s<<15|m, the FP16 subnormal +-m * 2^-24 (two integer
-// instructions per pair: the integer-only decode of section 3.3); widening to fp32 and multiplying by
-// 2^(E-109) (one factor while it is a normal fp32 number, two exact power-of-two factors above that) gives
-// m * 2^(E-133) exactly (fp32 subnormals and overflow to Inf included); its upper 16 bits are the BF16 value.
-// The sign rides along, so m = 0 keeps its sign.
+// The byte s<<7|m is first spread to the 16-bit pattern s<<15|m (the integer-only decode of section 3.3).
+// Common exponents (every result a normal BF16 number, no overflow): 0x4300|m is the BF16 number 128 + m, and one
+// packed BF16 fused multiply-add (128 + m) * 2^(E-133) - 2^(E-126) leaves m * 2^(E-133) exactly, two elements at a
+// time; the sign bit is put back with one logic instruction, so m = 0 keeps its sign.
+// Other exponents: the pattern is the FP16 subnormal +-m * 2^-24; widening to fp32 and multiplying by 2^(E-109) (one
+// factor while it is a normal fp32 number, two exact power-of-two factors above that) gives m * 2^(E-133) exactly
+// (fp32 subnormals and overflow to Inf included); its upper 16 bits are the BF16 value.
 __device__ __forceinline__ uint2 dequant4(uint32_t w, uint32_t E)
 {
     uint32_t h01, h23;
     asm("prmt.b32 %0, %1, 0, 0x1100;" : "=r"(h01) : "r"(w));
     asm("prmt.b32 %0, %1, 0, 0x3322;" : "=r"(h23) : "r"(w));
+    if (E - 20u <= 216u) {
+        const uint32_t sc = (E - 6u) * 0x00800080u;           // 2^(E-133) in both halves
+        const uint32_t off = sc + 0x83808380u;                // -2^(E-126) in both halves
+        uint32_t r01, r23;
+        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r01) : "r"((h01 & 0x007F007Fu) | 0x43004300u), "r"(sc), "r"(off));
+        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r23) : "r"((h23 & 0x007F007Fu) | 0x43004300u), "r"(sc), "r"(off));
+        return make_uint2(r01 | (h01 & 0x80008000u), r23 | (h23 & 0x80008000u));
+    }
     h01 &= 0x807F807Fu;
     h23 &= 0x807F807Fu;
     const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&h01));
@@ -136,14 +146,17 @@ __global__ void __launch_bounds__(128) dequant_paged_kernel(CacheView cv, int wh
 }
 
 // ---------------------------------------------------------------- the streaming rebuild of BFP8 pages
-// A few long-lived CTAs per SM walk all (layer, page, kv head) records of the request: each 4352-byte record arrives by
-// one bulk async copy into a four-deep ring; 256 threads rebuild it (K: one thread = 8 channels of a token, one 16-byte
-// store; V: a word of the record holds four tokens of one channel, so one thread takes four channels of two tokens,
-// transposes the bytes in registers and writes two 8-byte pieces); every store instruction of a warp covers whole
-// 256-byte output rows.  Bit-exact like the kernel above (same dequant4).
-constexpr int kRebuildStages = 4;
-constexpr int kRebuildThreads = 256;
+// One CTA per SM, sixteen warps, and every warp is a worker of its own: it walks (layer, page, kv head) records with a
+// private three-deep ring of 4352-byte slots that it feeds itself (one bulk async copy per record, one mbarrier per
+// slot), so no CTA-wide barrier sits between a record's arrival and its stores.  K: a lane takes 8 channels of a token
+// (two words of the record, one exponent) and stores 16 bytes, a warp's store covering two whole 256-byte rows.
+// V: a word of the record holds four tokens of one channel, so a lane takes four channels, transposes the bytes in
+// registers and writes an 8-byte piece for each of the four tokens.  Bit-exact like the kernels above (same dequant4).
+constexpr int kRebuildWarps = 16;
+constexpr int kRebuildDepth = 3;
+constexpr int kRebuildThreads = kRebuildWarps * 32;
 constexpr uint32_t kRebuildSpin = 1u << 22;
+constexpr int kRebuildSmem = kRebuildWarps * kRebuildDepth * (kBfp8Record + 8);
 
 struct RebuildArgs {
     void *const *layers;          // device array of layer pointers (NULL: cv.layer is the only layer)
@@ -168,71 +181,86 @@ __device__ __forceinline__ bool rb_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-__global__ void __launch_bounds__(kRebuildThreads) rebuild_stream_kernel(CacheView cv, RebuildArgs a)
+__global__ void __launch_bounds__(kRebuildThreads, 1) rebuild_stream_kernel(CacheView cv, RebuildArgs a)
 {
-    __shared__ __align__(128) uint8_t ring[kRebuildStages][kBfp8Record];
-    __shared__ __align__(8) uint64_t bars[kRebuildStages];
-    __shared__ int ok_stage[kRebuildStages];
-    const int tid = threadIdx.x, Hkv = cv.num_kv_heads;
-    const int64_t n_items = (int64_t)a.n_layers * a.n_pages * Hkv;      // item = (layer, page, head), head fastest
-    if (tid == 0) {
-        for (int s = 0; s < kRebuildStages; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(rb_smem_u32(bars + s)));
+    extern __shared__ __align__(128) uint8_t rb_smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *ring = rb_smem + (size_t)warp * kRebuildDepth * kBfp8Record;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(rb_smem + (size_t)kRebuildWarps * kRebuildDepth * kBfp8Record) + warp * kRebuildDepth;
+    const uint32_t Hkv = (uint32_t)cv.num_kv_heads, n_pages = (uint32_t)a.n_pages;
+    const uint32_t n_items = (uint32_t)a.n_layers * n_pages * Hkv;       // item = (layer, page, head), head fastest (the launcher keeps it below 2^31)
+    const uint32_t n_workers = gridDim.x * kRebuildWarps;
+    const uint32_t first = blockIdx.x * kRebuildWarps + warp;            // neighbouring warps take neighbouring heads: together they complete output rows
+    if (lane == 0) {
+        for (int s = 0; s < kRebuildDepth; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(rb_smem_u32(bars + s)));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    __syncthreads();
-    auto load = [&](int64_t item, int stage) {      // thread 0 only
-        const int h = (int)(item % Hkv);
-        const int64_t lp = item / Hkv;
-        const int pg = (int)(lp % a.n_pages), l = (int)(lp / a.n_pages);
+    __syncwarp();
+    // the whole record, or only the half that is wanted
+    const int off = a.out_k ? 0 : kBfp8Half, bytes = (a.out_k && a.out_v) ? kBfp8Record : kBfp8Half;
+    auto split = [&](uint32_t item, uint32_t &l, uint32_t &pg, uint32_t &h) {
+        const uint32_t lp = item / Hkv;
+        h = item - lp * Hkv;
+        l = lp / n_pages;
+        pg = lp - l * n_pages;
+    };
+    auto load = [&](uint32_t item, int slot) {      // lane 0 only
+        uint32_t l, pg, h;
+        split(item, l, pg, h);
         const int32_t pid = a.page_ids[pg];
-        const uint32_t bar = rb_smem_u32(bars + stage);
-        if (pid < 0 || pid >= cv.num_pages) {
-            ok_stage[stage] = 0;
-            atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_DEQUANT);
+        const uint32_t bar = rb_smem_u32(bars + slot);
+        if (pid < 0 || pid >= cv.num_pages) {       // nothing to fetch: the consumer sees the same page id and writes zeros
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
             return;
         }
-        ok_stage[stage] = 1;
         const uint8_t *base = a.layers ? (const uint8_t *)a.layers[l] : cv.layer;
-        // the whole record, or only the half that is wanted
-        const int off = a.out_k ? 0 : kBfp8Half, bytes = (a.out_k && a.out_v) ? kBfp8Record : kBfp8Half;
         const uint8_t *src = base + ((int64_t)pid * Hkv + h) * (int64_t)kBfp8Record + off;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(rb_smem_u32(ring[stage]) + off),
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         rb_smem_u32(ring + slot * kBfp8Record) + off),
                      "l"(src), "r"(bytes), "r"(bar)
                      : "memory");
     };
-    if (tid == 0)
-        for (int s = 0; s < kRebuildStages; ++s) {
-            const int64_t item = blockIdx.x + (int64_t)s * gridDim.x;
-            if (item < n_items) load(item, s);
+    if (lane == 0)
+        for (int s = 0; s < kRebuildDepth; ++s) {
+            const uint64_t item = first + (uint64_t)s * n_workers;
+            if (item < n_items) load((uint32_t)item, s);
         }
     const bool relayout = cv.key_layout == HMA_KEYS_INTERLEAVED;
     const int64_t first_page = a.token_begin / kPageTokens;
-    int n = 0;
+    const int64_t row_elems = (int64_t)Hkv * kHeadDim;
+    int slot = 0;
+    uint32_t parity = 0;
     bool gave_up = false;
-    for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-        const int stage = n % kRebuildStages;
+    for (uint64_t it64 = first; it64 < n_items; it64 += n_workers) {
+        const uint32_t item = (uint32_t)it64;
         {
-            const uint32_t bar = rb_smem_u32(bars + stage), parity = (n / kRebuildStages) & 1;
-            uint32_t it = 0;
+            const uint32_t bar = rb_smem_u32(bars + slot);
+            uint32_t spins = 0;
             bool here = rb_try_wait(bar, parity);
-            while (!here && ++it < kRebuildSpin) here = rb_try_wait(bar, parity);
-            gave_up = __syncthreads_or(!here);
+            while (!here && ++spins < kRebuildSpin) here = rb_try_wait(bar, parity);
+            gave_up = __any_sync(0xFFFFFFFFu, !here);
         }
         if (gave_up) break;
-        const int h = (int)(item % Hkv);
-        const int64_t lp = item / Hkv;
-        const int pg = (int)(lp % a.n_pages), l = (int)(lp / a.n_pages);
-        const bool ok = ok_stage[stage] != 0;
-        const uint8_t *rec = ring[stage];
-        const int64_t page_tok0 = (first_page + pg) * kPageTokens;            // request token of the page's first slot
+        uint32_t l, pg, h;
+        split(item, l, pg, h);
+        const int32_t pid = a.page_ids[pg];
+        const bool ok = pid >= 0 && pid < cv.num_pages;
+        if (!ok && lane == 0) atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_DEQUANT);
+        const uint8_t *rec = ring + slot * kBfp8Record;
+        // tokens [t_lo, t_hi) of this page belong to the request; rel = request row of the page's first slot
+        const int64_t rel = (first_page + pg) * kPageTokens - a.token_begin;
+        const int t_lo = rel < 0 ? (int)-rel : 0;
+        const int t_hi = (a.n_tokens - rel) < kPageTokens ? (int)(a.n_tokens - rel) : kPageTokens;
+        const int64_t base_el = (int64_t)l * a.layer_stride + rel * row_elems + (int64_t)h * kHeadDim;
         if (a.out_k) {
-            // K: lane = 8-channel group + 16 * (token & 1), warp = token >> 1: a warp's store covers two whole rows
-            const int tok = 2 * (tid >> 5) + ((tid >> 4) & 1), c0 = (tid & 15) * 8;
-            const int64_t gt = page_tok0 + tok;
-            if (gt >= a.token_begin && gt < a.token_begin + a.n_tokens) {
+            uint16_t *out0 = a.out_k + base_el;
+            const int c0 = (lane & 15) * 8;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                // lane = 8-channel group + 16 * (token & 1): a warp's store covers two whole rows
+                const int tok = 2 * i + (lane >> 4);
                 uint2 lo = make_uint2(0u, 0u), hi = lo;
                 if (ok) {
                     const uint32_t E = rec[bfp8_k_exp_off(tok, c0 >> 4)];
@@ -240,7 +268,8 @@ __global__ void __launch_bounds__(kRebuildThreads) rebuild_stream_kernel(CacheVi
                     lo = dequant4(*reinterpret_cast<const uint32_t *>(p), E);
                     hi = dequant4(*reinterpret_cast<const uint32_t *>(p + 16), E);
                 }
-                uint16_t *row = a.out_k + (int64_t)l * a.layer_stride + ((gt - a.token_begin) * Hkv + h) * kHeadDim;
+                if (tok < t_lo || tok >= t_hi) continue;
+                uint16_t *row = out0 + tok * row_elems;
                 if (relayout) {
                     // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout)
                     __stcs(reinterpret_cast<uint2 *>(row + (c0 >> 1)), make_uint2((lo.x & 0xFFFFu) | (lo.y << 16), (hi.x & 0xFFFFu) | (hi.y << 16)));
@@ -251,45 +280,51 @@ __global__ void __launch_bounds__(kRebuildThreads) rebuild_stream_kernel(CacheVi
             }
         }
         if (a.out_v) {
-            // V: a thread takes channels ch0 .. ch0+3 of tokens 2tq + 8*th and 2tq + 8*th + 1.  Lanes differ in tq and in
-            // which quad of a 32-channel span they hold (two-way bank conflicts at most; every store covers whole
-            // 64-byte pieces of output rows); warps differ in the span and in th.
-            const int lane = tid & 31, tq = lane & 3, th = tid >> 7;
-            const int j = 2 * ((tid >> 5) & 3) + ((lane >> 2) & 1), cb0 = 8 * ((lane >> 3) & 1) + 4 * (lane >> 4), ch0 = 16 * j + cb0;
+            // V: a lane takes channels ch0 .. ch0+3 of tokens 2tq, 2tq+1, 2tq+8, 2tq+9 (the four bytes of its words).
+            // Lanes differ in tq and in which quad of a 32-channel span they hold (two-way bank conflicts at most; every
+            // store instruction covers whole 64-byte pieces of four output rows); the loop walks the four spans.
+            uint16_t *out0 = a.out_v + base_el;
+            const int tq = lane & 3;
             const uint8_t *vb = rec + kBfp8Half;
-            uint32_t w[4] = {0u, 0u, 0u, 0u}, e2 = 0u;
-            if (ok) {
-                const uint8_t *p = vb + 128 + (j >> 1) * 512 + ((cb0 & 7) * 4 + tq) * 16 + ((j & 1) * 2 + (cb0 >> 3)) * 4;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) w[i] = *reinterpret_cast<const uint32_t *>(p + 64 * i);       // channel ch0 + i, four tokens
-                e2 = *reinterpret_cast<const uint32_t *>(vb + tq * 32 + j * 4);                           // exponents of the four tokens, block j
-            }
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = 2 * jj + ((lane >> 2) & 1), cb0 = 8 * ((lane >> 3) & 1) + 4 * (lane >> 4), ch0 = 16 * j + cb0;
+                uint32_t w[4] = {0u, 0u, 0u, 0u}, e4 = 0u;
+                if (ok) {
+                    const uint8_t *p = vb + 128 + (j >> 1) * 512 + ((cb0 & 7) * 4 + tq) * 16 + ((j & 1) * 2 + (cb0 >> 3)) * 4;
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                const int k = 2 * th + t, tok = 2 * tq + t + 8 * th;
-                const int64_t gt = page_tok0 + tok;
-                if (gt < a.token_begin || gt >= a.token_begin + a.n_tokens) continue;
-                // byte k of the four words = channels ch0 .. ch0+3 of this token
-                const uint32_t sel = (uint32_t)k | ((uint32_t)(4 + k) << 4);
-                const uint32_t word = __byte_perm(__byte_perm(w[0], w[1], sel), __byte_perm(w[2], w[3], sel), 0x5410u);
-                const uint2 r = ok ? dequant4(word, (e2 >> (8 * k)) & 0xFFu) : make_uint2(0u, 0u);
-                uint16_t *row = a.out_v + (int64_t)l * a.layer_stride + ((gt - a.token_begin) * Hkv + h) * kHeadDim;
-                __stcs(reinterpret_cast<uint2 *>(row + ch0), r);
+                    for (int i = 0; i < 4; ++i) w[i] = *reinterpret_cast<const uint32_t *>(p + 64 * i);       // channel ch0 + i, four tokens
+                    e4 = *reinterpret_cast<const uint32_t *>(vb + tq * 32 + j * 4);                           // exponents of the four tokens, block j
+                }
+                // byte k of the four words = channels ch0 .. ch0+3 of token 2tq + (k & 1) + 8 (k >> 1)
+                const uint32_t a01 = __byte_perm(w[0], w[1], 0x5140u), a23 = __byte_perm(w[2], w[3], 0x5140u);   // bytes 0 and 1 of each word
+                const uint32_t b01 = __byte_perm(w[0], w[1], 0x7362u), b23 = __byte_perm(w[2], w[3], 0x7362u);   // bytes 2 and 3
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int tok = 2 * tq + (k & 1) + 8 * (k >> 1);
+                    const uint32_t lo2 = k < 2 ? a01 : b01, hi2 = k < 2 ? a23 : b23;
+                    const uint32_t word = __byte_perm(lo2, hi2, (k & 1) ? 0x7632u : 0x5410u);
+                    const uint2 r = ok ? dequant4(word, (e4 >> (8 * k)) & 0xFFu) : make_uint2(0u, 0u);
+                    if (tok < t_lo || tok >= t_hi) continue;
+                    __stcs(reinterpret_cast<uint2 *>(out0 + tok * row_elems + ch0), r);
+                }
             }
         }
-        __syncthreads();                               // everybody is done with the slot
-        if (tid == 0) {
-            const int64_t next = item + (int64_t)kRebuildStages * gridDim.x;
+        __syncwarp();                                  // every lane is done with the slot
+        if (lane == 0) {
+            const uint64_t next = it64 + (uint64_t)kRebuildDepth * n_workers;
             if (next < n_items) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                load(next, stage);
+                load((uint32_t)next, slot);
             }
         }
+        if (++slot == kRebuildDepth) { slot = 0; parity ^= 1u; }
     }
-    if (tid == 0 && gave_up) {
+    if (gave_up && lane == 0) {
         atomicOr(cv.flags, HMA_FLAG_WAIT_TIMEOUT);
-        for (int s = 0; s < kRebuildStages; ++s)
-            for (uint32_t it = 0; it < (1u << 16) && !rb_try_wait(rb_smem_u32(bars + s), 0) && !rb_try_wait(rb_smem_u32(bars + s), 1); ++it) {}
+        // copies still in flight target this CTA's shared memory: give them a bounded time to land before leaving
+        for (int s = 0; s < kRebuildDepth; ++s)
+            for (uint32_t spins = 0; spins < (1u << 16) && !rb_try_wait(rb_smem_u32(bars + s), 0) && !rb_try_wait(rb_smem_u32(bars + s), 1); ++spins) {}
     }
 }
 
@@ -327,12 +362,11 @@ static hma_status_t launch_rebuild(const hma::CacheView &cv, const hma::RebuildA
     HMA_CUDA_OK(cudaGetDevice(&dev));
     HMA_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     const int64_t items = (int64_t)a.n_layers * a.n_pages * cv.num_kv_heads;
-    // one wave of CTAs: as many as are resident at once, each walking its share of the records
-    int per_sm = 0;
-    HMA_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, hma::rebuild_stream_kernel, hma::kRebuildThreads, 0));
-    if (per_sm < 1) per_sm = 1;
-    const int64_t cap = (int64_t)n_sm * per_sm;
-    hma::rebuild_stream_kernel<<<(unsigned)(items < cap ? items : cap), hma::kRebuildThreads, 0, (cudaStream_t)stream>>>(cv, a);
+    if (items > 0x7FFFFFFF) return HMA_ERR_INVALID_ARG;
+    HMA_CUDA_OK(cudaFuncSetAttribute(hma::rebuild_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hma::kRebuildSmem));
+    // one CTA per SM at most, every warp walking its share of the records
+    const int64_t want = (items + hma::kRebuildWarps - 1) / hma::kRebuildWarps;
+    hma::rebuild_stream_kernel<<<(unsigned)(want < n_sm ? want : n_sm), hma::kRebuildThreads, hma::kRebuildSmem, (cudaStream_t)stream>>>(cv, a);
     hma::count_launch();
     HMA_CUDA_OK(cudaGetLastError());
     return HMA_OK;
