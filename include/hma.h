@@ -126,7 +126,8 @@ void hma_cache_destroy(hma_cache_t *cache);
  *                     face*16 + row%16, elements at 64 + face*256 + (row%16)*16 + col%16.
  *                   HMA_WIRE_BF16_ROWS (BF16 caches only): [head][token][128] plain BF16 values, KV that was
  *                     made on the decode GPU itself (the paper keeps decode in BF16, section 3.1).
- *                   Both pointers 16-byte aligned.
+ *                   Both pointers 16-byte aligned (HMA_WIRE_ROWMAJOR: 8-byte aligned is enough, which is
+ *                   what hma_bfp8_encode_rows asks of its output).
  *   page_ids        device int32: page_ids[i] = physical page of the request's logical page
  *                   floor(token_begin/16) + i; ceil((token_begin%16 + n_tokens)/16) entries.
  * Token slots outside the range, other heads and other pages keep their bytes.  Pages being
@@ -203,7 +204,7 @@ hma_status_t hma_decode_attention_multi(const hma_cache_t *cache, int32_t layer,
  * hma_decode_attention for callers that cannot allocate.  (The paper has no counterpart: this exists for
  * the way the library gets embedded, not for the method.)  A decode loop that fixed its memory pool at
  * start-up, or code running where the host framework forbids allocation, has no workspace to pass; here
- * the scratch is a 5.1 MiB array that is part of the library image on every GPU that loads it
+ * the scratch is a 5.8 MiB array that is part of the library image on every GPU that loads it
  * (hma_decode_attention_static_limit_bytes returns the exact size).  The call allocates and frees nothing.
  *
  *   - same arguments and results as hma_decode_attention, without the workspace pair; the outputs of the

@@ -1495,7 +1495,9 @@ extern "C" hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_
 // below until the process exits.
 namespace hma {
 constexpr int kStaticMaxSegments = 512;       // batch * num_kv_heads
-constexpr size_t kStaticWsBytes = (size_t)kMaxBatch * kMaxKvHeads * 4 + 8192 + (size_t)(kMaxCtas + 2 * kStaticMaxSegments) * kTileFloats * 4;   // 5.1 MiB
+// counters | cum for up to 1000 rows | the per-CTA tiles and tail tiles of kStaticMaxSegments segments (the same sum as
+// hma_decode_attention_workspace_bytes)
+constexpr size_t kStaticWsBytes = (size_t)kMaxBatch * kMaxKvHeads * 4 + 8192 + (size_t)(2 * kMaxCtas + 2 * kStaticMaxSegments) * kTileFloats * 4;   // 5.8 MiB
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 static void *g_static_ws_ptr[kMaxDevices];    // device address of g_static_ws on each device, resolved on first use
 }  // namespace hma

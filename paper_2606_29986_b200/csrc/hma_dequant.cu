@@ -13,18 +13,27 @@ namespace hma {
 // Other exponents: the pattern is the FP16 subnormal +-m * 2^-24; widening to fp32 and multiplying by 2^(E-109) (one
 // factor while it is a normal fp32 number, two exact power-of-two factors above that) gives m * 2^(E-133) exactly
 // (fp32 subnormals and overflow to Inf included); its upper 16 bits are the BF16 value.
+// exponents for which the packed BF16 path below is exact: every result a normal BF16 number, no overflow
+__device__ __forceinline__ bool bf16_path_ok(uint32_t E) { return E - 20u <= 216u; }
+// 2^(E-133) in both halves of a BF16 pair
+__device__ __forceinline__ uint32_t bf16_scale2(uint32_t E) { return (E - 6u) * 0x00800080u; }
+// two elements whose bytes were spread to the halfwords b<<8|b -> two BF16 values (bf16_path_ok exponents only)
+__device__ __forceinline__ uint32_t dequant2_bf16(uint32_t h, uint32_t sc)
+{
+    uint32_t r;
+    const uint32_t off = sc + 0x83808380u;                    // -2^(E-126) in both halves
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"((h & 0x007F007Fu) | 0x43004300u), "r"(sc), "r"(off));
+    return r | (h & 0x80008000u);
+}
+
 __device__ __forceinline__ uint2 dequant4(uint32_t w, uint32_t E)
 {
     uint32_t h01, h23;
     asm("prmt.b32 %0, %1, 0, 0x1100;" : "=r"(h01) : "r"(w));
     asm("prmt.b32 %0, %1, 0, 0x3322;" : "=r"(h23) : "r"(w));
-    if (E - 20u <= 216u) {
-        const uint32_t sc = (E - 6u) * 0x00800080u;           // 2^(E-133) in both halves
-        const uint32_t off = sc + 0x83808380u;                // -2^(E-126) in both halves
-        uint32_t r01, r23;
-        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r01) : "r"((h01 & 0x007F007Fu) | 0x43004300u), "r"(sc), "r"(off));
-        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r23) : "r"((h23 & 0x007F007Fu) | 0x43004300u), "r"(sc), "r"(off));
-        return make_uint2(r01 | (h01 & 0x80008000u), r23 | (h23 & 0x80008000u));
+    if (bf16_path_ok(E)) {
+        const uint32_t sc = bf16_scale2(E);
+        return make_uint2(dequant2_bf16(h01, sc), dequant2_bf16(h23, sc));
     }
     h01 &= 0x807F807Fu;
     h23 &= 0x807F807Fu;
@@ -181,6 +190,84 @@ __device__ __forceinline__ bool rb_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// One record -> its K and V rows.  kPlain: a good page, all sixteen tokens wanted, every exponent takes the packed
+// BF16 path (the caller checked); otherwise bad pages give zeros, tokens outside [t_lo, t_hi) are skipped and every
+// block picks its decode by its exponent.
+template <bool kPlain>
+__device__ __forceinline__ void rebuild_record(const RebuildArgs &a, const uint8_t *rec, bool relayout, int64_t base_el,
+                                               int64_t row_elems, int lane, bool ok, int t_lo, int t_hi)
+{
+    if (a.out_k) {
+        uint16_t *out0 = a.out_k + base_el;
+        const int c0 = (lane & 15) * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            // lane = 8-channel group + 16 * (token & 1): a warp's store covers two whole rows
+            const int tok = 2 * i + (lane >> 4);
+            uint2 lo = make_uint2(0u, 0u), hi = lo;
+            if (kPlain || ok) {
+                const uint32_t E = rec[bfp8_k_exp_off(tok, c0 >> 4)];
+                const uint8_t *p = rec + bfp8_k_el_off(tok, c0);
+                const uint32_t w0 = *reinterpret_cast<const uint32_t *>(p), w1 = *reinterpret_cast<const uint32_t *>(p + 16);
+                if (kPlain) {
+                    const uint32_t sc = bf16_scale2(E);
+                    lo = make_uint2(dequant2_bf16(__byte_perm(w0, 0u, 0x1100u), sc), dequant2_bf16(__byte_perm(w0, 0u, 0x3322u), sc));
+                    hi = make_uint2(dequant2_bf16(__byte_perm(w1, 0u, 0x1100u), sc), dequant2_bf16(__byte_perm(w1, 0u, 0x3322u), sc));
+                } else {
+                    lo = dequant4(w0, E);
+                    hi = dequant4(w1, E);
+                }
+            }
+            if (!kPlain && (tok < t_lo || tok >= t_hi)) continue;
+            uint16_t *row = out0 + tok * row_elems;
+            if (relayout) {
+                // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout)
+                __stcs(reinterpret_cast<uint2 *>(row + (c0 >> 1)), make_uint2((lo.x & 0xFFFFu) | (lo.y << 16), (hi.x & 0xFFFFu) | (hi.y << 16)));
+                __stcs(reinterpret_cast<uint2 *>(row + 64 + (c0 >> 1)), make_uint2((lo.x >> 16) | (lo.y & 0xFFFF0000u), (hi.x >> 16) | (hi.y & 0xFFFF0000u)));
+            } else {
+                __stcs(reinterpret_cast<uint4 *>(row + c0), make_uint4(lo.x, lo.y, hi.x, hi.y));      // streaming: written once, read by somebody else
+            }
+        }
+    }
+    if (a.out_v) {
+        // V: a lane takes channels ch0 .. ch0+3 of tokens 2tq, 2tq+1, 2tq+8, 2tq+9 (the four bytes of its words).
+        // Lanes differ in tq and in which quad of a 32-channel span they hold (two-way bank conflicts at most; every
+        // store instruction covers whole 64-byte pieces of four output rows); the loop walks the four spans.
+        uint16_t *out0 = a.out_v + base_el;
+        const int tq = lane & 3;
+        const uint8_t *vb = rec + kBfp8Half;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const int j = 2 * jj + ((lane >> 2) & 1), cb0 = 8 * ((lane >> 3) & 1) + 4 * (lane >> 4), ch0 = 16 * j + cb0;
+            uint32_t w[4] = {0u, 0u, 0u, 0u}, e4 = 0u;
+            if (kPlain || ok) {
+                const uint8_t *p = vb + 128 + (j >> 1) * 512 + ((cb0 & 7) * 4 + tq) * 16 + ((j & 1) * 2 + (cb0 >> 3)) * 4;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) w[i] = *reinterpret_cast<const uint32_t *>(p + 64 * i);       // channel ch0 + i, four tokens
+                e4 = *reinterpret_cast<const uint32_t *>(vb + tq * 32 + j * 4);                           // exponents of the four tokens, block j
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                // byte k of the four words = channels ch0 .. ch0+3 of token 2tq + (k & 1) + 8 (k >> 1); one byte
+                // permutation per channel pair picks the two bytes and spreads each over a halfword
+                const int tok = 2 * tq + (k & 1) + 8 * (k >> 1);
+                const uint32_t sel = (uint32_t)(k | (k << 4) | ((4 + k) << 8) | ((4 + k) << 12));
+                const uint32_t h01 = __byte_perm(w[0], w[1], sel), h23 = __byte_perm(w[2], w[3], sel);
+                const uint32_t E = (e4 >> (8 * k)) & 0xFFu;
+                uint2 r = make_uint2(0u, 0u);
+                if (kPlain) {
+                    const uint32_t sc = bf16_scale2(E);
+                    r = make_uint2(dequant2_bf16(h01, sc), dequant2_bf16(h23, sc));
+                } else if (ok) {
+                    r = dequant4(__byte_perm(h01, h23, 0x6420u), E);
+                }
+                if (!kPlain && (tok < t_lo || tok >= t_hi)) continue;
+                __stcs(reinterpret_cast<uint2 *>(out0 + tok * row_elems + ch0), r);
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kRebuildThreads, 1) rebuild_stream_kernel(CacheView cv, RebuildArgs a)
 {
     extern __shared__ __align__(128) uint8_t rb_smem[];
@@ -254,62 +341,25 @@ __global__ void __launch_bounds__(kRebuildThreads, 1) rebuild_stream_kernel(Cach
         const int t_lo = rel < 0 ? (int)-rel : 0;
         const int t_hi = (a.n_tokens - rel) < kPageTokens ? (int)(a.n_tokens - rel) : kPageTokens;
         const int64_t base_el = (int64_t)l * a.layer_stride + rel * row_elems + (int64_t)h * kHeadDim;
-        if (a.out_k) {
-            uint16_t *out0 = a.out_k + base_el;
-            const int c0 = (lane & 15) * 8;
+        // The common case (a good page, all sixteen tokens wanted, every exponent in the range of the packed BF16
+        // path) runs without a single test per element; anything else takes the general path.
+        bool plain = ok && t_lo == 0 && t_hi == kPageTokens;
+        if (plain) {
+            bool in_range = true;
+            if (a.out_k) {
+                const uint32_t e = *reinterpret_cast<const uint32_t *>(rec + 4 * lane);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                // lane = 8-channel group + 16 * (token & 1): a warp's store covers two whole rows
-                const int tok = 2 * i + (lane >> 4);
-                uint2 lo = make_uint2(0u, 0u), hi = lo;
-                if (ok) {
-                    const uint32_t E = rec[bfp8_k_exp_off(tok, c0 >> 4)];
-                    const uint8_t *p = rec + bfp8_k_el_off(tok, c0);
-                    lo = dequant4(*reinterpret_cast<const uint32_t *>(p), E);
-                    hi = dequant4(*reinterpret_cast<const uint32_t *>(p + 16), E);
-                }
-                if (tok < t_lo || tok >= t_hi) continue;
-                uint16_t *row = out0 + tok * row_elems;
-                if (relayout) {
-                    // keys cached with rotary pairs interleaved leave in half-split order (section 3.3, key re-layout)
-                    __stcs(reinterpret_cast<uint2 *>(row + (c0 >> 1)), make_uint2((lo.x & 0xFFFFu) | (lo.y << 16), (hi.x & 0xFFFFu) | (hi.y << 16)));
-                    __stcs(reinterpret_cast<uint2 *>(row + 64 + (c0 >> 1)), make_uint2((lo.x >> 16) | (lo.y & 0xFFFF0000u), (hi.x >> 16) | (hi.y & 0xFFFF0000u)));
-                } else {
-                    __stcs(reinterpret_cast<uint4 *>(row + c0), make_uint4(lo.x, lo.y, hi.x, hi.y));      // streaming: written once, read by somebody else
-                }
+                for (int i = 0; i < 4; ++i) in_range &= bf16_path_ok((e >> (8 * i)) & 0xFFu);
             }
-        }
-        if (a.out_v) {
-            // V: a lane takes channels ch0 .. ch0+3 of tokens 2tq, 2tq+1, 2tq+8, 2tq+9 (the four bytes of its words).
-            // Lanes differ in tq and in which quad of a 32-channel span they hold (two-way bank conflicts at most; every
-            // store instruction covers whole 64-byte pieces of four output rows); the loop walks the four spans.
-            uint16_t *out0 = a.out_v + base_el;
-            const int tq = lane & 3;
-            const uint8_t *vb = rec + kBfp8Half;
+            if (a.out_v) {
+                const uint32_t e = *reinterpret_cast<const uint32_t *>(rec + kBfp8Half + 4 * lane);
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-                const int j = 2 * jj + ((lane >> 2) & 1), cb0 = 8 * ((lane >> 3) & 1) + 4 * (lane >> 4), ch0 = 16 * j + cb0;
-                uint32_t w[4] = {0u, 0u, 0u, 0u}, e4 = 0u;
-                if (ok) {
-                    const uint8_t *p = vb + 128 + (j >> 1) * 512 + ((cb0 & 7) * 4 + tq) * 16 + ((j & 1) * 2 + (cb0 >> 3)) * 4;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) w[i] = *reinterpret_cast<const uint32_t *>(p + 64 * i);       // channel ch0 + i, four tokens
-                    e4 = *reinterpret_cast<const uint32_t *>(vb + tq * 32 + j * 4);                           // exponents of the four tokens, block j
-                }
-                // byte k of the four words = channels ch0 .. ch0+3 of token 2tq + (k & 1) + 8 (k >> 1)
-                const uint32_t a01 = __byte_perm(w[0], w[1], 0x5140u), a23 = __byte_perm(w[2], w[3], 0x5140u);   // bytes 0 and 1 of each word
-                const uint32_t b01 = __byte_perm(w[0], w[1], 0x7362u), b23 = __byte_perm(w[2], w[3], 0x7362u);   // bytes 2 and 3
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int tok = 2 * tq + (k & 1) + 8 * (k >> 1);
-                    const uint32_t lo2 = k < 2 ? a01 : b01, hi2 = k < 2 ? a23 : b23;
-                    const uint32_t word = __byte_perm(lo2, hi2, (k & 1) ? 0x7632u : 0x5410u);
-                    const uint2 r = ok ? dequant4(word, (e4 >> (8 * k)) & 0xFFu) : make_uint2(0u, 0u);
-                    if (tok < t_lo || tok >= t_hi) continue;
-                    __stcs(reinterpret_cast<uint2 *>(out0 + tok * row_elems + ch0), r);
-                }
+                for (int i = 0; i < 4; ++i) in_range &= bf16_path_ok((e >> (8 * i)) & 0xFFu);
             }
+            plain = __all_sync(0xFFFFFFFFu, in_range);
         }
+        if (plain) rebuild_record<true>(a, rec, relayout, base_el, row_elems, lane, true, 0, kPageTokens);
+        else rebuild_record<false>(a, rec, relayout, base_el, row_elems, lane, ok, t_lo, t_hi);
         __syncwarp();                                  // every lane is done with the slot
         if (lane == 0) {
             const uint64_t next = it64 + (uint64_t)kRebuildDepth * n_workers;

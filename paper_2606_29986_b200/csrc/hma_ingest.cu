@@ -408,7 +408,9 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
     if (!page_ids) return HMA_ERR_INVALID_ARG;
     for (int s = 0; s < n_shards; ++s) {
         if (!a.k_wire[s] || !a.v_wire[s]) return HMA_ERR_INVALID_ARG;
-        if (((uintptr_t)a.k_wire[s] & 15u) || ((uintptr_t)a.v_wire[s] & 15u)) return HMA_ERR_ALIGNMENT;
+        // 136-byte rows are read in 8-byte pieces (what hma_bfp8_encode_rows promises for its output); tiles and BF16 rows in 16-byte pieces
+        const uintptr_t need = wire_layout == HMA_WIRE_ROWMAJOR ? 7u : 15u;
+        if (((uintptr_t)a.k_wire[s] & need) || ((uintptr_t)a.v_wire[s] & need)) return HMA_ERR_ALIGNMENT;
     }
     const int64_t first = token_begin / hma::kPageTokens;
     const int64_t last = (token_begin + n_tokens - 1) / hma::kPageTokens;

@@ -190,6 +190,27 @@ def test_bfp8_cache_holds_the_wire_bytes_unchanged():
             assert np.array_equal(np.sort(rec[p, h]), np.sort(wire))
 
 
+def test_rowmajor_wire_needs_only_the_encoders_alignment():
+    """hma_bfp8_encode_rows promises 8-byte aligned rows; a wire that starts 8 bytes off a 16-byte boundary is ingested as it is."""
+    sc = Scenario([48], 8, 2, seed=21, layers=1)
+    pages = sc.table[0, :3].contiguous()
+    want = sc.cache.layers[0].clone()
+    sc.cache.layers[0].fill_(0xA5)                  # the constructor's fill: pages nobody writes keep it
+    kw, vw = sc.k_wires[0][0], sc.v_wires[0][0]
+    def shifted(w):
+        buf = torch.zeros(w.size + 16, dtype=torch.uint8, device="cuda")
+        assert buf.data_ptr() % 16 == 0
+        buf[8:8 + w.size] = torch.from_numpy(w.reshape(-1)).cuda()
+        return buf[8:8 + w.size]
+    hma.hma_kv_ingest_layer(sc.cache, 0, shifted(kw), shifted(vw), hma.HMA_WIRE_ROWMAJOR, 0, 2, pages, 0, 48)
+    torch.cuda.synchronize()
+    assert hma.hma_error_flags(sc.cache) == 0
+    assert torch.equal(sc.cache.layers[0], want)
+    with pytest.raises(hma.HmaError) as e:      # a tiled wire is moved in 16-byte pieces
+        hma.hma_kv_ingest_layer(sc.cache, 0, shifted(kw), shifted(vw), hma.HMA_WIRE_TILE32, 0, 2, pages, 0, 48)
+    assert e.value.status == hma.HMA_ERR_ALIGNMENT
+
+
 def test_bad_arguments_and_bad_page_ids():
     sc = Scenario([40], 8, 2, seed=7, layers=1)
     kw = torch.from_numpy(sc.k_wires[0][0]).cuda()

@@ -41,6 +41,15 @@ def test_static_scratch_matches_workspace_entry_point_twice():
     assert torch.equal(o32, r32)
 
 
+def test_static_scratch_takes_the_largest_batch_it_promises():
+    sc = Scenario([40 + 3 * i for i in range(64)], 16, 8, seed=104, permute=True)      # 64 sequences x 8 kv heads = 512 segments
+    ws = hma.hma_decode_attention_workspace_bytes(sc.cache.desc, 64)
+    assert ws <= hma.hma_decode_attention_static_limit_bytes() < ws + 2 * 8 * 4160       # 65 sequences would not fit
+    r32, o32 = _both(sc, torch.float32)
+    assert torch.equal(o32, r32)
+    assert hma.hma_error_flags(sc.cache) == 0
+
+
 def test_static_scratch_rejects_what_does_not_fit():
     assert hma.hma_decode_attention_static_limit_bytes() < 16 * 1024 * 1024
     lens = [16] * 80                                                # 80 sequences x 8 kv heads = 640 segments > 512
