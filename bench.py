@@ -272,6 +272,29 @@ class Workload:
                 g.replay()
             e1.record()
             torch.cuda.synchronize(self.device)
+            # the same harness around the plainest kernel with the same byte counts: one launch per layer that reads the
+            # layer's wire bytes and writes as many to a buffer of its own
+            dst = torch.empty_like(self.wire_dev)
+            nbytes = self.wire_dev[0].numel()
+
+            def copies():
+                for l in range(self.L):
+                    self.hma.hma_hbm_copy_probe(self.wire_dev[l], nbytes, dst[l], nbytes, s)
+            copies()
+            torch.cuda.synchronize(self.device)
+            gc = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gc, stream=s):
+                copies()
+            gc.replay()
+            torch.cuda.synchronize(self.device)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            for _ in range(reps):
+                gc.replay()
+            c1.record()
+            torch.cuda.synchronize(self.device)
+            self.copy_probe_layer_s = c0.elapsed_time(c1) / 1e3 / reps / self.L
+            del dst
         torch.cuda.current_stream(self.device).wait_stream(s)
         return e0.elapsed_time(e1) / 1e3 / reps / self.L
 
@@ -371,6 +394,20 @@ class Workload:
         e1.record()
         torch.cuda.synchronize(self.device)
         self.naive_rebuild_s = e0.elapsed_time(e1) / 1e3
+        # the plainest kernel with the same byte counts: reads 17 bytes for every 32 it writes, from one layer's cache
+        src = cache.layers[0]
+        rd = min(int(elems * 17 // 16), src.numel()) // 16 * 16
+        wr_bytes = rd * 32 // 17 // 16 * 16
+        dst = out.view(-1)
+        self.hma.hma_hbm_copy_probe(src, rd, dst, wr_bytes)
+        torch.cuda.synchronize(self.device)
+        e0.record()
+        for _ in range(reps):
+            self.hma.hma_hbm_copy_probe(src, rd, dst, wr_bytes)
+        e1.record()
+        torch.cuda.synchronize(self.device)
+        # scaled to the rebuild's bytes when one layer's cache is smaller than what the rebuild reads
+        self.copy_probe_rebuild_s = e0.elapsed_time(e1) / 1e3 / reps * (elems * (17 / 16 + 2)) / (rd + wr_bytes)
         return fused, elems * (17 / 16 + 2), elems
 
 # ----------------------------------------------------------------------------- ranks
@@ -553,12 +590,16 @@ def main():
     extra["rebuild_request"] = {"ms": t_rb * 1e3, "tokens": int(wl.lens[0]), "layers": wl.L, "gbs": rb_bytes / t_rb / 1e9,
                                 "frac_of_peak": rb_bytes / t_rb / 1e9 / peak, "calls": 1,
                                 "naive_elementwise_ms": wl.naive_rebuild_s * 1e3, "fused_speedup_over_naive": wl.naive_rebuild_s / t_rb,
+                                "copy_probe_ms": wl.copy_probe_rebuild_s * 1e3, "frac_of_copy_probe": wl.copy_probe_rebuild_s / t_rb,
+                                "copy_probe": "hma_hbm_copy_probe: a plain streaming kernel that reads 17 bytes for every 32 it writes, same byte counts",
                                 "what": "hma_bfp8_rebuild_request: one request, K and V, all layers, one launch (1.0625 B in + 2 B out per element)"}
     if wl.ingest_tokens:
         t_ing = wl.time_ingest()
         layer_bytes = 2 * 4 * wl.shard_bytes
         extra["ingest_alone"] = {"us_per_layer": t_ing * 1e6, "gbs_read_plus_write": 2 * layer_bytes / t_ing / 1e9,
                                  "frac_of_peak": 2 * layer_bytes / t_ing / 1e9 / peak,
+                                 "copy_probe_us_per_layer": wl.copy_probe_layer_s * 1e6, "frac_of_copy_probe": wl.copy_probe_layer_s / t_ing,
+                                 "copy_probe": "hma_hbm_copy_probe in the same harness: one plain launch per layer that reads the layer's wire bytes and writes as many",
                                  "what": "hma_kv_ingest_layer_shards, one 8192-token layer (4 shards, TILE32), device-resident wire, CUDA-graph replay"}
     t_mixed = wl.time_mixed()
     extra["mixed_prefix_tail"] = {"us_per_call": t_mixed * 1e6, "tail_tokens_per_sequence": 64,

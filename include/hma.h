@@ -329,6 +329,12 @@ hma_status_t hma_attention_alu_probe(const hma_cache_t *cache, int32_t layer, co
  * the kernel may add to (it practically never does; it keeps the loads alive). */
 hma_status_t hma_hbm_read_probe(const void *src, size_t bytes, void *sink4, void *stream);
 
+/* A streaming read of read_bytes from `src` mixed with a streaming write of write_bytes to `dst` (both device,
+ * 16-byte aligned, read_bytes <= write_bytes; the written data is the source stretched to the output's length): the
+ * simplest kernel with the byte counts of a conversion that expands its input, for comparison with
+ * hma_bfp8_rebuild_request (17 bytes in for 32 out) and the ingest (1:1). */
+hma_status_t hma_hbm_copy_probe(const void *src, size_t read_bytes, void *dst, size_t write_bytes, void *stream);
+
 
 #ifdef HMA_TRACE
 /* Only in the instrumented build of the library (compiled with -DHMA_TRACE; the default build has neither this entry

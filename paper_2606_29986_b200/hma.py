@@ -79,6 +79,8 @@ def lib():
         L.hma_kv_read_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
         L.hma_hbm_read_probe.restype = i32
         L.hma_hbm_read_probe.argtypes = [vp, sz, vp, vp]
+        L.hma_hbm_copy_probe.restype = i32
+        L.hma_hbm_copy_probe.argtypes = [vp, sz, vp, sz, vp]
         L.hma_attention_alu_probe.restype = i32
         L.hma_attention_alu_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
         L.hma_decode_attention_mixed.restype = i32
@@ -253,6 +255,12 @@ def hma_attention_alu_probe(cache, layer, block_table, context_lens, workspace, 
 def hma_hbm_read_probe(src, sink, stream=None):
     """Contiguous streaming read of the whole tensor `src` (a read-only memory ceiling); `sink` is a 4-byte device tensor."""
     _check(lib().hma_hbm_read_probe(_ptr(src), src.numel() * src.element_size(), _ptr(sink), _stream(stream)), "hma_hbm_read_probe")
+
+
+def hma_hbm_copy_probe(src, read_bytes, dst, write_bytes, stream=None):
+    """Streaming read of `read_bytes` of `src` mixed with a streaming write of `write_bytes` of `dst` (a copy-like ceiling)."""
+    assert read_bytes <= src.numel() * src.element_size() and write_bytes <= dst.numel() * dst.element_size()
+    _check(lib().hma_hbm_copy_probe(_ptr(src), read_bytes, _ptr(dst), write_bytes, _stream(stream)), "hma_hbm_copy_probe")
 
 
 def hma_decode_attention_mixed(prefix, tail, layer, q, out, prefix_table, prefix_lens, tail_table, tail_lens, sm_scale,
