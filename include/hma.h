@@ -241,9 +241,12 @@ hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer
  * holding the KV of tokens generated since, which the paper's decode side produces in BF16, section 3.1; the
  * paper does not say where those live, this is one answer, hma_bfp8_encode_rows the other).  One softmax over
  * both.  Same q/out/sm_scale conventions as hma_decode_attention; both caches must have the same head counts and
- * HMA_KEYS_AS_QUERIES.  workspace: 2 * hma_decode_attention_workspace_bytes(desc, batch), rounded up to 256 each
- * (no zero-filling needed for this call).
- * Three launches: attention over each cache leaving one partial per CTA and segment, then a merge that completes the softmax.
+ * HMA_KEYS_AS_QUERIES.  workspace: 2 * hma_decode_attention_workspace_bytes(desc, batch), rounded up to 256 each,
+ * under the same zero-once contract as hma_decode_attention's (hma_decode_attention_workspace_init over all of it).
+ * Two launches: the tail cache first, every finished (sequence, kv head) segment leaving its unnormalised tile (vectors,
+ * maxima, sums) in the workspace's second half; then the prefix cache, whose kernel folds that tile into the segment
+ * right before it writes it.  The second kernel waits for the first only when it first needs a tile, so it sets up
+ * and streams records on every SM the first, usually tiny, kernel leaves free.
  */
 hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
                                         const void *q, void *out, int32_t out_dtype,

@@ -70,11 +70,10 @@ struct AttnArgs {
                                     // to sequence r / rows_per_seq and holds its queries (r % rows_per_seq) * kQ ..
     float sm_scale;
     int32_t *counters;              // workspace: one arrival counter per (sequence, kv head); zero between calls
-    int32_t *cum;                   // workspace: pages before each sequence, then pages + segment costs before each
-                                    // sequence, batch + 1 entries each (written for the two-cache merge kernel only)
+    int32_t *cum;                   // workspace: a reserved region between the counters and the tiles (unused)
     float *tiles;                   // workspace: per-CTA partial tiles; CTA c's partial of segment s is tile c + s
     float *tails;                   // workspace: one tile per segment, for the warp that holds the segment's end and goes on
-    int always_partial;             // 1: never write `out`; every segment leaves per-CTA partial tiles (two-cache attention)
+    const float *extra;             // kMode 3: the tiles such a launch left (its `tails`), folded into every segment before it is written
 #ifdef HMA_TRACE
     unsigned long long *trace;      // workspace, after the tiles: kTraceWords words per worker (see trace_stamp)
     long long drill_record;         // timeout drill: this record of the work list is announced 16 bytes too long (-1: none)
@@ -291,7 +290,21 @@ __host__ __device__ inline void segment_ctas(const Split &s, int64_t WX, int64_t
     *count = (int)(cta_of_worker(s, u1) - *c0 + 1);
 }
 
-// ---------------------------------------------------------------- the kernel
+// Two-cache attention: folds the tile that the other cache's launch left for a segment into the running (acc, M, den) of
+// q head h; this lane holds channels 4 * lane .. 4 * lane + 3.  `tile` is that segment's tile.
+__device__ __forceinline__ void fold_extra(const float *tile, int h, int lane, float4 &acc, float &M, float &den)
+{
+    const float mi = __ldcg(tile + 8 * kHeadDim + h), li = __ldcg(tile + 8 * kHeadDim + 8 + h);
+    const float4 v = __ldcg(reinterpret_cast<const float4 *>(tile + h * kHeadDim) + lane);
+    if (mi == -INFINITY) return;                   // nothing of this segment in the other cache (its vector is not meaningful)
+    const float Mn = fmaxf(M, mi);
+    const float keep = M == -INFINITY ? 0.f : ex2f(M - Mn), wgt = ex2f(mi - Mn);
+    acc.x = fmaf(wgt, v.x, acc.x * keep); acc.y = fmaf(wgt, v.y, acc.y * keep);
+    acc.z = fmaf(wgt, v.z, acc.z * keep); acc.w = fmaf(wgt, v.w, acc.w * keep);
+    den = fmaf(wgt, li, den * keep);
+    M = Mn;
+}
+
 // ---------------------------------------------------------------- CTA-level reduction and cross-CTA merge
 // Runs once per CTA after all of its warps have parked their last partial (a function of its own so that its
 // registers do not weigh on the record loop).
@@ -299,8 +312,9 @@ struct EpilogueArgs {       // what the reduction needs of AttnArgs, by value (r
     void *out;
     float *tiles, *tails;
     int32_t *counters;
-    int out_dtype, always_partial, batch, q_len, rows_per_seq;
+    int out_dtype, batch, q_len, rows_per_seq;
     struct { int num_kv_heads, num_q_heads; } cv;
+    const float *extra;
 #ifdef HMA_TRACE
     unsigned long long *trace;      // this warp's trace words
 #endif
@@ -320,7 +334,7 @@ constexpr int kGroupInts = 6;        // sequence, kv head, member mask, flags (1
 // and went on contributes its tail tile (ring slot 1) after them.  If the CTA holds only part of the segment,
 // parts = number of CTAs that share it, first CTA = the lowest.  gstate[0] = number of groups.
 template <int kFmt, int kQ>
-__device__ __noinline__ void plan_groups(int always_partial, int Hkv, int B, const long long *wr, const int *wseg, const int *cum,
+__device__ __noinline__ void plan_groups(int Hkv, int B, const long long *wr, const int *wseg, const int *cum,
                                          const int *ecum, int *gdesc, int *gstate)
 {
     constexpr int kWarps = Geo<kFmt, kQ>::warps;
@@ -348,7 +362,7 @@ __device__ __noinline__ void plan_groups(int always_partial, int Hkv, int B, con
             if (lane == 0) {
                 int parts = 0;
                 int64_t c0 = 0;
-                if (!whole_seg && !always_partial) {
+                if (!whole_seg) {
                     const int64_t WX = (int64_t)Hkv * ecum[B];
                     const Split sp = make_split(WX, (int)gridDim.x, kWarps);
                     const int64_t first = (int64_t)Hkv * ecum[sb] + (int64_t)sg * (npb + kSegCost) + kSegCost;   // cost position of the first record
@@ -390,7 +404,7 @@ __device__ __forceinline__ float4 lds_f4(uint32_t addr)
 // lane; lane i weighs the partial of warp i (lane kWarps: the tail tile), so the weights of a group cost one round of
 // loads and two shuffle reductions, and the 128-vectors are then summed in warp order, all loads in flight.  With two
 // query tiles per warp every (segment, q head) item exists once per tile.
-template <int kFmt, int kQ>
+template <int kFmt, int kQ, bool kExtra, bool kEmit>
 __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *ring,
                                           int *misc, const int *gdesc, const int *gstate)
 {
@@ -442,7 +456,12 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
                     acc.x = fmaf(wgt, v[i].x, acc.x); acc.y = fmaf(wgt, v[i].y, acc.y);
                     acc.z = fmaf(wgt, v[i].z, acc.z); acc.w = fmaf(wgt, v[i].w, acc.w);
                 }
-                if (whole_seg && !a.always_partial) {
+                if (whole_seg && kEmit) {                 // the finished segment, as a tile for the other cache's launch
+                    float *tp = a.tails + (((int64_t)sb * Hkv + sg) * kQ + t) * kTileFloats;
+                    *reinterpret_cast<float4 *>(tp + h * kHeadDim + 4 * lane) = acc;
+                    if (lane == 0) { tp[8 * kHeadDim + h] = M; tp[8 * kHeadDim + 8 + h] = den; }
+                } else if (whole_seg) {
+                    if (kExtra) fold_extra(a.extra + ((int64_t)sb * Hkv + sg) * kTileFloats, h, lane, acc, M, den);
                     const float inv = den > 0.f ? 1.f / den : 0.f;
                     store_quad(a.out, a.out_dtype, (query_row(a.q_len, a.rows_per_seq, kQ, sb, t) * Hq + (int64_t)sg * G + h) * kHeadDim + 4 * lane,
                                acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
@@ -507,6 +526,13 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
             }
             M = Mn;
         }
+        if (kEmit) {
+            float *tp = a.tails + (((int64_t)ob * Hkv + og) * kQ + t) * kTileFloats;
+            *reinterpret_cast<float4 *>(tp + h * kHeadDim + 4 * lane) = acc;
+            if (lane == 0) { tp[8 * kHeadDim + h] = M; tp[8 * kHeadDim + 8 + h] = den; }
+            continue;
+        }
+        if (kExtra) fold_extra(a.extra + ((int64_t)ob * Hkv + og) * kTileFloats, h, lane, acc, M, den);
         const float inv = den > 0.f ? 1.f / den : 0.f;
         store_quad(a.out, a.out_dtype, (query_row(a.q_len, a.rows_per_seq, kQ, ob, t) * Hq + (int64_t)og * G + h) * kHeadDim + 4 * lane,
                    acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
@@ -519,6 +545,13 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
 
 // kMode 0: attention.  1: stream the records through the ring, no arithmetic (bandwidth probe).
 // 2: the arithmetic of every record on whatever the ring holds, nothing loaded or written (issue-rate probe).
+// 4: attention over two caches, first launch: `out` is never written; every finished segment leaves its unnormalised tile
+//    (vectors, maxima, sums) in tails[segment] instead.
+// 3: attention over two caches, second launch: the launch before this one (the other cache, mode 4) left
+//    tiles that are folded into every segment before it is written.  Nothing that launch writes is read before
+//    the grid-dependency wait, which here comes late: right before the first fold.  Everything else this kernel reads
+//    was complete before that launch passed its own wait (it releases its dependents only after it), so the record loop
+//    of this launch runs beside it.
 extern __shared__ __align__(128) uint8_t smem_raw[];
 
 template <int kMode, int kFmt, int kQ>
@@ -527,6 +560,8 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     constexpr int kWarps = Geo<kFmt, kQ>::warps, kThreads = Geo<kFmt, kQ>::threads, kStages = Geo<kFmt, kQ>::stages;
     constexpr int kRecord = Geo<kFmt, kQ>::record, kDepth = Geo<kFmt, kQ>::depth;
     static_assert(kQ == 1 || kFmt == HMA_KV_BFP8, "two query tiles per warp exist for BFP8 caches only");
+    static_assert(kMode != 3 || kQ == 1, "two-cache attention takes one query token per sequence");
+    constexpr bool kAttn = kMode == 0 || kMode == 3 || kMode == 4, kExtra = kMode == 3, kEmit = kMode == 4;
     constexpr bool kBfp8 = kFmt == HMA_KV_BFP8;
     uint8_t *ring = smem_raw;                                                     // kStages records
     uint8_t *scratch = ring + kStages * kRecord;                                  // kWarps x kScratch (BFP8 only)
@@ -556,7 +591,7 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
 #ifdef HMA_TRACE
     const unsigned long long tr_entry = trace_now();
 #endif
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!kExtra) asm volatile("griddepcontrol.wait;" ::: "memory");
 #ifdef HMA_TRACE
     const unsigned long long tr_wait = trace_now();
 #endif
@@ -600,8 +635,6 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
 #endif
     // the next kernel of the stream may be placed as SMs free up; it waits on this grid by itself
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (blockIdx.x == 0 && kMode == 0 && a.always_partial)
-        for (int b = tid; b <= B; b += kThreads) { a.cum[b] = cum[b]; a.cum[B + 1 + b] = ecum[b]; }
     // from here to the CTA-level reduction at the end the warps never synchronise with one another
     const int64_t W = (int64_t)Hkv * cum[B];
     // The work list is cut by cost, not by record count: every (sequence, kv head) segment is charged kSegCost
@@ -625,19 +658,36 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         int cnt = 0;
         if (lane == 0) { __threadfence_block(); cnt = atomicAdd(&misc[1], 1); }
         cnt = __shfl_sync(0xFFFFFFFFu, cnt, 0);
-        if (cnt == kWarps - 1 && kMode == 0) {
+        if (cnt == kWarps - 1 && kAttn) {
             __threadfence_block();
-            plan_groups<kFmt, kQ>(a.always_partial, Hkv, B, wr, wseg, cum, ecum, gdesc, gstate);
+            plan_groups<kFmt, kQ>(Hkv, B, wr, wseg, cum, ecum, gdesc, gstate);
         }
     };
 
     do {    // ---- this warp's share of the work list; `break` leaves for the CTA-level reduction ----
     if (warp >= nmine) { publish(); break; }
-    if (kMode == 0 && !a.always_partial)                          // empty sequences get rows of zeros
+    if (kAttn)                                                    // empty sequences get rows of zeros
         for (int64_t b = u; b < B; b += NWK)
-            if (cum[b + 1] == cum[b])
-                for (int i = lane; i < kQ * Hq * kHeadDim; i += 32)
-                    store_out(a, query_row(a.q_len, a.rows_per_seq, kQ, (int)b, i / (Hq * kHeadDim)) * Hq * kHeadDim + i % (Hq * kHeadDim), 0.f);
+            if (cum[b + 1] == cum[b]) {
+                if (kEmit) {
+                    // as tiles: maximum -inf, sum 0 (the vectors are not read then)
+                    for (int i = lane; i < Hkv * kQ * 16; i += 32)
+                        a.tails[(b * Hkv * kQ + i / 16) * kTileFloats + 8 * kHeadDim + (i & 15)] = (i & 8) ? 0.f : -INFINITY;
+                } else if (kExtra) {
+                    // nothing in this cache: the row is whatever the other cache's launch left for it
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    for (int gh = 0; gh < Hkv * G; ++gh) {
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float M = -INFINITY, den = 0.f;
+                        fold_extra(a.extra + (b * Hkv + gh / G) * kTileFloats, gh % G, lane, acc, M, den);
+                        const float inv = den > 0.f ? 1.f / den : 0.f;
+                        store_quad(a.out, a.out_dtype, (b * Hq + gh) * kHeadDim + 4 * lane, acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                    }
+                } else {
+                    for (int i = lane; i < kQ * Hq * kHeadDim; i += 32)
+                        store_out(a, query_row(a.q_len, a.rows_per_seq, kQ, (int)b, i / (Hq * kHeadDim)) * Hq * kHeadDim + i % (Hq * kHeadDim), 0.f);
+                }
+            }
 
     // number of records that lie before cost position p
     auto records_before = [&](int64_t p) -> int64_t {
@@ -756,7 +806,7 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         tail = T - (np - 1) * kPageTokens;
         whole = page == 0 && Rw - k >= np;
         // Q fragments of this (sequence, kv head), per query token: FP16, one power-of-two scale per head
-        const bool hv = gq < G && kMode == 0;      // the probes have no Q: nothing is read through a.q
+        const bool hv = gq < G && kAttn;           // the probes have no Q: nothing is read through a.q
         const bool inter = a.cv.key_layout == HMA_KEYS_INTERLEAVED;
 #pragma unroll
         for (int t = 0; t < kQ; ++t) {
@@ -838,11 +888,34 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
             }
             const float l0 = lacc[t][0], l1 = lacc[t][1];
             // a softmax sum that is not finite: scores overflowed fp32 (K exponents beyond the supported range)
-            if (kMode == 0 && (!(l0 < INFINITY) || !(l1 < INFINITY))) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);
+            if (kAttn && (!(l0 < INFINITY) || !(l1 < INFINITY))) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);
             if (kMode == 2 && a.batch >= 0) continue;    // the issue-rate probe never stores, but keeps its arithmetic live
-            if (whole && !a.always_partial) {
+            if (whole && !kEmit) {
                 const int64_t ob = (query_row(a.q_len, a.rows_per_seq, kQ, b, t) * Hq + (int64_t)g * G) * kHeadDim;
-                const float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+                float i0 = l0 > 0.f ? 1.f / l0 : 0.f, i1 = l1 > 0.f ? 1.f / l1 : 0.f;
+                if (kExtra) {
+                    // the other cache's parts of this segment, folded in the accumulator layout (heads h0, h1 of this lane)
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    const float *tp = a.extra + seg * kTileFloats;
+                    float ll0 = l0, ll1 = l1;
+                    const float e0 = __ldcg(tp + 8 * kHeadDim + h0), e1 = __ldcg(tp + 8 * kHeadDim + h1);
+                    const float n0 = fmaxf(m0[t], e0), n1 = fmaxf(m1[t], e1);
+                    const float k0 = m0[t] == -INFINITY ? 0.f : ex2f(m0[t] - n0), k1 = m1[t] == -INFINITY ? 0.f : ex2f(m1[t] - n1);
+                    const float w0 = e0 == -INFINITY ? 0.f : ex2f(e0 - n0), w1 = e1 == -INFINITY ? 0.f : ex2f(e1 - n1);
+                    ll0 = fmaf(w0, __ldcg(tp + 8 * kHeadDim + 8 + h0), ll0 * k0);
+                    ll1 = fmaf(w1, __ldcg(tp + 8 * kHeadDim + 8 + h1), ll1 * k1);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            // a head the other cache holds nothing of contributes nothing, whatever its vector's bytes are
+                            const float wv = (c & 1) ? w1 : w0;
+                            const float x = __ldcg(tp + ((c & 1) ? h1 : h0) * kHeadDim + 16 * j + gq + 8 * (c >> 1));
+                            o[t][j][c] = fmaf(wv, wv > 0.f ? x : 0.f, o[t][j][c] * ((c & 1) ? k1 : k0));
+                        }
+                    i0 = ll0 > 0.f ? 1.f / ll0 : 0.f;
+                    i1 = ll1 > 0.f ? 1.f / ll1 : 0.f;
+                }
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
 #pragma unroll
@@ -854,8 +927,8 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
             }
             float *tp;
             int hs;           // floats between heads
-            if (whole) {      // two-cache attention: nobody else touches this segment, its tile goes straight to global memory
-                tp = a.tiles + (((int64_t)blockIdx.x + seg) * kQ + t) * kTileFloats;
+            if (whole) {      // two-cache attention, first launch: the finished segment's tile, for the other cache's launch
+                tp = a.tails + (seg * kQ + t) * kTileFloats;
                 hs = kHeadDim;
             } else if (at_end) {
                 tp = reinterpret_cast<float *>(ring + (warp * kDepth + t) * kRecord);
@@ -898,7 +971,7 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         --left;
         const uint32_t sp = ring0 + slot * kRecord;
         const int s_idx = warp * kDepth + slot;
-        if (kMode < 2) {
+        if (kMode != 2) {
 #ifdef HMA_TRACE
             alive = mbar_wait(full0 + 8 * slot, par, abort_word, a.cv.flags, a.spin_limit);
 #else
@@ -944,7 +1017,7 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
                     emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 8));
                     emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, 16));
                     const int Rnew = max(Rmine, emax);
-                    if (kMode == 0 && Rnew > 250) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);   // beyond the supported range
+                    if (kAttn && Rnew > 250) atomicOr(a.cv.flags, HMA_FLAG_EXPONENT_RANGE);   // beyond the supported range
     #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int dlt = __shfl_sync(0xFFFFFFFFu, Rmine, j) - __shfl_sync(0xFFFFFFFFu, Rnew, j);   // <= 0
@@ -1137,7 +1210,7 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     HMA_TRACE_STAMP(a, u, 4, trace_now());
     if (alive) {
         finish_segment(true);
-        if (tail_seg >= 0 && kMode == 0) {
+        if (tail_seg >= 0 && kAttn) {
             // the last tail tile this warp wrote (it can only be shared with other warps if it was the warp's first
             // segment, and a warp writes at most one such) comes back from L2 into ring slot 1, same layout
             __syncwarp();
@@ -1156,109 +1229,26 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         }
     }
     HMA_TRACE_STAMP(a, u, 5, trace_now());
-    if (!alive && lane == 0 && kMode < 2) {
+    if (!alive && lane == 0 && kMode != 2) {
         // a wait ran out: give the copies still in flight a bounded chance to land before the warp leaves
         for (int s = 0; s < kDepth; ++s)
             for (uint32_t it = 0; it < (1u << 16) && !mbar_try_wait(full0 + 8 * s, 0) && !mbar_try_wait(full0 + 8 * s, 1); ++it) {}
     }
     } while (0);
 
+    if (kExtra) asm volatile("griddepcontrol.wait;" ::: "memory");     // the other cache's tiles are read from here on
     __syncthreads();
-    if (kMode == 0) {
+    if (kAttn) {
         EpilogueArgs e;
         e.out = a.out; e.tiles = a.tiles; e.tails = a.tails; e.counters = a.counters;
-        e.out_dtype = a.out_dtype; e.always_partial = a.always_partial; e.batch = a.batch;
+        e.out_dtype = a.out_dtype; e.batch = a.batch;
         e.q_len = a.q_len; e.rows_per_seq = a.rows_per_seq;
         e.cv.num_kv_heads = a.cv.num_kv_heads; e.cv.num_q_heads = a.cv.num_q_heads;
+        e.extra = a.extra;
 #ifdef HMA_TRACE
         e.trace = a.trace + (((int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * sp.nwk / sp.ctas : 0) + warp) * kTraceWords;
 #endif
-        cta_epilogue<kFmt, kQ>(e, ring, misc, gdesc, gstate);
-    }
-}
-
-// Merge for attention over two caches (a BFP8 prefix and a BF16 tail of every sequence): both main kernels ran with
-// always_partial, so every segment of either cache left one partial tile per CTA that touched it; the softmax is
-// completed over the parts of both, prefix parts first, in CTA order.  One CTA per (sequence, kv head), one warp
-// per q head, four channels per lane.
-struct MergeSource {
-    const int32_t *cum;      // pages, then pages + segment costs, before each sequence
-    const float *tiles;
-    int grid_ctas;           // CTAs the main kernel was launched with
-    int warps;               // warps per CTA of that kernel
-};
-
-__device__ __forceinline__ void segment_parts(const MergeSource &s, int batch, int Hkv, int b, int g, int64_t *c0, int *count)
-{
-    const int np = s.cum[b + 1] - s.cum[b];
-    *count = 0;
-    *c0 = 0;
-    if (np == 0) return;
-    const int32_t *ecum = s.cum + batch + 1;
-    const int64_t WX = (int64_t)Hkv * ecum[batch];
-    const Split sp = make_split(WX, s.grid_ctas, s.warps);
-    const int64_t first = (int64_t)Hkv * ecum[b] + (int64_t)g * (np + kSegCost) + kSegCost;
-    segment_ctas(sp, WX, first, np, c0, count);
-}
-
-__global__ void __launch_bounds__(256) attn_merge_mixed_kernel(const AttnArgs a, MergeSource sa, MergeSource sb)
-{
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv;
-    const int b = blockIdx.x / Hkv, g = blockIdx.x % Hkv, h = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (h >= G) return;
-    int64_t ua, ub;
-    int pa, pb;
-    segment_parts(sa, a.batch, Hkv, b, g, &ua, &pa);
-    segment_parts(sb, a.batch, Hkv, b, g, &ub, &pb);
-    const int P = pa + pb;
-    auto part = [&](int j) -> const float * {
-        return j < pa ? sa.tiles + (ua + j + blockIdx.x) * kTileFloats : sb.tiles + (ub + (j - pa) + blockIdx.x) * kTileFloats;
-    };
-    float M = -INFINITY;
-    for (int c0 = 0; c0 < P; c0 += 32) {
-        float mm = c0 + lane < P ? __ldcg(part(c0 + lane) + 8 * kHeadDim + h) : -INFINITY;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, d));
-        M = fmaxf(M, mm);
-    }
-    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-    float den = 0.f;
-    for (int c0 = 0; c0 < P; c0 += 32) {
-        float wgt = 0.f, dsum = 0.f;
-        if (c0 + lane < P) {
-            const float *pt = part(c0 + lane);
-            const float mm = __ldcg(pt + 8 * kHeadDim + h);
-            wgt = mm == -INFINITY ? 0.f : ex2f(mm - M);
-            dsum = wgt * __ldcg(pt + 8 * kHeadDim + 8 + h);
-        }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) dsum += __shfl_xor_sync(0xFFFFFFFFu, dsum, d);     // fixed butterfly order
-        den += dsum;
-        const int cnt = min(32, P - c0);
-        for (int j0 = 0; j0 < cnt; j0 += 4) {
-            float4 v[4];
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj)
-                v[jj] = j0 + jj < cnt ? __ldcg(reinterpret_cast<const float4 *>(part(c0 + j0 + jj) + h * kHeadDim) + lane)
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-                const float wj = __shfl_sync(0xFFFFFFFFu, wgt, (j0 + jj) & 31);
-                num.x = fmaf(wj, v[jj].x, num.x); num.y = fmaf(wj, v[jj].y, num.y);
-                num.z = fmaf(wj, v[jj].z, num.z); num.w = fmaf(wj, v[jj].w, num.w);
-            }
-        }
-    }
-    const float inv = den > 0.f ? 1.f / den : 0.f;       // no tokens in either cache: a row of zeros
-    const int64_t oi = ((int64_t)b * Hq + (int64_t)g * G + h) * kHeadDim + 4 * lane;
-    if (a.out_dtype == HMA_OUT_F32) {
-        reinterpret_cast<float4 *>(a.out)[oi >> 2] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
-    } else {
-        const uint32_t lo = f32_to_bf16_rne(num.x * inv) | ((uint32_t)f32_to_bf16_rne(num.y * inv) << 16);
-        const uint32_t hi = f32_to_bf16_rne(num.z * inv) | ((uint32_t)f32_to_bf16_rne(num.w * inv) << 16);
-        reinterpret_cast<uint2 *>(a.out)[oi >> 2] = make_uint2(lo, hi);
+        cta_epilogue<kFmt, kQ, kExtra, kEmit>(e, ring, misc, gdesc, gstate);
     }
 }
 
@@ -1270,7 +1260,7 @@ static size_t attn_smem_bytes(int batch)
            (size_t)G::warps * 24 + (kMaxGroups * kGroupInts + 4) * 4 + ((size_t)batch + 1) * 8;
 }
 
-// Workspace layout: arrival counters | cum (two-cache merge only) | per-CTA tiles | per-segment tail tiles [| trace]
+// Workspace layout: arrival counters | a reserved region | per-CTA tiles | per-segment tiles [| trace]
 static size_t cum_bytes(int batch) { return (((size_t)batch + 1) * 8 + 255) & ~(size_t)255; }
 // The counters sit at the head of the workspace in a region of one size for every call, whatever its batch and head
 // count, so that calls of different shapes can share a workspace without one's tiles landing on the other's counters.
@@ -1316,7 +1306,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
                                      const int32_t *block_table, int32_t max_pages_per_seq, const int32_t *context_lens,
                                      int32_t n_seqs, float sm_scale, void *workspace, size_t workspace_bytes, void *stream,
                                      int probe, int always_partial = 0, hma::AttnArgs *args_out = nullptr, int *ctas_out = nullptr,
-                                     int32_t q_len = 1)
+                                     int32_t q_len = 1, const float *extra = nullptr)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || n_seqs < 0 || max_pages_per_seq < 0 || q_len < 1) return HMA_ERR_INVALID_ARG;
     if ((int64_t)n_seqs * q_len > hma::kMaxBatch) return HMA_ERR_UNSUPPORTED_SHAPE;
@@ -1331,7 +1321,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     if (bf16 && probe == 2) return HMA_ERR_UNSUPPORTED_SHAPE;
     // Two query tokens per warp (they share the unpacked K and V operands) when the query count is even, on BFP8 caches;
     // otherwise every query token is a row of its own.
-    const int kq = (!bf16 && probe == 0 && !always_partial && q_len % 2 == 0) ? 2 : 1;
+    const int kq = (!bf16 && probe == 0 && !always_partial && !extra && q_len % 2 == 0) ? 2 : 1;
     const int32_t rows = batch / kq;              // rows of the work list
     // per-device set-up, done by the first call on each device: SM count and the kernels' shared-memory opt-in
     static std::mutex setup_lock;
@@ -1351,6 +1341,10 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<2, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<0, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<1, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<3, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<3, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<4, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<4, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             sm_count[dev] = n;
         }
     }
@@ -1376,7 +1370,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.cum = (int32_t *)((uint8_t *)workspace + hma::counter_bytes(batch, hkv));
     a.tiles = (float *)((uint8_t *)a.cum + hma::cum_bytes(batch));
     a.tails = a.tiles + hma::cta_tiles(batch, hkv) * hma::kTileFloats;      // batch = rows x query tiles per row
-    a.always_partial = always_partial;
+    a.extra = extra;
 #ifdef HMA_TRACE
     a.trace = (unsigned long long *)(a.tails + (size_t)batch * hkv * hma::kTileFloats);
     a.drill_record = g_drill_record;
@@ -1398,7 +1392,11 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (bf16 && probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BF16, 1>, a));
+    if (always_partial && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<4, HMA_KV_BF16, 1>, a));
+    else if (always_partial) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<4, HMA_KV_BFP8, 1>, a));
+    else if (extra && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<3, HMA_KV_BF16, 1>, a));
+    else if (extra) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<3, HMA_KV_BFP8, 1>, a));
+    else if (bf16 && probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BF16, 1>, a));
     else if (bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<1, HMA_KV_BF16, 1>, a));
     else if (probe == 0 && kq == 2) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BFP8, 2>, a));
     else if (probe == 0) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<0, HMA_KV_BFP8, 1>, a));
@@ -1444,29 +1442,16 @@ extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, co
     const size_t half = (hma_decode_attention_workspace_bytes(&prefix->desc, batch) + 255) & ~(size_t)255;
     if (!workspace) return HMA_ERR_INVALID_ARG;
     if (workspace_bytes < 2 * half) return HMA_ERR_WORKSPACE_TOO_SMALL;
-    hma::AttnArgs aa, ab;
-    int wa = 0, wb = 0;
-    hma_status_t st = launch_attention(prefix, layer, q, out, out_dtype, prefix_table, prefix_max_pages, prefix_lens, batch, sm_scale,
-                                       workspace, half, stream, 0, 1, &aa, &wa);
+    // The tail cache first: every finished segment leaves its unnormalised tile (vectors, maxima, sums) instead of an
+    // output row.  Then the prefix cache, whose kernel folds that tile into the segment right before it writes it.  The
+    // second kernel reads nothing of the first before a late grid-dependency wait: on the SMs that the first, usually
+    // tiny, kernel leaves free it sets up and streams records at once.
+    hma::AttnArgs ab;
+    hma_status_t st = launch_attention(tail, layer, q, out, out_dtype, tail_table, tail_max_pages, tail_lens, batch, sm_scale,
+                                       (uint8_t *)workspace + half, half, stream, 0, 1, &ab);
     if (st != HMA_OK) return st;
-    st = launch_attention(tail, layer, q, out, out_dtype, tail_table, tail_max_pages, tail_lens, batch, sm_scale,
-                          (uint8_t *)workspace + half, half, stream, 0, 1, &ab, &wb);
-    if (st != HMA_OK) return st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(batch * prefix->desc.num_kv_heads));
-    cfg.blockDim = dim3(256);
-    cfg.stream = (cudaStream_t)stream;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    hma::MergeSource sa{aa.cum, aa.tiles, wa, hma::Geo<HMA_KV_BFP8>::warps}, sb{ab.cum, ab.tiles, wb, hma::Geo<HMA_KV_BF16>::warps};
-    if (prefix->desc.format != HMA_KV_BFP8) sa.warps = hma::Geo<HMA_KV_BF16>::warps;
-    if (tail->desc.format == HMA_KV_BFP8) sb.warps = hma::Geo<HMA_KV_BFP8>::warps;
-    HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_merge_mixed_kernel, aa, sa, sb));
-    hma::count_launch();
-    return HMA_OK;
+    return launch_attention(prefix, layer, q, out, out_dtype, prefix_table, prefix_max_pages, prefix_lens, batch, sm_scale,
+                            workspace, half, stream, 0, 0, nullptr, nullptr, 1, ab.tails);
 }
 
 extern "C" hma_status_t hma_kv_read_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,

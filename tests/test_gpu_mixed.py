@@ -64,6 +64,35 @@ def test_bfp8_prefix_plus_bf16_tail(hq, hkv):
     assert not out[2].any()                                  # no tokens in either cache
 
 
+def test_long_tails_short_prefixes_and_a_larger_batch():
+    """Tails that several CTAs share (their partials arrive as several tiles per segment), prefixes that one warp holds
+    entirely, sequences that live in one cache only; twice on the same workspace."""
+    prefix_lens = [112, 3000, 0, 40, 0] + [100 + 13 * i for i in range(19)]
+    tail_lens = [2100, 900, 700, 0, 0] + [(7 * i) % 50 for i in range(19)]
+    sc = Scenario(prefix_lens, 16, 4, seed=320, permute=True)
+    tail, ttable, tlens, ks, vs = _tail_scenario(sc, tail_lens, 321)
+    ws = hma.new_workspace(sc.desc, sc.B, copies=2)
+    ref64, _ = orc.decode_attention_mixed(bf16_bits(sc.q), sc.k_wires[0], sc.v_wires[0], ks, vs, 4)
+    outs = []
+    for rep in range(2):
+        o32 = torch.full((sc.B, 16, 128), float("nan"), dtype=torch.float32, device="cuda")
+        o16 = torch.full((sc.B, 16, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+        hma.hma_decode_attention_mixed(sc.cache, tail, 0, sc.q, o32, sc.table, sc.ctx, ttable, tlens, 1.0 / np.sqrt(128.0), ws)
+        hma.hma_decode_attention_mixed(sc.cache, tail, 0, sc.q, o16, sc.table, sc.ctx, ttable, tlens, 1.0 / np.sqrt(128.0), ws)
+        torch.cuda.synchronize()
+        check_attention(o32.cpu().numpy(), bf16_bits(o16), ref64)
+        outs.append(o32)
+    assert torch.equal(outs[0], outs[1])                     # fixed orders everywhere: bitwise repeatable
+    assert not outs[0][4].any()                              # no tokens in either cache
+    assert hma.hma_error_flags(sc.cache) == 0 and hma.hma_error_flags(tail) == 0
+    # the ordinary one-cache call still finds the workspace's counters at zero
+    ws1 = ws[:ws.numel() // 2]
+    out = torch.empty((sc.B, 16, 128), dtype=torch.float32, device="cuda")
+    hma.hma_decode_attention(sc.cache, 0, sc.q, out, sc.table, sc.ctx, 1.0 / np.sqrt(128.0), ws1)
+    torch.cuda.synchronize()
+    assert torch.equal(out, sc.attention(0, torch.float32))
+
+
 def test_bf16_rows_ingest_round_trip_and_rejection():
     sc = Scenario([40], 8, 2, seed=310, fmt=hma.HMA_KV_BF16)
     k = torch.randn((2, 40, 128), generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
