@@ -169,8 +169,18 @@ class Workload:
 
     _ingest_next = 0
 
-    def step(self, fmt="bfp8", ingest=True, host=False, staged=True, ingest_layers=None):
-        """One decode pass over all layers (+ the concurrent ingest).  Everything is enqueued; nothing syncs."""
+    def plan_for(self, fmt):
+        """The plan buffer of a cache (allocated once); hma_decode_attention_plan refills it at the start of every step."""
+        if not hasattr(self, "plans"):
+            self.plans = {}
+        if fmt not in self.plans:
+            self.plans[fmt] = self.hma.hma_decode_attention_plan(self.caches[fmt], self.table, self.ctx)
+        return self.plans[fmt]
+
+    def step(self, fmt="bfp8", ingest=True, host=False, staged=True, ingest_layers=None, planned=True):
+        """One decode pass over all layers (+ the concurrent ingest).  Everything is enqueued; nothing syncs.  With `planned`
+        the kernel's set-up is computed once per step (hma_decode_attention_plan, inside the step) and every layer's call
+        reads it; without, every call works it out again (hma_decode_attention)."""
         hma = self.hma
         main = torch.cuda.current_stream(self.device)
         do_ingest = ingest and self.ingest_tokens and fmt == "bfp8"
@@ -178,12 +188,17 @@ class Workload:
             self.side.wait_stream(main)
             self._ingest_all(self.wire_host if host else self.wire_dev, self.side, staged=host and staged, layers=ingest_layers)
         cache = self.caches[fmt]
+        if planned:
+            plan = hma.hma_decode_attention_plan(cache, self.table, self.ctx, plan=self.plan_for(fmt), stream=main)
         for l in range(self.L):
             q = self.q[l]
             if host:
                 self.q_stage[l].copy_(self.q_host[l], non_blocking=True)
                 q = self.q_stage[l]
-            hma.hma_decode_attention(cache, l, q, self.out[l], self.table, self.ctx, self.sm_scale, self.workspace, main)
+            if planned:
+                hma.hma_decode_attention_planned(cache, l, q, self.out[l], self.table, self.ctx, self.sm_scale, plan, self.workspace, main)
+            else:
+                hma.hma_decode_attention(cache, l, q, self.out[l], self.table, self.ctx, self.sm_scale, self.workspace, main)
             if host:
                 self.out_host[l].copy_(self.out[l], non_blocking=True)
         if do_ingest:
@@ -206,13 +221,15 @@ class Workload:
 
     def time_calls(self, kinds, passes, fmt="bfp8"):
         """Duration of single calls, CUDA events around every call on its stream.  `kinds` lists what to time
-        ("attn": hma_decode_attention, "probe": hma_kv_read_probe, "alu": hma_attention_alu_probe, "hbm": a plain
+        ("attn": hma_decode_attention_planned with the step's plan, "attn_self": hma_decode_attention, "probe": hma_kv_read_probe, "alu": hma_attention_alu_probe, "hbm": a plain
         contiguous read of the layer's bytes); the kinds are interleaved call by call, layer after layer, so that
         every kind sees the same clocks and the same cold L2.  Returns kind -> (mean, median, min) in seconds."""
         cache = self.caches[fmt]
         if not hasattr(self, "sink"):
             self.sink = torch.zeros(1, dtype=torch.int32, device=self.device)
         evs = {k: [] for k in kinds}
+        plan = self.plan_for(fmt)
+        self.hma.hma_decode_attention_plan(cache, self.table, self.ctx, plan=plan)
         for r in range(passes):
             for l in range(self.L):
                 for kind in kinds:
@@ -224,8 +241,11 @@ class Workload:
                         self.hma.hma_kv_read_probe(cache, l, self.table, self.ctx, self.workspace)
                     elif kind == "hbm":
                         self.hma.hma_hbm_read_probe(cache.layers[l], self.sink)
-                    else:
+                    elif kind == "attn_self":
                         self.hma.hma_decode_attention(cache, l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, self.workspace)
+                    else:
+                        self.hma.hma_decode_attention_planned(cache, l, self.q[l], self.out[l], self.table, self.ctx, self.sm_scale, plan,
+                                                              self.workspace)
                     b.record()
                     evs[kind].append((a, b))
         torch.cuda.synchronize(self.device)
@@ -523,8 +543,9 @@ def main():
     # (back to back, as inside a decode pass), then the two read ceilings interleaved with it call by call
     wl.time_layer_calls("bfp8", 1)
     call_mean, call_med, call_min = wl.time_layer_calls("bfp8", 5)
-    wl.time_calls(["attn", "probe", "hbm"], 1)
-    ceil = wl.time_calls(["attn", "probe", "hbm"], 5)
+    wl.time_calls(["attn", "attn_self", "probe", "hbm"], 1)
+    ceil = wl.time_calls(["attn", "attn_self", "probe", "hbm"], 5)
+    self_mean, self_med, self_min = ceil["attn_self"]
     probe_mean, probe_med, probe_min = ceil["probe"]
     hbm_mean, hbm_med, hbm_min = ceil["hbm"]
     inter_mean, inter_med, inter_min = ceil["attn"]
@@ -553,6 +574,8 @@ def main():
     torch.cuda.synchronize(device)
 
     sec_decode_only = wl.time_steps(args.steps, args.warmup, ingest=False)
+    # what the plan buys: steps with one plan per step against steps whose every call sets itself up, in alternation
+    alt_planned, alt_self = wl.time_alternating([dict(ingest=False), dict(ingest=False, planned=False)])
     # the ingest's cost to decode, each pair measured in alternation (same clocks for both sides)
     alt_ingest, alt_plain = wl.time_alternating([dict(), dict(ingest=False)]) if wl.ingest_tokens else (sec, sec)
     # the same request arriving at the rate of the paper's 100 Gb link (92.3 Gb/s measured, section 3.2): layers per step
@@ -644,13 +667,16 @@ def main():
                      "frac_of_probe": probe_med / inter_med,
                      "hbm_read_gbs": wl.caches["bfp8"].layers[0].numel() / hbm_med / 1e9,
                      "frac_of_hbm_read": (wl.kv_bytes_per_layer("bfp8") / inter_med) / (wl.caches["bfp8"].layers[0].numel() / hbm_med),
-                     "ceilings": {"what": "hma_decode_attention, hma_kv_read_probe (same records, no arithmetic) and hma_hbm_read_probe "
+                     "ceilings": {"what": "hma_decode_attention_planned, hma_decode_attention (sets itself up in every call), "
+                                          "hma_kv_read_probe (same records, no arithmetic) and hma_hbm_read_probe "
                                           "(plain contiguous read of the layer) interleaved call by call, 5 passes over all layers; "
                                           "[mean, median, min] us per call",
                                   "attention_us": [inter_mean * 1e6, inter_med * 1e6, inter_min * 1e6],
+                                  "attention_self_planned_us": [self_mean * 1e6, self_med * 1e6, self_min * 1e6],
                                   "kv_read_probe_us": [probe_mean * 1e6, probe_med * 1e6, probe_min * 1e6],
                                   "hbm_read_us": [hbm_mean * 1e6, hbm_med * 1e6, hbm_min * 1e6]},
-                     "kernel": "hma_decode_attention (attn_kernel<0,0>: attention and cross-split reduction in one launch)",
+                     "kernel": "hma_decode_attention_planned (attn_kernel<6,0,1>: attention and cross-split reduction in one launch, set-up "
+                               "read from the step's plan; one hma_decode_attention_plan launch per step is inside the timed steps)",
                      "bytes_per_launch": wl.kv_bytes_per_layer("bfp8"), "us_per_launch_mean": call_mean * 1e6,
                      "us_per_launch_median": call_med * 1e6, "us_per_launch_min": call_min * 1e6},
         "decode_only": {"tokens_per_s": aggregate_value(wl.B, sec_decode_only, ws), "ms_per_step": sec_decode_only * 1e3,
@@ -658,6 +684,9 @@ def main():
                         "how": "ms_per_step from its own run of the timed steps; the slowdown from steps with and without the ingest "
                                "timed in alternation (4 rounds of 4 steps each)"},
         "ingest_paced_at_link_rate": paced,
+        "plan": {"what": "decode pass (no ingest) with one hma_decode_attention_plan per step + planned calls, against the same pass "
+                         "with hma_decode_attention (every call repeats the set-up); timed in alternation, 4 rounds of 4 steps each",
+                 "ms_per_step_planned": alt_planned * 1e3, "ms_per_step_self_planned": alt_self * 1e3, "speedup": alt_self / alt_planned},
     }
     line.update(extra)
     if rank == 0 and ws == 1 and not args.no_cpu:

@@ -70,6 +70,8 @@ typedef enum { HMA_KEYS_AS_QUERIES = 0, HMA_KEYS_INTERLEAVED = 1 } hma_key_layou
 #define HMA_FLAG_BAD_VALUE_ENCODE  16u  /* hma_bfp8_encode_rows met NaN/Inf: encoded as zero      */
 #define HMA_FLAG_EXPONENT_RANGE   32u  /* attention met a V block exponent above 250, or a softmax
                                           sum that is not finite (K exponents that overflow fp32)   */
+#define HMA_FLAG_BAD_PLAN         64u  /* hma_decode_attention_planned was given a plan made for another launch shape:
+                                         nothing was computed                                  */
 
 typedef struct {
     int32_t num_layers;
@@ -234,6 +236,30 @@ hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer
                                          const int32_t *block_table, int32_t max_pages_per_seq,
                                          const int32_t *context_lens, int32_t batch, float sm_scale,
                                          void *stream);
+
+/*
+ * Plan once, run per layer.  Everything hma_decode_attention works out from the context lengths and the block table
+ * alone (page prefixes, the cut of the work list into per-warp record ranges, every warp's first record addresses,
+ * every CTA's reduction plan) is the same for all layers of one decode step; it costs each call about 4 us before
+ * its first record is even requested.  hma_decode_attention_plan runs that set-up once (one small launch) and writes it
+ * to `plan`; hma_decode_attention_planned is hma_decode_attention_multi with the set-up read from the plan.
+ *
+ *   plan         device, 256-byte aligned, >= hma_decode_attention_plan_bytes(batch * q_len) bytes.  Valid for calls with
+ *                the same cache geometry (format, head counts, num_pages), batch, q_len, max_pages_per_seq, on the same GPU
+ *                model, and only while block_table and context_lens hold what they held when the plan was made: make a
+ *                new plan whenever either changes (every decode step).  A plan made for another launch shape is detected:
+ *                the call computes nothing and raises HMA_FLAG_BAD_PLAN.  Stale table contents are not detectable.
+ *   results      identical, bit for bit, to hma_decode_attention_multi with the same arguments.
+ * The plan call is ordinary stream work: later planned calls on the same stream see it without further synchronisation.
+ */
+size_t hma_decode_attention_plan_bytes(int32_t rows);
+hma_status_t hma_decode_attention_plan(const hma_cache_t *cache, const int32_t *block_table, int32_t max_pages_per_seq,
+                                       const int32_t *context_lens, int32_t batch, int32_t q_len, void *plan,
+                                       size_t plan_bytes, void *stream);
+hma_status_t hma_decode_attention_planned(const hma_cache_t *cache, int32_t layer, const void *q, void *out,
+                                          int32_t out_dtype, const int32_t *block_table, int32_t max_pages_per_seq,
+                                          const int32_t *context_lens, int32_t batch, int32_t q_len, float sm_scale,
+                                          const void *plan, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Decode attention over two caches: the first prefix_lens[b] tokens of sequence b are pages of `prefix` (the BFP8

@@ -55,6 +55,30 @@ constexpr int kSegCost = 2;                        // what starting a segment co
 constexpr int kMaxCtas = 192;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
 constexpr int kMinRecords = 4;                    // fewest records a worker takes
 constexpr int kMaxDevices = 64;
+constexpr int kMaxGroups = 32;       // more than a CTA can have: a group holds a boundary between two of its (at most 16) warps, or one of its own ends
+constexpr int kGroupInts = 6;        // sequence, kv head, member mask, flags (1 whole segment, 2 has tail, tail warp << 8), parts, first CTA
+
+// A plan holds what the kernel's set-up works out from the context lengths and the block table alone, so that the calls
+// of one decode step (same lengths and table for every layer) do it once: the two page prefixes, every warp's record
+// range with its first segment and its first 32 record addresses, and every CTA's reduction plan.  Written by kMode 5,
+// read by kMode 6.  Layout: header (256 B) | cum, ecum | one PlanWorker per warp slot | 32 record offsets per warp slot |
+// kPlanGroupInts ints per CTA.
+constexpr uint32_t kPlanMagic = 0x504C414Eu;
+constexpr int kPlanGroupInts = kMaxGroups * kGroupInts + 4;
+struct PlanHeader {
+    uint32_t magic;
+    int32_t rows, hkv, warps, grid, kq, fmt, q_len, max_pages, num_pages;
+};
+struct __align__(16) PlanWorker {
+    long long wlo, whi;          // record range of the warp
+    int32_t u;                   // worker index, -1: the warp is no worker
+    int32_t b, g, page;          // segment and page of record wlo
+};
+__host__ __device__ inline size_t plan_cum_bytes(int rows) { return ((size_t)2 * (rows + 1) * 4 + 255) & ~(size_t)255; }
+__host__ __device__ inline size_t plan_workers_off(int rows) { return 256 + plan_cum_bytes(rows); }
+__host__ __device__ inline size_t plan_roff_off(int rows) { return plan_workers_off(rows) + (size_t)kMaxCtas * kWarps * sizeof(PlanWorker); }
+__host__ __device__ inline size_t plan_groups_off(int rows) { return plan_roff_off(rows) + (size_t)kMaxCtas * kWarps * 32 * 4; }
+__host__ __device__ inline size_t plan_total_bytes(int rows) { return plan_groups_off(rows) + (size_t)kMaxCtas * kPlanGroupInts * 4; }
 
 struct AttnArgs {
     CacheView cv;
@@ -73,6 +97,7 @@ struct AttnArgs {
     int32_t *cum;                   // workspace: a reserved region between the counters and the tiles (unused)
     float *tiles;                   // workspace: per-CTA partial tiles; CTA c's partial of segment s is tile c + s
     float *tails;                   // workspace: one tile per segment, for the warp that holds the segment's end and goes on
+    uint8_t *plan;                  // kMode 5 writes it, kMode 6 reads it (see PlanHeader)
     const float *extra;             // kMode 3: the tiles such a launch left (its `tails`), folded into every segment before it is written
 #ifdef HMA_TRACE
     unsigned long long *trace;      // workspace, after the tiles: kTraceWords words per worker (see trace_stamp)
@@ -86,8 +111,9 @@ struct AttnArgs {
 //   0 SM id   1 after the grid-dependency wait   2 end of the prologue   3 first record landed
 //   4 end of the record loop   5 after the last partial/output store   6 records taken   7 kernel entry (before the wait)
 //   8 CTA-level reduction begins (all warps of the CTA are done)   9 its segments are reduced
-//   10 arrivals on the shared segments' counters are done   11 the CTA leaves   12 walk begins   13-15 first segments done
-// Words 1-5 are %globaltimer nanoseconds; words 8-15 are the SM's cycle counter (only differences inside a CTA mean anything).
+//   10 arrivals on the shared segments' counters are done   11 the CTA leaves   12 the CTA leaves (wall clock)
+//   13 record range known   14 first record requested   15 after the reduction was planned
+// Words 1-5, 7 and 12-15 are %globaltimer nanoseconds; words 8-11 are the SM's cycle counter (only differences inside a CTA mean anything).
 constexpr int kTraceWords = 16;
 #ifdef HMA_TRACE
 __device__ __forceinline__ unsigned long long trace_now()
@@ -326,9 +352,6 @@ struct EpilogueArgs {       // what the reduction needs of AttnArgs, by value (r
 #endif
 // ---- group descriptors: what the CTA-level reduction has to do, worked out once per CTA right after the warps know
 // their ranges (everybody is waiting for first data then), so that nothing of it is on the critical path at the end
-constexpr int kMaxGroups = 32;       // more than a CTA can have: a group holds a boundary between two of its (at most 16) warps, or one of its own ends
-constexpr int kGroupInts = 6;        // sequence, kv head, member mask, flags (1 whole segment, 2 has tail, tail warp << 8), parts, first CTA
-
 // One full warp plans the groups of the CTA.  A group is a segment of the CTA's record range that no single warp held
 // entirely: `members` are the warps whose last partial (ring slot 0) belongs to it; a warp that held the segment's end
 // and went on contributes its tail tile (ring slot 1) after them.  If the CTA holds only part of the segment,
@@ -547,6 +570,7 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
 // 2: the arithmetic of every record on whatever the ring holds, nothing loaded or written (issue-rate probe).
 // 4: attention over two caches, first launch: `out` is never written; every finished segment leaves its unnormalised tile
 //    (vectors, maxima, sums) in tails[segment] instead.
+// 5: only the set-up, written out as a plan (no record is touched).  6: attention that takes its set-up from a plan.
 // 3: attention over two caches, second launch: the launch before this one (the other cache, mode 4) left
 //    tiles that are folded into every segment before it is written.  Nothing that launch writes is read before
 //    the grid-dependency wait, which here comes late: right before the first fold.  Everything else this kernel reads
@@ -561,7 +585,8 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     constexpr int kRecord = Geo<kFmt, kQ>::record, kDepth = Geo<kFmt, kQ>::depth;
     static_assert(kQ == 1 || kFmt == HMA_KV_BFP8, "two query tiles per warp exist for BFP8 caches only");
     static_assert(kMode != 3 || kQ == 1, "two-cache attention takes one query token per sequence");
-    constexpr bool kAttn = kMode == 0 || kMode == 3 || kMode == 4, kExtra = kMode == 3, kEmit = kMode == 4;
+    constexpr bool kAttn = kMode == 0 || kMode == 3 || kMode == 4 || kMode == 6, kExtra = kMode == 3, kEmit = kMode == 4;
+    constexpr bool kPlanOnly = kMode == 5, kPlanned = kMode == 6;
     constexpr bool kBfp8 = kFmt == HMA_KV_BFP8;
     uint8_t *ring = smem_raw;                                                     // kStages records
     uint8_t *scratch = ring + kStages * kRecord;                                  // kWarps x kScratch (BFP8 only)
@@ -595,9 +620,24 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
 #ifdef HMA_TRACE
     const unsigned long long tr_wait = trace_now();
 #endif
-    // Exclusive prefixes per sequence of (pages) and of (pages + kSegCost if the sequence is not empty): each thread
-    // owns `per` consecutive sequences, warps scan with shuffles, one warp scans the warp totals.
-    {
+    PlanWorker pw = {0, 0, -1, 0, 0, 0};
+    if constexpr (kPlanned) {
+        // the plan must have been made for this very launch shape; a call with any other is refused as a whole
+        const PlanHeader *ph = reinterpret_cast<const PlanHeader *>(a.plan);
+        if (ph->magic != kPlanMagic || ph->rows != B || ph->hkv != Hkv || ph->warps != kWarps || ph->grid != (int)gridDim.x ||
+            ph->kq != kQ || ph->fmt != kFmt || ph->q_len != a.q_len || ph->max_pages != a.max_pages || ph->num_pages != (int32_t)a.cv.num_pages) {
+            if (tid == 0) atomicOr(a.cv.flags, HMA_FLAG_BAD_PLAN);
+            return;
+        }
+        const int *pc = reinterpret_cast<const int *>(a.plan + 256);
+        for (int i = tid; i < 2 * (B + 1); i += kThreads) cum[i] = pc[i];            // cum and ecum are neighbours
+        const int *pg = reinterpret_cast<const int *>(a.plan + plan_groups_off(B)) + (size_t)blockIdx.x * kPlanGroupInts;
+        for (int i = tid; i < kPlanGroupInts; i += kThreads) gdesc[i] = pg[i];       // gdesc and gstate are neighbours
+        pw = reinterpret_cast<const PlanWorker *>(a.plan + plan_workers_off(B))[blockIdx.x * kWarps + warp];
+        __syncthreads();
+    } else {
+        // Exclusive prefixes per sequence of (pages) and of (pages + kSegCost if the sequence is not empty): each thread
+        // owns `per` consecutive sequences, warps scan with shuffles, one warp scans the warp totals.
         const int per = (B + kThreads - 1) / kThreads;
         const int b0 = min(B, tid * per), b1 = min(B, b0 + per);
         int mine = 0, emine = 0;
@@ -646,26 +686,40 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     // [c * NWK / C, (c + 1) * NWK / C) of the C CTAs in use), so a CTA owns one contiguous range of records.
     const Split sp = make_split(WX, (int)gridDim.x, kWarps);
     const int64_t NWK = sp.nwk;
-    const int64_t ubase = (int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * NWK / sp.ctas : NWK;
-    const int nmine = (int64_t)blockIdx.x < sp.ctas ? (int)(((int64_t)blockIdx.x + 1) * NWK / sp.ctas - ubase) : 0;
-    const int64_t u = ubase + warp;                                 // this warp's worker index (if warp < nmine)
-    if (lane == 0) { wr[2 * warp] = 0; wr[2 * warp + 1] = 0; }      // no records until shown otherwise
+    int64_t u;                                                      // this warp's worker index (if it is a worker)
+    bool worker;
+    if constexpr (kPlanned) {
+        u = pw.u;
+        worker = pw.u >= 0;
+    } else {
+        const int64_t ubase = (int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * NWK / sp.ctas : NWK;
+        const int nmine = (int64_t)blockIdx.x < sp.ctas ? (int)(((int64_t)blockIdx.x + 1) * NWK / sp.ctas - ubase) : 0;
+        u = ubase + warp;
+        worker = warp < nmine;
+        if (lane == 0) { wr[2 * warp] = 0; wr[2 * warp + 1] = 0; }  // no records until shown otherwise
+    }
+    PlanWorker *pw_out = nullptr;
+    if constexpr (kPlanOnly) {
+        pw_out = reinterpret_cast<PlanWorker *>(a.plan + plan_workers_off(B)) + blockIdx.x * kWarps + warp;
+        if (lane == 0) *pw_out = PlanWorker{0, 0, worker ? (int32_t)u : -1, 0, 0, 0};
+    }
 
     // Every warp publishes its record range exactly once; the warp that publishes last plans the CTA-level reduction
     // (who has to combine what at the end) while everybody is still waiting for first data.
     auto publish = [&]() {
+        if (kPlanned) return;                      // the plan holds the CTA's reduction plan already
         __syncwarp();
         int cnt = 0;
         if (lane == 0) { __threadfence_block(); cnt = atomicAdd(&misc[1], 1); }
         cnt = __shfl_sync(0xFFFFFFFFu, cnt, 0);
-        if (cnt == kWarps - 1 && kAttn) {
+        if (cnt == kWarps - 1 && (kAttn || kPlanOnly)) {
             __threadfence_block();
             plan_groups<kFmt, kQ>(Hkv, B, wr, wseg, cum, ecum, gdesc, gstate);
         }
     };
 
     do {    // ---- this warp's share of the work list; `break` leaves for the CTA-level reduction ----
-    if (warp >= nmine) { publish(); break; }
+    if (!worker) { publish(); break; }
     if (kAttn)                                                    // empty sequences get rows of zeros
         for (int64_t b = u; b < B; b += NWK)
             if (cum[b + 1] == cum[b]) {
@@ -702,7 +756,14 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         const int gg = (int)(off / (n + kSegCost)), r = (int)(off - (int64_t)gg * (n + kSegCost));
         return (int64_t)Hkv * cum[lo] + (int64_t)gg * n + max(0, r - kSegCost);
     };
-    const int64_t wlo = records_before(u * WX / NWK), whi = records_before((u + 1) * WX / NWK);
+    int64_t wlo, whi;
+    if constexpr (kPlanned) {
+        wlo = pw.wlo;
+        whi = pw.whi;
+    } else {
+        wlo = records_before(u * WX / NWK);
+        whi = records_before((u + 1) * WX / NWK);
+    }
     if (wlo >= whi) { publish(); break; }
     const int Rw = (int)(whi - wlo);
     HMA_TRACE_STAMP(a, u, 0, (unsigned long long)trace_smid());
@@ -710,10 +771,14 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     HMA_TRACE_STAMP(a, u, 2, tr_pro);
     HMA_TRACE_STAMP(a, u, 7, tr_entry);
     HMA_TRACE_STAMP(a, u, 6, (unsigned long long)Rw);
+    HMA_TRACE_STAMP(a, u, 13, trace_now());      // the warp knows its record range
 
     // the segment (b, g) and page that hold record wlo
     int b, g, page, np;
-    {
+    if constexpr (kPlanned) {
+        b = pw.b; g = pw.g; page = pw.page;
+        np = cum[b + 1] - cum[b];
+    } else {
         int lo = 0, hi = B - 1;
         while (lo < hi) {   // largest b with Hkv*cum[b] <= wlo
             int mid = (lo + hi + 1) >> 1;
@@ -726,7 +791,7 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         g = (int)(off / np);
         page = (int)(off - (int64_t)g * np);
     }
-    if (lane == 0) { wr[2 * warp] = wlo; wr[2 * warp + 1] = whi; wseg[2 * warp] = b; wseg[2 * warp + 1] = g; }
+    if (!kPlanned && lane == 0) { wr[2 * warp] = wlo; wr[2 * warp + 1] = whi; wseg[2 * warp] = b; wseg[2 * warp + 1] = g; }
 
     // ---- the warp's own feed: three ring slots; record addresses are worked out 32 at a time, one per lane ----
     const uint32_t full0 = smem_u32(bars + warp * kDepth);
@@ -778,11 +843,20 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         if (++islot == kDepth) islot = 0;
         if (++kissue == kwin + 32 && kissue < Rw) { kwin = kissue; refill(); }
     };
-    if (kMode != 2) refill();
+    if constexpr (kPlanned) roff = reinterpret_cast<const uint32_t *>(a.plan + plan_roff_off(B))[(blockIdx.x * kWarps + warp) * 32 + lane];
+    else if (kMode != 2) refill();
+    if constexpr (kPlanOnly) {
+        if (lane == 0) *pw_out = PlanWorker{wlo, whi, (int32_t)u, b, g, page};
+        reinterpret_cast<uint32_t *>(a.plan + plan_roff_off(B))[(blockIdx.x * kWarps + warp) * 32 + lane] = roff;
+        publish();
+        break;
+    }
     // Only the first record is requested now; the other slots are armed after the first segment's Q loads have been
     // issued, so that across the GPU every warp's first record is ahead of anybody's second in the memory queues.
     issue();
+    HMA_TRACE_STAMP(a, u, 14, trace_now());      // block table read, first record requested
     publish();
+    HMA_TRACE_STAMP(a, u, 15, trace_now());      // (the last warp of the CTA planned the reduction)
 
     // ---- consumer state ----
     const int gq = lane >> 2, t4 = lane & 3;
@@ -1238,6 +1312,19 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
 
     if (kExtra) asm volatile("griddepcontrol.wait;" ::: "memory");     // the other cache's tiles are read from here on
     __syncthreads();
+    if constexpr (kPlanOnly) {
+        int *pg = reinterpret_cast<int *>(a.plan + plan_groups_off(B)) + (size_t)blockIdx.x * kPlanGroupInts;
+        const int used = gstate[0] * kGroupInts;
+        for (int i = tid; i < kPlanGroupInts; i += kThreads) pg[i] = i < used ? gdesc[i] : i == kMaxGroups * kGroupInts ? gstate[0] : 0;
+        if (blockIdx.x == 0) {
+            int *pc = reinterpret_cast<int *>(a.plan + 256);
+            for (int i = tid; i < 2 * (B + 1); i += kThreads) pc[i] = cum[i];
+            if (tid == 0)
+                *reinterpret_cast<PlanHeader *>(a.plan) =
+                    PlanHeader{kPlanMagic, B, Hkv, kWarps, (int)gridDim.x, kQ, kFmt, a.q_len, a.max_pages, (int32_t)a.cv.num_pages};
+        }
+        return;
+    }
     if (kAttn) {
         EpilogueArgs e;
         e.out = a.out; e.tiles = a.tiles; e.tails = a.tails; e.counters = a.counters;
@@ -1306,17 +1393,18 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
                                      const int32_t *block_table, int32_t max_pages_per_seq, const int32_t *context_lens,
                                      int32_t n_seqs, float sm_scale, void *workspace, size_t workspace_bytes, void *stream,
                                      int probe, int always_partial = 0, hma::AttnArgs *args_out = nullptr, int *ctas_out = nullptr,
-                                     int32_t q_len = 1, const float *extra = nullptr)
+                                     int32_t q_len = 1, const float *extra = nullptr, void *plan = nullptr, int plan_mode = 0)
 {
     if (!cache || layer < 0 || layer >= cache->desc.num_layers || n_seqs < 0 || max_pages_per_seq < 0 || q_len < 1) return HMA_ERR_INVALID_ARG;
     if ((int64_t)n_seqs * q_len > hma::kMaxBatch) return HMA_ERR_UNSUPPORTED_SHAPE;
     const int32_t batch = n_seqs * q_len;         // rows of q and out
     if (out_dtype != HMA_OUT_BF16 && out_dtype != HMA_OUT_F32) return HMA_ERR_INVALID_ARG;
     if (batch == 0) return HMA_OK;
-    if (!block_table || !context_lens || !workspace || (!probe && (!q || !out))) return HMA_ERR_INVALID_ARG;
+    if (!block_table || !context_lens || (!workspace && plan_mode != 5) || (!probe && plan_mode != 5 && (!q || !out))) return HMA_ERR_INVALID_ARG;
     if (((uintptr_t)q & 15u) || ((uintptr_t)out & 15u) || ((uintptr_t)workspace & 255u)) return HMA_ERR_ALIGNMENT;
     if (batch > hma::kMaxBatch || max_pages_per_seq > (1 << 26)) return HMA_ERR_UNSUPPORTED_SHAPE;
-    if (workspace_bytes < hma_decode_attention_workspace_bytes(&cache->desc, batch)) return HMA_ERR_WORKSPACE_TOO_SMALL;
+    if (plan_mode != 5 && workspace_bytes < hma_decode_attention_workspace_bytes(&cache->desc, batch)) return HMA_ERR_WORKSPACE_TOO_SMALL;
+    if (plan_mode && (!plan || ((uintptr_t)plan & 255u))) return plan ? HMA_ERR_ALIGNMENT : HMA_ERR_INVALID_ARG;
     const bool bf16 = cache->desc.format != HMA_KV_BFP8;
     if (bf16 && probe == 2) return HMA_ERR_UNSUPPORTED_SHAPE;
     // Two query tokens per warp (they share the unpacked K and V operands) when the query count is even, on BFP8 caches;
@@ -1345,6 +1433,12 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<3, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<4, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<4, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<5, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<5, HMA_KV_BFP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<5, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<6, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<6, HMA_KV_BFP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<6, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             sm_count[dev] = n;
         }
     }
@@ -1367,10 +1461,15 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.sm_scale = sm_scale;
     const int hkv = cache->desc.num_kv_heads;
     a.counters = (int32_t *)workspace;
-    a.cum = (int32_t *)((uint8_t *)workspace + hma::counter_bytes(batch, hkv));
-    a.tiles = (float *)((uint8_t *)a.cum + hma::cum_bytes(batch));
-    a.tails = a.tiles + hma::cta_tiles(batch, hkv) * hma::kTileFloats;      // batch = rows x query tiles per row
+    a.cum = nullptr;
+    a.tiles = a.tails = nullptr;
+    if (workspace) {
+        a.cum = (int32_t *)((uint8_t *)workspace + hma::counter_bytes(batch, hkv));
+        a.tiles = (float *)((uint8_t *)a.cum + hma::cum_bytes(batch));
+        a.tails = a.tiles + hma::cta_tiles(batch, hkv) * hma::kTileFloats;      // batch = rows x query tiles per row
+    }
     a.extra = extra;
+    a.plan = (uint8_t *)plan;
 #ifdef HMA_TRACE
     a.trace = (unsigned long long *)(a.tails + (size_t)batch * hkv * hma::kTileFloats);
     a.drill_record = g_drill_record;
@@ -1392,7 +1491,13 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (always_partial && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<4, HMA_KV_BF16, 1>, a));
+    if (plan_mode == 5 && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<5, HMA_KV_BF16, 1>, a));
+    else if (plan_mode == 5 && kq == 2) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<5, HMA_KV_BFP8, 2>, a));
+    else if (plan_mode == 5) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<5, HMA_KV_BFP8, 1>, a));
+    else if (plan_mode == 6 && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<6, HMA_KV_BF16, 1>, a));
+    else if (plan_mode == 6 && kq == 2) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<6, HMA_KV_BFP8, 2>, a));
+    else if (plan_mode == 6) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<6, HMA_KV_BFP8, 1>, a));
+    else if (always_partial && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<4, HMA_KV_BF16, 1>, a));
     else if (always_partial) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<4, HMA_KV_BFP8, 1>, a));
     else if (extra && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<3, HMA_KV_BF16, 1>, a));
     else if (extra) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<3, HMA_KV_BFP8, 1>, a));
@@ -1424,6 +1529,30 @@ extern "C" hma_status_t hma_decode_attention_multi(const hma_cache_t *cache, int
 {
     return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
                             workspace, workspace_bytes, stream, 0, 0, nullptr, nullptr, q_len);
+}
+
+extern "C" size_t hma_decode_attention_plan_bytes(int32_t batch)
+{
+    return batch < 0 || batch > hma::kMaxBatch ? 0 : hma::plan_total_bytes(batch);
+}
+
+extern "C" hma_status_t hma_decode_attention_plan(const hma_cache_t *cache, const int32_t *block_table, int32_t max_pages_per_seq,
+                                                  const int32_t *context_lens, int32_t batch, int32_t q_len, void *plan,
+                                                  size_t plan_bytes, void *stream)
+{
+    if (q_len < 1 || batch < 0 || (int64_t)batch * q_len > hma::kMaxBatch) return batch < 0 || q_len < 1 ? HMA_ERR_INVALID_ARG : HMA_ERR_UNSUPPORTED_SHAPE;
+    if (batch > 0 && plan_bytes < hma::plan_total_bytes(batch * q_len)) return HMA_ERR_WORKSPACE_TOO_SMALL;
+    return launch_attention(cache, 0, nullptr, nullptr, HMA_OUT_BF16, block_table, max_pages_per_seq, context_lens, batch, 1.0f,
+                            nullptr, 0, stream, 0, 0, nullptr, nullptr, q_len, nullptr, plan, 5);
+}
+
+extern "C" hma_status_t hma_decode_attention_planned(const hma_cache_t *cache, int32_t layer, const void *q, void *out,
+                                                     int32_t out_dtype, const int32_t *block_table, int32_t max_pages_per_seq,
+                                                     const int32_t *context_lens, int32_t batch, int32_t q_len, float sm_scale,
+                                                     const void *plan, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return launch_attention(cache, layer, q, out, out_dtype, block_table, max_pages_per_seq, context_lens, batch, sm_scale,
+                            workspace, workspace_bytes, stream, 0, 0, nullptr, nullptr, q_len, nullptr, (void *)plan, 6);
 }
 
 extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,

@@ -21,7 +21,7 @@ HMA_WIRE_TILE32, HMA_WIRE_ROWMAJOR, HMA_WIRE_BF16_ROWS = 0, 1, 2
 HMA_OUT_BF16, HMA_OUT_F32 = 0, 1
 HMA_KEYS_AS_QUERIES, HMA_KEYS_INTERLEAVED = 0, 1
 HMA_FLAG_BAD_PAGE_ATTENTION, HMA_FLAG_BAD_PAGE_INGEST, HMA_FLAG_BAD_PAGE_DEQUANT, HMA_FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
-HMA_FLAG_BAD_VALUE_ENCODE, HMA_FLAG_EXPONENT_RANGE = 16, 32
+HMA_FLAG_BAD_VALUE_ENCODE, HMA_FLAG_EXPONENT_RANGE, HMA_FLAG_BAD_PLAN = 16, 32, 64
 
 
 class CacheDesc(ctypes.Structure):
@@ -71,6 +71,12 @@ def lib():
         L.hma_decode_attention.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp, sz, vp]
         L.hma_decode_attention_multi.restype = i32
         L.hma_decode_attention_multi.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, i32, f32, vp, sz, vp]
+        L.hma_decode_attention_plan_bytes.restype = sz
+        L.hma_decode_attention_plan_bytes.argtypes = [i32]
+        L.hma_decode_attention_plan.restype = i32
+        L.hma_decode_attention_plan.argtypes = [vp, vp, i32, vp, i32, i32, vp, sz, vp]
+        L.hma_decode_attention_planned.restype = i32
+        L.hma_decode_attention_planned.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, i32, f32, vp, vp, sz, vp]
         L.hma_decode_attention_static.restype = i32
         L.hma_decode_attention_static.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
         L.hma_decode_attention_static_limit_bytes.restype = sz
@@ -222,6 +228,34 @@ def hma_decode_attention_multi(cache, layer, q, out, block_table, context_lens, 
                                             block_table.shape[1], _ptr(context_lens), q.shape[0], q.shape[1], float(sm_scale),
                                             _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "hma_decode_attention_multi")
+
+
+def hma_decode_attention_plan_bytes(rows):
+    """Bytes of a plan for `rows` = sequences x query tokens per sequence."""
+    return int(lib().hma_decode_attention_plan_bytes(rows))
+
+
+def hma_decode_attention_plan(cache, block_table, context_lens, q_len=1, plan=None, stream=None):
+    """Runs the attention kernel's set-up for this block table and these context lengths once and returns the plan (a uint8
+    device tensor, reused when given); valid for every layer until the table or the lengths change."""
+    batch = context_lens.shape[0]
+    need = hma_decode_attention_plan_bytes(batch * q_len)
+    if plan is None:
+        plan = torch.empty(need, dtype=torch.uint8, device=context_lens.device)
+    _check(lib().hma_decode_attention_plan(cache.handle, _ptr(block_table), block_table.shape[1], _ptr(context_lens), batch, q_len,
+                                           _ptr(plan), plan.numel(), _stream(stream)), "hma_decode_attention_plan")
+    return plan
+
+
+def hma_decode_attention_planned(cache, layer, q, out, block_table, context_lens, sm_scale, plan, workspace, stream=None):
+    """hma_decode_attention (q, out: [batch][Hq][128]) or hma_decode_attention_multi (q, out: [batch][q_len][Hq][128]) with the
+    set-up taken from `plan` (hma_decode_attention_plan with the same table, lengths and q_len)."""
+    out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
+    q_len = q.shape[1] if q.dim() == 4 else 1
+    _check(lib().hma_decode_attention_planned(cache.handle, layer, _ptr(q), _ptr(out), out_dtype, _ptr(block_table),
+                                              block_table.shape[1], _ptr(context_lens), q.shape[0], q_len, float(sm_scale),
+                                              _ptr(plan), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                              _stream(stream)), "hma_decode_attention_planned")
 
 
 def hma_decode_attention_static(cache, layer, q, out, block_table, context_lens, sm_scale, stream=None):

@@ -65,6 +65,8 @@ def main():
         sm_mean = np.array([loop_end[smid == s].mean() for s in sms])
         within = np.array([loop_end[smid == s].max() - loop_end[smid == s].min() for s in sms])
         rows.append(dict(call_us=call_us, workers=len(tr), sms=len(sms), enter_spread=wait.max(), prologue_end=pro.mean(),
+                         range_known_mean=us(13).mean(), range_known_max=us(13).max(), first_request_mean=us(14).mean(),
+                         first_request_max=us(14).max(), planned_mean=us(15).mean(), planned_max=us(15).max(),
                          first_mean=first.mean(), first_max=first.max(), end_min=loop_end.min(), end_mean=loop_end.mean(),
                          end_p90=np.percentile(loop_end, 90), end_max=loop_end.max(), done_max=done.max(),
                          sm_mean_min=sm_mean.min(), sm_mean_max=sm_mean.max(), sm_mean_std=sm_mean.std(),

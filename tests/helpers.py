@@ -105,15 +105,19 @@ def check_attention(out_f32, out_bf16, ref64):
 
 def parity_sample(wl):
     """Outputs of the sequences a bench.Workload kept wire bytes of, against the oracle on those bytes, in the
-    full-size launch configuration.  The bar (max-abs 1e-2, rel-L2 2e-3) is taken on the F32 output; the BF16 output
+    full-size launch configuration that bench.py times (one plan, then planned calls); the call that plans for itself
+    must give the same bits.  The bar (max-abs 1e-2, rel-L2 2e-3) is taken on the F32 output; the BF16 output
     must be exactly its rounding; the BF16 numbers and the oracle's own BF16 rounding floor are returned beside it."""
     from oracle import oracle as orc
     res = []
     out32 = torch.empty((wl.B, wl.hq, 128), dtype=torch.float32, device=wl.device)
+    self32 = torch.empty_like(out32)
+    c = wl.caches["bfp8"]
+    plan = hma.hma_decode_attention_plan(c, wl.table, wl.ctx, plan=wl.plan_for("bfp8"))     # as at the start of a bench step
     for (l, b), (kw, vw) in sorted(wl.sample_wires.items()):
-        c = wl.caches["bfp8"]
-        hma.hma_decode_attention(c, l, wl.q[l], out32, wl.table, wl.ctx, wl.sm_scale, wl.workspace)
-        hma.hma_decode_attention(c, l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wl.workspace)
+        hma.hma_decode_attention_planned(c, l, wl.q[l], out32, wl.table, wl.ctx, wl.sm_scale, plan, wl.workspace)
+        hma.hma_decode_attention_planned(c, l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, plan, wl.workspace)
+        hma.hma_decode_attention(c, l, wl.q[l], self32, wl.table, wl.ctx, wl.sm_scale, wl.workspace)
         torch.cuda.synchronize(wl.device)
         qb = bf16_bits(wl.q[l][b:b + 1])
         ref64, ref16 = orc.decode_attention(qb, [kw], [vw], wl.hkv, wl.sm_scale)
@@ -125,5 +129,6 @@ def parity_sample(wl):
                     "f32_max_abs": float(np.abs(g32 - ref).max()), "f32_rel_l2": rel(g32),
                     "bf16_max_abs": float(np.abs(g16 - ref).max()), "bf16_rel_l2": rel(g16),
                     "bf16_is_rne_of_f32": bool(torch.equal(out32[b].to(torch.bfloat16), wl.out[l][b])),
+                    "planned_equals_self_planned": bool(torch.equal(out32.view(torch.int32), self32.view(torch.int32))),
                     "bf16_floor_rel_l2": rel(bf16_bits_to_f64(ref16[0]))})
     return res

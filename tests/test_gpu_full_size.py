@@ -28,6 +28,7 @@ def test_sampled_parity_full_batch(name):
     for r in res:
         assert r["f32_max_abs"] <= 1e-2 and r["f32_rel_l2"] <= 2e-3, (name, r)      # the bar, literally, on the F32 output
         assert r["bf16_is_rne_of_f32"], (name, r)                                     # BF16 output = exact rounding of it
+        assert r["planned_equals_self_planned"], (name, r)
         assert r["bf16_max_abs"] <= 1e-2 + 2.0 ** -8 * 25.0, (name, r)
         # rel-L2 of the BF16 output: the literal bar where the oracle's own rounded result meets it, else within 5 % of that floor
         assert r["bf16_rel_l2"] <= (2e-3 if r["bf16_floor_rel_l2"] <= 1.9e-3 else 1.05 * r["bf16_floor_rel_l2"]), (name, r)
