@@ -128,7 +128,7 @@ __device__ __forceinline__ unsigned trace_smid()
     asm volatile("mov.u32 %0, %%smid;" : "=r"(v));
     return v;
 }
-#define HMA_TRACE_STAMP(a, u, i, v)  do { if ((threadIdx.x & 31) == 0) (a).trace[(u) * kTraceWords + (i)] = (v); } while (0)
+#define HMA_TRACE_STAMP(a, u, i, v)  do { if ((threadIdx.x & 31) == 0 && (a).trace) (a).trace[(u) * kTraceWords + (i)] = (v); } while (0)   /* a plan launch has no workspace, hence no trace area */
 #else
 #define HMA_TRACE_STAMP(a, u, i, v)  do { } while (0)
 #endif
@@ -1471,7 +1471,7 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     a.extra = extra;
     a.plan = (uint8_t *)plan;
 #ifdef HMA_TRACE
-    a.trace = (unsigned long long *)(a.tails + (size_t)batch * hkv * hma::kTileFloats);
+    a.trace = workspace ? (unsigned long long *)(a.tails + (size_t)batch * hkv * hma::kTileFloats) : nullptr;
     a.drill_record = g_drill_record;
     a.spin_limit = g_drill_record >= 0 ? g_drill_spin_limit : hma::kSpinLimit;
     g_drill_record = -1;

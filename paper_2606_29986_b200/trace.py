@@ -1,8 +1,9 @@
 """Per-warp timing of the attention kernel, from the instrumented build of the library (-DHMA_TRACE).
 
-    python -m paper_2606_29986_b200.trace [--workload NAME] [--layers N] [--reps R]
+    python -m paper_2606_29986_b200.trace [--workload NAME] [--layers N] [--reps R] [--self-planned]
 
-Builds libhma_trace.so if needed, runs hma_decode_attention on a benchmark workload with that image, reads the
+Builds libhma_trace.so if needed, runs hma_decode_attention_planned (with --self-planned: hma_decode_attention, which
+repeats the set-up in every call) on a benchmark workload with that image, reads the
 time stamps every worker (warp) left behind its partial tiles, and prints a summary: when warps start, when their
 first record lands, when they leave the record loop, how that spreads inside an SM and between SMs, what the CTA-level
 reduction costs, and how three consecutive calls hand over to one another.  The default
@@ -23,6 +24,7 @@ def main():
     ap.add_argument("--workload", default="qwen3-32b-b32-ctx8k")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--self-planned", action="store_true")
     args = ap.parse_args()
 
     from paper_2606_29986_b200 import build
@@ -37,14 +39,22 @@ def main():
     n_workers = 192 * 16
     trace_off = ws_bytes - n_workers * TRACE_WORDS * 8
     assert wl.workspace.numel() >= ws_bytes
+    cache = wl.caches["bfp8"]
+    plan = hma.hma_decode_attention_plan(cache, wl.table, wl.ctx)
+
+    def attention(l, ws):
+        if args.self_planned:
+            hma.hma_decode_attention(cache, l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, ws)
+        else:
+            hma.hma_decode_attention_planned(cache, l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, plan, ws)
 
     def run(l):
         wl.workspace[trace_off:ws_bytes].zero_()
         # two calls back to back: the second one starts the way a call inside a decode pass does
-        hma.hma_decode_attention(wl.caches["bfp8"], (l + 1) % wl.L, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wl.workspace)
+        attention((l + 1) % wl.L, wl.workspace)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        hma.hma_decode_attention(wl.caches["bfp8"], l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wl.workspace)
+        attention(l, wl.workspace)
         e1.record()
         torch.cuda.synchronize()
         tr = wl.workspace[trace_off:ws_bytes].view(torch.int64).cpu().numpy().reshape(-1, TRACE_WORDS).copy()
@@ -79,7 +89,7 @@ def main():
     wss = [hma.new_workspace(wl.caches["bfp8"].desc, wl.B, dev) for _ in range(3)]
     for i in range(24):
         l = i % wl.L
-        hma.hma_decode_attention(wl.caches["bfp8"], l, wl.q[l], wl.out[l], wl.table, wl.ctx, wl.sm_scale, wss[i % 3])
+        attention(l, wss[i % 3])
     torch.cuda.synchronize()
     chain = []
     for ws in wss:
@@ -96,8 +106,8 @@ def main():
             i, f(T[:, 7].min()), f(T[:, 7].max()), f(T[:, 1].min()), f(T[:, 1].max()), f(T[:, 3].mean()), f(T[:, 4].mean()), f(T[:, 4].max()),
             f(ex.min()), f(ex.mean()), f(ex.max())))
     keys = [k for k in rows[0] if k != "slow"]
-    print("workload %s, %d layers built, %d traced calls (all times in us after the first warp passed the grid-dependency wait)" %
-          (args.workload, wl.L, len(rows)))
+    print("workload %s, %d layers built, %d traced %s calls (all times in us after the first warp passed the grid-dependency wait)" %
+          (args.workload, wl.L, len(rows), "self-planning" if args.self_planned else "planned"))
     print("| quantity | " + " | ".join("call %d" % i for i in range(len(rows))) + " |")
     print("|---|" + "---|" * len(rows))
     for k in keys:
