@@ -70,8 +70,8 @@ typedef enum { HMA_KEYS_AS_QUERIES = 0, HMA_KEYS_INTERLEAVED = 1 } hma_key_layou
 #define HMA_FLAG_BAD_VALUE_ENCODE  16u  /* hma_bfp8_encode_rows met NaN/Inf: encoded as zero      */
 #define HMA_FLAG_EXPONENT_RANGE   32u  /* attention met a V block exponent above 250, or a softmax
                                           sum that is not finite (K exponents that overflow fp32)   */
-#define HMA_FLAG_BAD_PLAN         64u  /* hma_decode_attention_planned was given a plan made for another launch shape:
-                                         nothing was computed                                  */
+#define HMA_FLAG_BAD_PLAN         64u  /* hma_decode_attention_planned was given a plan made for another launch shape
+                                         (nothing was computed) or for other page counts (results void) */
 
 typedef struct {
     int32_t num_layers;
@@ -246,9 +246,12 @@ hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer
  *
  *   plan         device, 256-byte aligned, >= hma_decode_attention_plan_bytes(batch * q_len) bytes.  Valid for calls with
  *                the same cache geometry (format, head counts, num_pages), batch, q_len, max_pages_per_seq, on the same GPU
- *                model, and only while block_table and context_lens hold what they held when the plan was made: make a
- *                new plan whenever either changes (every decode step).  A plan made for another launch shape is detected:
- *                the call computes nothing and raises HMA_FLAG_BAD_PLAN.  Stale table contents are not detectable.
+ *                model, while the block table holds what it held when the plan was made and every sequence still has
+ *                the same number of pages: context lengths may grow inside their last pages (the lengths themselves are
+ *                read at every call), so a plan lasts until a sequence starts a new page or the batch changes.  A plan
+ *                made for another launch shape is detected and the call computes nothing; page counts that no longer
+ *                match are detected while the call runs and its results are void; both raise HMA_FLAG_BAD_PLAN.  Changed
+ *                table entries under unchanged page counts are not detectable.
  *   results      identical, bit for bit, to hma_decode_attention_multi with the same arguments.
  * The plan call is ordinary stream work: later planned calls on the same stream see it without further synchronisation.
  */

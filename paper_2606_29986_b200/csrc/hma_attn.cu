@@ -341,6 +341,10 @@ struct EpilogueArgs {       // what the reduction needs of AttnArgs, by value (r
     int out_dtype, batch, q_len, rows_per_seq;
     struct { int num_kv_heads, num_q_heads; } cv;
     const float *extra;
+    const int32_t *ctx;             // planned calls: what the plan's page counts are checked against at the very end
+    const int *cum;
+    uint32_t *flags;
+    int max_pages;
 #ifdef HMA_TRACE
     unsigned long long *trace;      // this warp's trace words
 #endif
@@ -427,7 +431,7 @@ __device__ __forceinline__ float4 lds_f4(uint32_t addr)
 // lane; lane i weighs the partial of warp i (lane kWarps: the tail tile), so the weights of a group cost one round of
 // loads and two shuffle reductions, and the 128-vectors are then summed in warp order, all loads in flight.  With two
 // query tiles per warp every (segment, q head) item exists once per tile.
-template <int kFmt, int kQ, bool kExtra, bool kEmit>
+template <int kFmt, int kQ, bool kExtra, bool kEmit, bool kPlanned>
 __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *ring,
                                           int *misc, const int *gdesc, const int *gstate)
 {
@@ -502,6 +506,15 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
             }
         }
     }
+    // A planned call checks, once and after its own work, that the plan's page counts are those of the context lengths it
+    // was called with (lengths may have grown inside their last pages since the plan was made).  Nothing unsafe happens
+    // otherwise (pages are looked up in the live table and range-checked), but the results are void and the call says so.
+    if constexpr (kPlanned)
+        for (int bb = blockIdx.x * kWarps * 32 + tid; bb < a.batch; bb += gridDim.x * kWarps * 32) {
+            const int s = bb / a.rows_per_seq, i = (bb - s * a.rows_per_seq) * kQ + kQ - 1;
+            const int T = max(0, max(0, min(a.ctx[s], a.max_pages * kPageTokens)) - (a.q_len - 1 - i));
+            if ((T + kPageTokens - 1) / kPageTokens != a.cum[bb + 1] - a.cum[bb]) atomicOr(a.flags, HMA_FLAG_BAD_PLAN);
+        }
     HMA_TRACE_EPI(a, 9);
     if (n_open == 0) return;                      // the same for every thread of the CTA
     // Arrival: the CTA's tile stores happen before the barrier, the release of the arriving thread's atomic carries
@@ -1332,10 +1345,11 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         e.q_len = a.q_len; e.rows_per_seq = a.rows_per_seq;
         e.cv.num_kv_heads = a.cv.num_kv_heads; e.cv.num_q_heads = a.cv.num_q_heads;
         e.extra = a.extra;
+        e.ctx = a.ctx; e.cum = cum; e.flags = a.cv.flags; e.max_pages = a.max_pages;
 #ifdef HMA_TRACE
         e.trace = a.trace + (((int64_t)blockIdx.x < sp.ctas ? (int64_t)blockIdx.x * sp.nwk / sp.ctas : 0) + warp) * kTraceWords;
 #endif
-        cta_epilogue<kFmt, kQ, kExtra, kEmit>(e, ring, misc, gdesc, gstate);
+        cta_epilogue<kFmt, kQ, kExtra, kEmit, kPlanned>(e, ring, misc, gdesc, gstate);
     }
 }
 

@@ -80,6 +80,27 @@ def test_a_plan_for_another_shape_is_refused():
     assert torch.equal(out, sc.attention(0, torch.float32)) and hma.hma_error_flags(sc.cache) == 0
 
 
+def test_a_plan_lasts_until_a_sequence_starts_a_new_page():
+    sc = Scenario([200, 50, 900, 33], 16, 4, seed=440, permute=True)
+    plan = hma.hma_decode_attention_plan(sc.cache, sc.table, sc.ctx)
+    # shorter contexts inside the same pages (as if the plan had been made a few decode steps ago): still the right plan
+    ctx = torch.tensor([195, 49, 897, 33], dtype=torch.int32, device="cuda")
+    ref = torch.empty((sc.B, 16, 128), dtype=torch.float32, device="cuda")
+    out = torch.empty_like(ref)
+    hma.hma_decode_attention(sc.cache, 0, sc.q, ref, sc.table, ctx, SCALE, sc.workspace)
+    hma.hma_decode_attention_planned(sc.cache, 0, sc.q, out, sc.table, ctx, SCALE, plan, sc.workspace)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref) and hma.hma_error_flags(sc.cache) == 0
+    assert not torch.equal(ref, sc.attention(0, torch.float32))          # and the lengths did matter
+    # one sequence a page shorter: the plan no longer fits, the call says so (and stays inside its memory)
+    ctx[2] = 880
+    hma.hma_decode_attention_planned(sc.cache, 0, sc.q, out, sc.table, ctx, SCALE, plan, sc.workspace)
+    torch.cuda.synchronize()
+    assert hma.hma_error_flags(sc.cache) & hma.HMA_FLAG_BAD_PLAN          # (a page without a valid token may raise more)
+    hma.hma_decode_attention_workspace_init(sc.workspace)                 # a void call may leave counters behind
+    assert torch.equal(sc.attention(0, torch.float32), sc.attention(0, torch.float32))
+
+
 def test_plan_argument_checks():
     sc = Scenario([40], 8, 2, seed=430)
     need = hma.hma_decode_attention_plan_bytes(1)
