@@ -364,15 +364,19 @@ class Workload:
         return src.numel() / best / 1e9
 
     def time_multi_query(self, q_len, reps=3):
-        """hma_decode_attention_multi with q_len query tokens per sequence (the last q_len cached tokens): mean seconds per call."""
+        """hma_decode_attention_planned with q_len query tokens per sequence (the last q_len cached tokens; the planned form of
+        hma_decode_attention_multi): mean seconds per call, the pass's one plan launch included."""
         hma = self.hma
         q = synth.make_q(self.B * q_len, self.hq, 4321, self.device).view(self.B, q_len, self.hq, 128)
         out = torch.empty_like(q)
         ws = hma.new_workspace(self.caches["bfp8"].desc, self.B * q_len, self.device)
 
-        def run():
+        plan = hma.hma_decode_attention_plan(self.caches["bfp8"], self.table, self.ctx, q_len=q_len)
+
+        def run():          # one plan per pass over the layers, as in step()
+            hma.hma_decode_attention_plan(self.caches["bfp8"], self.table, self.ctx, q_len=q_len, plan=plan)
             for l in range(self.L):
-                hma.hma_decode_attention_multi(self.caches["bfp8"], l, q, out, self.table, self.ctx, self.sm_scale, ws)
+                hma.hma_decode_attention_planned(self.caches["bfp8"], l, q, out, self.table, self.ctx, self.sm_scale, plan, ws)
         run()
         torch.cuda.synchronize(self.device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -628,7 +632,8 @@ def main():
     extra["mixed_prefix_tail"] = {"us_per_call": t_mixed * 1e6, "tail_tokens_per_sequence": 64,
                                   "what": "hma_decode_attention_mixed: BFP8 prefix cache + BF16 cache with 64 decode-side tokens per sequence",
                                   "overhead_vs_prefix_only": t_mixed / call_mean - 1.0}
-    mq = {"what": "hma_decode_attention_multi: q_len query tokens per sequence over the same cache (speculative / chunked decode); "
+    mq = {"what": "hma_decode_attention_planned with q_len query tokens per sequence over the same cache (speculative / chunked decode; "
+                  "the planned form of hma_decode_attention_multi, one plan per pass over the layers); "
                   "tokens/s counts query tokens, attention only, all layers"}
     base_call = wl.time_multi_query(1)
     for q_len in (1, 2, 4):
