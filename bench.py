@@ -333,11 +333,15 @@ class Workload:
             for b in range(self.B):
                 hma.hma_kv_ingest_layer(tail, l, rows, rows, hma.HMA_WIRE_BF16_ROWS, 0, self.hkv, ttable[b].contiguous(), 0, tail_tokens)
         ws = hma.new_workspace(self.caches["bfp8"].desc, self.B, self.device, copies=2)
+        pplan = hma.hma_decode_attention_plan(self.caches["bfp8"], self.table, self.ctx)
+        tplan = hma.hma_decode_attention_plan(tail, ttable, tlens)
 
-        def run():
+        def run():          # two plans per pass over the layers, then planned calls
+            hma.hma_decode_attention_plan(self.caches["bfp8"], self.table, self.ctx, plan=pplan)
+            hma.hma_decode_attention_plan(tail, ttable, tlens, plan=tplan)
             for l in range(self.L):
-                hma.hma_decode_attention_mixed(self.caches["bfp8"], tail, l, self.q[l], self.out[l], self.table, self.ctx, ttable, tlens,
-                                               self.sm_scale, ws)
+                hma.hma_decode_attention_mixed_planned(self.caches["bfp8"], tail, l, self.q[l], self.out[l], self.table, self.ctx, ttable,
+                                                       tlens, self.sm_scale, pplan, tplan, ws)
         run()
         torch.cuda.synchronize(self.device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -630,7 +634,7 @@ def main():
                                  "what": "hma_kv_ingest_layer_shards, one 8192-token layer (4 shards, TILE32), device-resident wire, CUDA-graph replay"}
     t_mixed = wl.time_mixed()
     extra["mixed_prefix_tail"] = {"us_per_call": t_mixed * 1e6, "tail_tokens_per_sequence": 64,
-                                  "what": "hma_decode_attention_mixed: BFP8 prefix cache + BF16 cache with 64 decode-side tokens per sequence",
+                                  "what": "hma_decode_attention_mixed_planned: BFP8 prefix cache + BF16 cache with 64 decode-side tokens per sequence (two plans per pass)",
                                   "overhead_vs_prefix_only": t_mixed / call_mean - 1.0}
     mq = {"what": "hma_decode_attention_planned with q_len query tokens per sequence over the same cache (speculative / chunked decode; "
                   "the planned form of hma_decode_attention_multi, one plan per pass over the layers); "

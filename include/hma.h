@@ -283,6 +283,15 @@ hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cac
                                         const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens,
                                         int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes,
                                         void *stream);
+/* The same with both launches' set-up taken from plans: prefix_plan from hma_decode_attention_plan(prefix, prefix_table,
+ * prefix_max_pages, prefix_lens, batch, 1, ..), tail_plan likewise for the tail cache (two plan buffers).  Same results bit
+ * for bit; the rules for a plan's lifetime are those of hma_decode_attention_planned. */
+hma_status_t hma_decode_attention_mixed_planned(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
+                                                const void *q, void *out, int32_t out_dtype,
+                                                const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,
+                                                const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens,
+                                                int32_t batch, float sm_scale, const void *prefix_plan, const void *tail_plan,
+                                                void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * One-shot reconstruction (section 3.3): tokens [token_begin, token_begin+n_tokens) of a request,

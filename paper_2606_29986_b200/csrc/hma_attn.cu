@@ -584,6 +584,7 @@ __device__ __noinline__ void cta_epilogue(const EpilogueArgs a, const uint8_t *r
 // 4: attention over two caches, first launch: `out` is never written; every finished segment leaves its unnormalised tile
 //    (vectors, maxima, sums) in tails[segment] instead.
 // 5: only the set-up, written out as a plan (no record is touched).  6: attention that takes its set-up from a plan.
+// 7, 8: modes 3 and 4 with the set-up taken from a plan.
 // 3: attention over two caches, second launch: the launch before this one (the other cache, mode 4) left
 //    tiles that are folded into every segment before it is written.  Nothing that launch writes is read before
 //    the grid-dependency wait, which here comes late: right before the first fold.  Everything else this kernel reads
@@ -597,9 +598,9 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     constexpr int kWarps = Geo<kFmt, kQ>::warps, kThreads = Geo<kFmt, kQ>::threads, kStages = Geo<kFmt, kQ>::stages;
     constexpr int kRecord = Geo<kFmt, kQ>::record, kDepth = Geo<kFmt, kQ>::depth;
     static_assert(kQ == 1 || kFmt == HMA_KV_BFP8, "two query tiles per warp exist for BFP8 caches only");
-    static_assert(kMode != 3 || kQ == 1, "two-cache attention takes one query token per sequence");
-    constexpr bool kAttn = kMode == 0 || kMode == 3 || kMode == 4 || kMode == 6, kExtra = kMode == 3, kEmit = kMode == 4;
-    constexpr bool kPlanOnly = kMode == 5, kPlanned = kMode == 6;
+    static_assert((kMode != 3 && kMode != 7) || kQ == 1, "two-cache attention takes one query token per sequence");
+    constexpr bool kAttn = kMode == 0 || kMode == 3 || kMode == 4 || kMode >= 6, kExtra = kMode == 3 || kMode == 7, kEmit = kMode == 4 || kMode == 8;
+    constexpr bool kPlanOnly = kMode == 5, kPlanned = kMode >= 6;
     constexpr bool kBfp8 = kFmt == HMA_KV_BFP8;
     uint8_t *ring = smem_raw;                                                     // kStages records
     uint8_t *scratch = ring + kStages * kRecord;                                  // kWarps x kScratch (BFP8 only)
@@ -1453,6 +1454,10 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<6, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<6, HMA_KV_BFP8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<6, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<7, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<7, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<8, HMA_KV_BFP8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            HMA_CUDA_OK(cudaFuncSetAttribute(hma::attn_kernel<8, HMA_KV_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             sm_count[dev] = n;
         }
     }
@@ -1508,6 +1513,10 @@ static hma_status_t launch_attention(const hma_cache_t *cache, int32_t layer, co
     if (plan_mode == 5 && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<5, HMA_KV_BF16, 1>, a));
     else if (plan_mode == 5 && kq == 2) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<5, HMA_KV_BFP8, 2>, a));
     else if (plan_mode == 5) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<5, HMA_KV_BFP8, 1>, a));
+    else if (plan_mode == 6 && extra && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<7, HMA_KV_BF16, 1>, a));
+    else if (plan_mode == 6 && extra) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<7, HMA_KV_BFP8, 1>, a));
+    else if (plan_mode == 6 && always_partial && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<8, HMA_KV_BF16, 1>, a));
+    else if (plan_mode == 6 && always_partial) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<8, HMA_KV_BFP8, 1>, a));
     else if (plan_mode == 6 && bf16) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<6, HMA_KV_BF16, 1>, a));
     else if (plan_mode == 6 && kq == 2) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<6, HMA_KV_BFP8, 2>, a));
     else if (plan_mode == 6) HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::attn_kernel<6, HMA_KV_BFP8, 1>, a));
@@ -1569,12 +1578,11 @@ extern "C" hma_status_t hma_decode_attention_planned(const hma_cache_t *cache, i
                             workspace, workspace_bytes, stream, 0, 0, nullptr, nullptr, q_len, nullptr, (void *)plan, 6);
 }
 
-extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
-                                                   const void *q, void *out, int32_t out_dtype,
-                                                   const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,
-                                                   const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens,
-                                                   int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes,
-                                                   void *stream)
+static hma_status_t launch_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer, const void *q, void *out,
+                                 int32_t out_dtype, const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,
+                                 const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens, int32_t batch,
+                                 float sm_scale, const void *prefix_plan, const void *tail_plan, void *workspace,
+                                 size_t workspace_bytes, void *stream)
 {
     if (!prefix || !tail) return HMA_ERR_INVALID_ARG;
     if (prefix->desc.num_q_heads != tail->desc.num_q_heads || prefix->desc.num_kv_heads != tail->desc.num_kv_heads ||
@@ -1585,16 +1593,41 @@ extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, co
     const size_t half = (hma_decode_attention_workspace_bytes(&prefix->desc, batch) + 255) & ~(size_t)255;
     if (!workspace) return HMA_ERR_INVALID_ARG;
     if (workspace_bytes < 2 * half) return HMA_ERR_WORKSPACE_TOO_SMALL;
+    const int pm = prefix_plan ? 6 : 0;
     // The tail cache first: every finished segment leaves its unnormalised tile (vectors, maxima, sums) instead of an
     // output row.  Then the prefix cache, whose kernel folds that tile into the segment right before it writes it.  The
     // second kernel reads nothing of the first before a late grid-dependency wait: on the SMs that the first, usually
-    // tiny, kernel leaves free it sets up and streams records at once.
+    // tiny, kernel leaves free it sets up and streams records at once.  (With plans: whatever made them ran before the
+    // first kernel passed its own wait, so the second kernel may read its plan at once, too.)
     hma::AttnArgs ab;
     hma_status_t st = launch_attention(tail, layer, q, out, out_dtype, tail_table, tail_max_pages, tail_lens, batch, sm_scale,
-                                       (uint8_t *)workspace + half, half, stream, 0, 1, &ab);
+                                       (uint8_t *)workspace + half, half, stream, 0, 1, &ab, nullptr, 1, nullptr, (void *)tail_plan, pm);
     if (st != HMA_OK) return st;
     return launch_attention(prefix, layer, q, out, out_dtype, prefix_table, prefix_max_pages, prefix_lens, batch, sm_scale,
-                            workspace, half, stream, 0, 0, nullptr, nullptr, 1, ab.tails);
+                            workspace, half, stream, 0, 0, nullptr, nullptr, 1, ab.tails, (void *)prefix_plan, pm);
+}
+
+extern "C" hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
+                                                   const void *q, void *out, int32_t out_dtype,
+                                                   const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,
+                                                   const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens,
+                                                   int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes,
+                                                   void *stream)
+{
+    return launch_mixed(prefix, tail, layer, q, out, out_dtype, prefix_table, prefix_max_pages, prefix_lens, tail_table, tail_max_pages,
+                        tail_lens, batch, sm_scale, nullptr, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" hma_status_t hma_decode_attention_mixed_planned(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
+                                                           const void *q, void *out, int32_t out_dtype,
+                                                           const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,
+                                                           const int32_t *tail_table, int32_t tail_max_pages, const int32_t *tail_lens,
+                                                           int32_t batch, float sm_scale, const void *prefix_plan, const void *tail_plan,
+                                                           void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!prefix_plan || !tail_plan) return HMA_ERR_INVALID_ARG;
+    return launch_mixed(prefix, tail, layer, q, out, out_dtype, prefix_table, prefix_max_pages, prefix_lens, tail_table, tail_max_pages,
+                        tail_lens, batch, sm_scale, prefix_plan, tail_plan, workspace, workspace_bytes, stream);
 }
 
 extern "C" hma_status_t hma_kv_read_probe(const hma_cache_t *cache, int32_t layer, const int32_t *block_table,

@@ -91,6 +91,8 @@ def lib():
         L.hma_attention_alu_probe.argtypes = [vp, i32, vp, i32, vp, i32, vp, sz, vp]
         L.hma_decode_attention_mixed.restype = i32
         L.hma_decode_attention_mixed.argtypes = [vp, vp, i32, vp, vp, i32, vp, i32, vp, vp, i32, vp, i32, f32, vp, sz, vp]
+        L.hma_decode_attention_mixed_planned.restype = i32
+        L.hma_decode_attention_mixed_planned.argtypes = [vp, vp, i32, vp, vp, i32, vp, i32, vp, vp, i32, vp, i32, f32, vp, vp, vp, sz, vp]
         L.hma_decode_attention_simple.restype = i32
         L.hma_decode_attention_simple.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp, i32, f32, vp]
         L.hma_bfp8_dequant_bf16.restype = i32
@@ -306,6 +308,18 @@ def hma_decode_attention_mixed(prefix, tail, layer, q, out, prefix_table, prefix
                                             _ptr(tail_table), tail_table.shape[1], _ptr(tail_lens), q.shape[0],
                                             float(sm_scale), _ptr(workspace), workspace.numel() * workspace.element_size(),
                                             _stream(stream)), "hma_decode_attention_mixed")
+
+
+def hma_decode_attention_mixed_planned(prefix, tail, layer, q, out, prefix_table, prefix_lens, tail_table, tail_lens, sm_scale,
+                                       prefix_plan, tail_plan, workspace, stream=None):
+    """hma_decode_attention_mixed with both launches' set-up taken from plans (one per cache, hma_decode_attention_plan)."""
+    out_dtype = HMA_OUT_F32 if out.dtype == torch.float32 else HMA_OUT_BF16
+    _check(lib().hma_decode_attention_mixed_planned(prefix.handle, tail.handle, layer, _ptr(q), _ptr(out), out_dtype,
+                                                    _ptr(prefix_table), prefix_table.shape[1], _ptr(prefix_lens),
+                                                    _ptr(tail_table), tail_table.shape[1], _ptr(tail_lens), q.shape[0],
+                                                    float(sm_scale), _ptr(prefix_plan), _ptr(tail_plan), _ptr(workspace),
+                                                    workspace.numel() * workspace.element_size(), _stream(stream)),
+           "hma_decode_attention_mixed_planned")
 
 
 def hma_decode_attention_simple(cache, layer, q, out, block_table, context_lens, sm_scale, stream=None):

@@ -83,6 +83,16 @@ def test_long_tails_short_prefixes_and_a_larger_batch():
         check_attention(o32.cpu().numpy(), bf16_bits(o16), ref64)
         outs.append(o32)
     assert torch.equal(outs[0], outs[1])                     # fixed orders everywhere: bitwise repeatable
+    # with both launches' set-up taken from plans: the same bits
+    pplan = hma.hma_decode_attention_plan(sc.cache, sc.table, sc.ctx)
+    tplan = hma.hma_decode_attention_plan(tail, ttable, tlens)
+    o32 = torch.full((sc.B, 16, 128), float("nan"), dtype=torch.float32, device="cuda")
+    hma.hma_decode_attention_mixed_planned(sc.cache, tail, 0, sc.q, o32, sc.table, sc.ctx, ttable, tlens, 1.0 / np.sqrt(128.0), pplan, tplan, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(o32, outs[0])
+    hma.hma_decode_attention_mixed_planned(sc.cache, tail, 0, sc.q, o32, sc.table, sc.ctx, ttable, tlens, 1.0 / np.sqrt(128.0), tplan, pplan, ws)
+    torch.cuda.synchronize()                                 # plans swapped: refused
+    assert hma.hma_error_flags(tail) | hma.hma_error_flags(sc.cache) == hma.HMA_FLAG_BAD_PLAN and torch.equal(o32, outs[0])
     assert not outs[0][4].any()                              # no tokens in either cache
     assert hma.hma_error_flags(sc.cache) == 0 and hma.hma_error_flags(tail) == 0
     # the ordinary one-cache call still finds the workspace's counters at zero
