@@ -61,8 +61,9 @@ constexpr int kGroupInts = 6;        // sequence, kv head, member mask, flags (1
 // A plan holds what the kernel's set-up works out from the context lengths and the block table alone, so that the calls
 // of one decode step (same lengths and table for every layer) do it once: the two page prefixes, every warp's record
 // range with its first segment and its first 32 record addresses, and every CTA's reduction plan.  Written by kMode 5,
-// read by kMode 6.  Layout: header (256 B) | cum, ecum | one PlanWorker per warp slot | 32 record offsets per warp slot |
-// kPlanGroupInts ints per CTA.
+// read by kMode 6.  Layout: header (256 B) | one PlanWorker per warp slot | 32 record offsets per warp slot |
+// kPlanGroupInts ints per CTA | cum, ecum.  Everything but the prefixes sits at offsets that do not depend on the batch, so
+// a planned kernel may load its own entries before it has checked the header: any plan buffer is large enough for that.
 constexpr uint32_t kPlanMagic = 0x504C414Eu;
 constexpr int kPlanGroupInts = kMaxGroups * kGroupInts + 4;
 struct PlanHeader {
@@ -75,10 +76,11 @@ struct __align__(16) PlanWorker {
     int32_t b, g, page;          // segment and page of record wlo
 };
 __host__ __device__ inline size_t plan_cum_bytes(int rows) { return ((size_t)2 * (rows + 1) * 4 + 255) & ~(size_t)255; }
-__host__ __device__ inline size_t plan_workers_off(int rows) { return 256 + plan_cum_bytes(rows); }
+__host__ __device__ inline size_t plan_workers_off(int) { return 256; }
 __host__ __device__ inline size_t plan_roff_off(int rows) { return plan_workers_off(rows) + (size_t)kMaxCtas * kWarps * sizeof(PlanWorker); }
 __host__ __device__ inline size_t plan_groups_off(int rows) { return plan_roff_off(rows) + (size_t)kMaxCtas * kWarps * 32 * 4; }
-__host__ __device__ inline size_t plan_total_bytes(int rows) { return plan_groups_off(rows) + (size_t)kMaxCtas * kPlanGroupInts * 4; }
+__host__ __device__ inline size_t plan_cum_off(int rows) { return plan_groups_off(rows) + (size_t)kMaxCtas * kPlanGroupInts * 4; }
+__host__ __device__ inline size_t plan_total_bytes(int rows) { return plan_cum_off(rows) + plan_cum_bytes(rows); }
 
 struct AttnArgs {
     CacheView cv;
@@ -114,7 +116,7 @@ struct AttnArgs {
 //   10 arrivals on the shared segments' counters are done   11 the CTA leaves   12 the CTA leaves (wall clock)
 //   13 record range known   14 first record requested   15 after the reduction was planned
 // Words 1-5, 7 and 12-15 are %globaltimer nanoseconds; words 8-11 are the SM's cycle counter (only differences inside a CTA mean anything).
-constexpr int kTraceWords = 16;
+[[maybe_unused]] constexpr int kTraceWords = 16;
 #ifdef HMA_TRACE
 __device__ __forceinline__ unsigned long long trace_now()
 {
@@ -618,8 +620,16 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Hkv = a.cv.num_kv_heads, Hq = a.cv.num_q_heads, G = Hq / Hkv, B = a.batch;
 
+    constexpr bool kPlannedMode = kMode >= 7;       // the planned two-cache modes, whose short first launch is all head
+    if (kPlannedMode && lane == 0) {
+        // a planned warp requests its first record before the CTA's first barrier: it prepares its own slots
+        for (int s = 0; s < kDepth; ++s) mbar_init(smem_u32(bars + warp * kDepth + s), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(bars + s), 1);
+        if (!kPlannedMode)
+            for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(bars + s), 1);
         misc[0] = 0;
         misc[1] = 0;                     // warps that have published their record range
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -635,7 +645,10 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     const unsigned long long tr_wait = trace_now();
 #endif
     PlanWorker pw = {0, 0, -1, 0, 0, 0};
-    if constexpr (kPlanned) {
+    constexpr uint32_t kNoRecord = 0xFFFFFFFFu;
+    uint32_t plan_roff = kNoRecord;               // planned: this lane's record of the warp's first window
+    bool first_requested = false;                 // planned: the warp's first record is already on its way
+    if constexpr (kMode == 6) {
         // the plan must have been made for this very launch shape; a call with any other is refused as a whole
         const PlanHeader *ph = reinterpret_cast<const PlanHeader *>(a.plan);
         if (ph->magic != kPlanMagic || ph->rows != B || ph->hkv != Hkv || ph->warps != kWarps || ph->grid != (int)gridDim.x ||
@@ -643,11 +656,49 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
             if (tid == 0) atomicOr(a.cv.flags, HMA_FLAG_BAD_PLAN);
             return;
         }
-        const int *pc = reinterpret_cast<const int *>(a.plan + 256);
+        const int *pc = reinterpret_cast<const int *>(a.plan + plan_cum_off(B));
         for (int i = tid; i < 2 * (B + 1); i += kThreads) cum[i] = pc[i];            // cum and ecum are neighbours
         const int *pg = reinterpret_cast<const int *>(a.plan + plan_groups_off(B)) + (size_t)blockIdx.x * kPlanGroupInts;
         for (int i = tid; i < kPlanGroupInts; i += kThreads) gdesc[i] = pg[i];       // gdesc and gstate are neighbours
         pw = reinterpret_cast<const PlanWorker *>(a.plan + plan_workers_off(B))[blockIdx.x * kWarps + warp];
+        __syncthreads();
+    } else if constexpr (kPlanned) {
+        // The planned two-cache modes: their first launch is short and nearly all head, so the head is cut further (the same
+        // order of loads in the one-cache kernel made its record loop 0.8 us slower through different code generation).
+        // One trip to L2 for the header, the warp's entry, its first record addresses and the CTA's reduction plan (all at
+        // offsets that hold for any plan buffer); then the header is checked: the plan must have been made for this very
+        // launch shape, a call with any other is refused as a whole.
+        const PlanHeader hd = *reinterpret_cast<const PlanHeader *>(a.plan);
+        pw = reinterpret_cast<const PlanWorker *>(a.plan + plan_workers_off(B))[blockIdx.x * kWarps + warp];
+        plan_roff = reinterpret_cast<const uint32_t *>(a.plan + plan_roff_off(B))[(blockIdx.x * kWarps + warp) * 32 + lane];
+        const int *pg = reinterpret_cast<const int *>(a.plan + plan_groups_off(B)) + (size_t)blockIdx.x * kPlanGroupInts;
+        static_assert(kPlanGroupInts <= kThreads, "one thread per word of the CTA's reduction plan");
+        const int gword = tid < kPlanGroupInts ? pg[tid] : 0;
+        if (hd.magic != kPlanMagic || hd.rows != B || hd.hkv != Hkv || hd.warps != kWarps || hd.grid != (int)gridDim.x ||
+            hd.kq != kQ || hd.fmt != kFmt || hd.q_len != a.q_len || hd.max_pages != a.max_pages || hd.num_pages != (int32_t)a.cv.num_pages) {
+            if (tid == 0) atomicOr(a.cv.flags, HMA_FLAG_BAD_PLAN);
+            return;
+        }
+        // the warp's first record is requested right away (its slots were prepared by its own lane 0 above)
+        const uint32_t r0 = __shfl_sync(0xFFFFFFFFu, plan_roff, 0);
+        if (kPlannedMode && pw.u >= 0 && pw.wlo < pw.whi && r0 != kNoRecord) {
+            if (lane == 0) {
+                uint64_t pol;
+                asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+                const uint32_t bar0 = smem_u32(bars + warp * kDepth);
+                stage_ok[warp * kDepth] = 1;
+#ifdef HMA_TRACE
+                mbar_arrive_expect_tx(bar0, kRecord + (pw.wlo == a.drill_record ? 16 : 0));
+#else
+                mbar_arrive_expect_tx(bar0, kRecord);
+#endif
+                bulk_load(smem_u32(ring + warp * kDepth * kRecord), a.cv.layer + (uint64_t)r0 * 128u, kRecord, bar0, pol);
+            }
+            first_requested = true;
+        }
+        if (tid < kPlanGroupInts) gdesc[tid] = gword;                                // gdesc and gstate are neighbours
+        const int *pc = reinterpret_cast<const int *>(a.plan + plan_cum_off(B));
+        for (int i = tid; i < 2 * (B + 1); i += kThreads) cum[i] = pc[i];            // cum and ecum are neighbours
         __syncthreads();
     } else {
         // Exclusive prefixes per sequence of (pages) and of (pages + kSegCost if the sequence is not empty): each thread
@@ -810,7 +861,6 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     // ---- the warp's own feed: three ring slots; record addresses are worked out 32 at a time, one per lane ----
     const uint32_t full0 = smem_u32(bars + warp * kDepth);
     const uint32_t ring0 = smem_u32(ring + warp * kDepth * kRecord);
-    constexpr uint32_t kNoRecord = 0xFFFFFFFFu;
     uint32_t roff = kNoRecord;                    // this lane's record of the current window, in units of 128 bytes
     int kwin = 0;                                 // the window covers records [kwin, kwin + 32) of this warp
     int kissue = 0;                               // next record to request
@@ -857,7 +907,8 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         if (++islot == kDepth) islot = 0;
         if (++kissue == kwin + 32 && kissue < Rw) { kwin = kissue; refill(); }
     };
-    if constexpr (kPlanned) roff = reinterpret_cast<const uint32_t *>(a.plan + plan_roff_off(B))[(blockIdx.x * kWarps + warp) * 32 + lane];
+    if constexpr (kMode == 6) roff = reinterpret_cast<const uint32_t *>(a.plan + plan_roff_off(B))[(blockIdx.x * kWarps + warp) * 32 + lane];
+    else if constexpr (kPlanned) roff = plan_roff;
     else if (kMode != 2) refill();
     if constexpr (kPlanOnly) {
         if (lane == 0) *pw_out = PlanWorker{wlo, whi, (int32_t)u, b, g, page};
@@ -867,7 +918,13 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     }
     // Only the first record is requested now; the other slots are armed after the first segment's Q loads have been
     // issued, so that across the GPU every warp's first record is ahead of anybody's second in the memory queues.
-    issue();
+    if (kPlanned && first_requested) {            // record 0 went out before the CTA's first barrier
+        kissue = 1;
+        islot = kDepth > 1 ? 1 : 0;
+        if (kissue == kwin + 32 && kissue < Rw) { kwin = kissue; refill(); }      // (never: a window holds 32 records)
+    } else {
+        issue();
+    }
     HMA_TRACE_STAMP(a, u, 14, trace_now());      // block table read, first record requested
     publish();
     HMA_TRACE_STAMP(a, u, 15, trace_now());      // (the last warp of the CTA planned the reduction)
@@ -1331,7 +1388,7 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         const int used = gstate[0] * kGroupInts;
         for (int i = tid; i < kPlanGroupInts; i += kThreads) pg[i] = i < used ? gdesc[i] : i == kMaxGroups * kGroupInts ? gstate[0] : 0;
         if (blockIdx.x == 0) {
-            int *pc = reinterpret_cast<int *>(a.plan + 256);
+            int *pc = reinterpret_cast<int *>(a.plan + plan_cum_off(B));
             for (int i = tid; i < 2 * (B + 1); i += kThreads) pc[i] = cum[i];
             if (tid == 0)
                 *reinterpret_cast<PlanHeader *>(a.plan) =
