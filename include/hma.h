@@ -7,7 +7,9 @@
  *
  *   hma_kv_ingest_layer     scatter one layer of arriving wire bytes into the paged cache
  *                           (consumer half of the compute-transfer pipeline, section 3.2)
- *   hma_decode_attention    GQA paged decode attention reading raw BFP8 pages (section 3.3)
+ *   hma_decode_attention    GQA paged decode attention reading raw BFP8 pages (section 3.3);
+ *                           hma_decode_attention_plan once per decode step + hma_decode_attention_planned
+ *                           per layer is the same computation with its set-up done once
  *   hma_bfp8_dequant_bf16   one-shot BFP8 -> BF16 rebuild of a request's KV (the whole-request
  *                           reconstruction kernel of section 3.3)
  *
