@@ -315,6 +315,22 @@ class Workload:
             torch.cuda.synchronize(self.device)
             self.copy_probe_layer_s = c0.elapsed_time(c1) / 1e3 / reps / self.L
             del dst
+            # every layer of the request in one call (hma_kv_ingest_request_shards): the same bytes in one launch
+            hs = self.hkv // 4
+            w = self.wire_dev
+
+            def whole():
+                self.hma.hma_kv_ingest_request_shards(self.caches["bfp8"], [w[0, 0, i] for i in range(4)], [w[0, 1, i] for i in range(4)],
+                                                      2 * 4 * self.shard_bytes, self.hma.HMA_WIRE_TILE32, [i * hs for i in range(4)],
+                                                      [hs] * 4, self.spare, 0, self.ingest_tokens, s)
+            whole()
+            torch.cuda.synchronize(self.device)
+            c0.record()
+            for _ in range(reps):
+                whole()
+            c1.record()
+            torch.cuda.synchronize(self.device)
+            self.ingest_request_s = c0.elapsed_time(c1) / 1e3 / reps
         torch.cuda.current_stream(self.device).wait_stream(s)
         return e0.elapsed_time(e1) / 1e3 / reps / self.L
 
@@ -630,6 +646,9 @@ def main():
         extra["ingest_alone"] = {"us_per_layer": t_ing * 1e6, "gbs_read_plus_write": 2 * layer_bytes / t_ing / 1e9,
                                  "frac_of_peak": 2 * layer_bytes / t_ing / 1e9 / peak,
                                  "copy_probe_us_per_layer": wl.copy_probe_layer_s * 1e6, "frac_of_copy_probe": wl.copy_probe_layer_s / t_ing,
+                                 "whole_request_one_call": {"ms": wl.ingest_request_s * 1e3, "gbs_read_plus_write": 2 * layer_bytes * wl.L / wl.ingest_request_s / 1e9,
+                                                            "frac_of_peak": 2 * layer_bytes * wl.L / wl.ingest_request_s / 1e9 / peak,
+                                                            "what": "hma_kv_ingest_request_shards: every layer of the same request in one launch"},
                                  "copy_probe": "hma_hbm_copy_probe in the same harness: one plain launch per layer that reads the layer's wire bytes and writes as many",
                                  "what": "hma_kv_ingest_layer_shards, one 8192-token layer (4 shards, TILE32), device-resident wire, CUDA-graph replay"}
     t_mixed = wl.time_mixed()

@@ -153,6 +153,16 @@ hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t layer, int32
                                         const int32_t *head_begins, const int32_t *head_counts,
                                         const int32_t *page_ids, int64_t token_begin, int64_t n_tokens, void *stream);
 
+/* Every layer of the cache in one call, for a request whose bytes have all arrived (the counterpart of
+ * hma_bfp8_rebuild_request): layer l's wire of shard s starts l * layer_stride_bytes after k_wires[s] / v_wires[s]
+ * (a multiple of 16).  Same contents as num_layers calls of hma_kv_ingest_layer_shards; whole pages of a tiled wire into a
+ * BFP8 cache go through one launch of the streaming kernel (a 36-MB layer alone is too short a launch to reach the
+ * memory system's rate), everything else layer by layer. */
+hma_status_t hma_kv_ingest_request_shards(hma_cache_t *cache, int32_t n_shards, const void *const *k_wires,
+                                          const void *const *v_wires, size_t layer_stride_bytes, int32_t wire_layout,
+                                          const int32_t *head_begins, const int32_t *head_counts, const int32_t *page_ids,
+                                          int64_t token_begin, int64_t n_tokens, void *stream);
+
 /*
  * Decode attention over block tables (section 3.3; one query token per sequence, section 1).
  * For sequence b, q head h, kv head g = h / (num_q_heads/num_kv_heads), T = context_lens[b]:

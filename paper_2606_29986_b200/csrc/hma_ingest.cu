@@ -195,7 +195,9 @@ __device__ __forceinline__ bool ing_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-__global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView cv, IngestArgs a, int tile_rows, int full_pages)
+template <bool kMulti>      // kMulti: items run over several layers (the whole-request call)
+__global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView cv, IngestArgs a, int tile_rows, int full_pages,
+                                                                      void *const *__restrict__ layers, int n_layers, int64_t layer_stride)
 {
     extern __shared__ __align__(128) uint8_t ing_smem[];
     uint8_t *in = ing_smem;                                              // [stages][2 tensors][4352]
@@ -204,7 +206,8 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
     const int tid = threadIdx.x;
     int heads = 0;
     for (int s = 0; s < a.n_shards; ++s) heads += a.head_count[s];
-    const int n_items = heads * tile_rows;
+    const int per_layer = heads * tile_rows;
+    const int n_items = (kMulti ? n_layers : 1) * per_layer;      // item = (layer, head, tile row); !kMulti: cv.layer is the only layer
     if (tid == 0) {
         for (int s = 0; s < kIngestStages; ++s)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(ing_smem_u32(bars + s)));
@@ -215,8 +218,10 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
     // launched with programmatic stream serialisation: nothing a predecessor may have written is read before this
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // item -> (shard, head inside the shard, tile row)
+    // item -> (layer, shard, head inside the shard, tile row)
+    auto layer_of = [&](int item) { return kMulti ? item / per_layer : 0; };      // one layer: no division
     auto locate = [&](int item, int *shard, int *hs, int *tr) {
+        if (kMulti) item %= per_layer;
         int hi = item / tile_rows;
         *tr = item - hi * tile_rows;
         int sh = 0;
@@ -227,7 +232,7 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
     auto load = [&](int item, int stage) {      // thread 0 only
         int shard, hs, tr;
         locate(item, &shard, &hs, &tr);
-        const int64_t off = ((int64_t)hs * tile_rows + tr) * kTileRowBytes;
+        const int64_t off = ((int64_t)hs * tile_rows + tr) * kTileRowBytes + (int64_t)layer_of(item) * layer_stride;
         const uint32_t bar = ing_smem_u32(bars + stage), dst = ing_smem_u32(in + stage * 2 * kTileRowBytes);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * kTileRowBytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -251,7 +256,7 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
         // the physical pages of this item are asked for now, so that the table read is over when the records are ready to leave
         int32_t pid2[2] = {-1, -1};
         if (tid == 0) {
-            const int tr0 = item % tile_rows;
+            const int tr0 = (kMulti ? item % per_layer : item) % tile_rows;
             if (2 * tr0 < full_pages) pid2[0] = a.page_ids[2 * tr0];
             if (2 * tr0 + 1 < full_pages) pid2[1] = a.page_ids[2 * tr0 + 1];
         }
@@ -328,7 +333,8 @@ __global__ void __launch_bounds__(kIngestThreads) ingest_tiles_kernel(CacheView 
                 if (lpp >= full_pages) continue;
                 const int32_t pid = pid2[pp];
                 if (pid < 0 || pid >= cv.num_pages) { atomicOr(cv.flags, HMA_FLAG_BAD_PAGE_INGEST); continue; }
-                uint8_t *dst = cv.layer + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)kBfp8Record;
+                uint8_t *base = kMulti ? (uint8_t *)layers[layer_of(item)] : cv.layer;
+                uint8_t *dst = base + ((int64_t)pid * cv.num_kv_heads + h) * (int64_t)kBfp8Record;
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
                              "r"(ing_smem_u32(out + ((n % kIngestOut) * 2 + pp) * kBfp8Record)), "r"(kBfp8Record)
                              : "memory");
@@ -384,9 +390,11 @@ __global__ void __launch_bounds__(128) ingest_bf16_rows_kernel(CacheView cv, Ing
 static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_shards, const void *const *k_wires,
                                   const void *const *v_wires, int32_t wire_layout, const int32_t *head_begins,
                                   const int32_t *head_counts, const int32_t *page_ids, int64_t token_begin, int64_t n_tokens,
-                                  void *stream)
+                                  void *stream, int32_t n_layers = 1, size_t layer_stride = 0)
 {
-    if (!cache || layer < 0 || layer >= cache->desc.num_layers) return HMA_ERR_INVALID_ARG;
+    // layers [layer, layer + n_layers); layer l's wire of shard s starts l * layer_stride bytes after k_wires[s] / v_wires[s]
+    if (!cache || layer < 0 || n_layers < 1 || layer + n_layers > cache->desc.num_layers) return HMA_ERR_INVALID_ARG;
+    if (n_layers > 1 && (layer_stride & 15u)) return HMA_ERR_ALIGNMENT;
     if (!hma::on_cache_device(cache)) return HMA_ERR_INVALID_ARG;
     if (wire_layout != HMA_WIRE_TILE32 && wire_layout != HMA_WIRE_ROWMAJOR && wire_layout != HMA_WIRE_BF16_ROWS) return HMA_ERR_INVALID_ARG;
     if (wire_layout == HMA_WIRE_BF16_ROWS && cache->desc.format != HMA_KV_BF16) return HMA_ERR_INVALID_ARG;
@@ -426,8 +434,24 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
     a.wire_tokens = n_tokens;
     a.layout = wire_layout;
     cudaStream_t st = (cudaStream_t)stream;
-    if (wire_layout == HMA_WIRE_TILE32 && cache->desc.format == HMA_KV_BFP8 && (token_begin & 15) == 0 && n_tokens >= hma::kPageTokens &&
-        n_tokens / hma::kPageTokens <= 0x3FFFFFFF) {
+    const bool streaming = wire_layout == HMA_WIRE_TILE32 && cache->desc.format == HMA_KV_BFP8 && (token_begin & 15) == 0 &&
+                           n_tokens >= hma::kPageTokens && n_tokens / hma::kPageTokens <= 0x3FFFFFFF &&
+                           (int64_t)n_layers * heads * ((n_tokens + 31) / 32) <= 0x7FFFFFFF;
+    if (n_layers > 1 && !streaming) {
+        // no streaming path for this case: layer by layer
+        for (int l = 0; l < n_layers; ++l) {
+            const void *kw[hma::kMaxShards], *vw[hma::kMaxShards];
+            for (int s = 0; s < n_shards; ++s) {
+                kw[s] = (const uint8_t *)k_wires[s] + (size_t)l * layer_stride;
+                vw[s] = (const uint8_t *)v_wires[s] + (size_t)l * layer_stride;
+            }
+            const hma_status_t r = launch_ingest(cache, layer + l, n_shards, kw, vw, wire_layout, head_begins, head_counts, page_ids,
+                                                 token_begin, n_tokens, stream);
+            if (r != HMA_OK) return r;
+        }
+        return HMA_OK;
+    }
+    if (streaming) {
         // whole pages of a tiled wire: the streaming kernel; a ragged last page (if any) follows through the general kernel
         static std::mutex setup_lock;
         static int sm_count[64] = {};
@@ -440,7 +464,8 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
             if (!sm_count[dev]) {
                 int n = 0;
                 HMA_CUDA_OK(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
-                HMA_CUDA_OK(cudaFuncSetAttribute(hma::ingest_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                HMA_CUDA_OK(cudaFuncSetAttribute(hma::ingest_tiles_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                HMA_CUDA_OK(cudaFuncSetAttribute(hma::ingest_tiles_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
                 sm_count[dev] = n;
             }
         }
@@ -450,7 +475,7 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
         // items are numbered over all tile rows of the wire; a last tile row without a whole page holds no item to do,
         // but keeping the wire's own row count in the numbering keeps the addressing plain
         (void)items;
-        const int64_t n_items = (int64_t)heads * tile_rows;
+        const int64_t n_items = (int64_t)n_layers * heads * tile_rows;
         const int64_t max_ctas = (int64_t)sm_count[dev] * 4;
         const unsigned grid_x = (unsigned)(n_items < max_ctas ? n_items : max_ctas);
         cudaLaunchAttribute attr[1];
@@ -463,7 +488,11 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
         cfg.stream = st;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::ingest_tiles_kernel, cv, a, tile_rows, full_pages));
+        void *const *layers = n_layers > 1 ? (void *const *)(cache->d_layers + layer) : nullptr;
+        if (n_layers > 1)
+            HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::ingest_tiles_kernel<true>, cv, a, tile_rows, full_pages, layers, (int)n_layers, (int64_t)layer_stride));
+        else
+            HMA_CUDA_OK(cudaLaunchKernelEx(&cfg, hma::ingest_tiles_kernel<false>, cv, a, tile_rows, full_pages, layers, 1, (int64_t)0));
         hma::count_launch();
         const int64_t rest = n_tokens - (int64_t)full_pages * hma::kPageTokens;
         if (rest == 0) return HMA_OK;
@@ -471,8 +500,15 @@ static hma_status_t launch_ingest(hma_cache_t *cache, int32_t layer, int32_t n_s
         a.n_tokens = rest;
         a.page_ids = page_ids + full_pages;
         dim3 tail_grid(1u, (unsigned)heads);
-        hma::ingest_kernel<<<tail_grid, 128, 0, st>>>(cv, a);
-        hma::count_launch();
+        for (int l = 0; l < n_layers; ++l) {      // the ragged last page, layer by layer, through the general kernel
+            cv.layer = (uint8_t *)cache->layers[layer + l];
+            for (int s = 0; s < n_shards; ++s) {
+                a.k_wire[s] = (const uint8_t *)k_wires[s] + (size_t)l * layer_stride;
+                a.v_wire[s] = (const uint8_t *)v_wires[s] + (size_t)l * layer_stride;
+            }
+            hma::ingest_kernel<<<tail_grid, 128, 0, st>>>(cv, a);
+            hma::count_launch();
+        }
         HMA_CUDA_OK(cudaGetLastError());
         return HMA_OK;
     }
@@ -500,3 +536,14 @@ extern "C" hma_status_t hma_kv_ingest_layer_shards(hma_cache_t *cache, int32_t l
     return launch_ingest(cache, layer, n_shards, k_wires, v_wires, wire_layout, head_begins, head_counts, page_ids,
                          token_begin, n_tokens, stream);
 }
+
+extern "C" hma_status_t hma_kv_ingest_request_shards(hma_cache_t *cache, int32_t n_shards, const void *const *k_wires,
+                                                     const void *const *v_wires, size_t layer_stride_bytes, int32_t wire_layout,
+                                                     const int32_t *head_begins, const int32_t *head_counts, const int32_t *page_ids,
+                                                     int64_t token_begin, int64_t n_tokens, void *stream)
+{
+    if (!cache) return HMA_ERR_INVALID_ARG;
+    return launch_ingest(cache, 0, n_shards, k_wires, v_wires, wire_layout, head_begins, head_counts, page_ids, token_begin, n_tokens,
+                         stream, cache->desc.num_layers, layer_stride_bytes);
+}
+

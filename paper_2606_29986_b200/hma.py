@@ -63,6 +63,9 @@ def lib():
         L.hma_kv_ingest_layer_shards.restype = i32
         L.hma_kv_ingest_layer_shards.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), i32,
                                                  ctypes.POINTER(i32), ctypes.POINTER(i32), vp, i64, i64, vp]
+        L.hma_kv_ingest_request_shards.restype = i32
+        L.hma_kv_ingest_request_shards.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), sz, i32,
+                                                   ctypes.POINTER(i32), ctypes.POINTER(i32), vp, i64, i64, vp]
         L.hma_decode_attention_workspace_bytes.restype = sz
         L.hma_decode_attention_workspace_bytes.argtypes = [ctypes.POINTER(CacheDesc), i32]
         L.hma_decode_attention_workspace_init.restype = i32
@@ -193,6 +196,19 @@ def hma_kv_ingest_layer_shards(cache, layer, k_wires, v_wires, wire_layout, head
     hc = (ctypes.c_int32 * n)(*head_counts)
     _check(lib().hma_kv_ingest_layer_shards(cache.handle, layer, n, kp, vp_, wire_layout, hb, hc, _ptr(page_ids),
                                             token_begin, n_tokens, _stream(stream)), "hma_kv_ingest_layer_shards")
+
+
+def hma_kv_ingest_request_shards(cache, k_wires, v_wires, layer_stride_bytes, wire_layout, head_begins, head_counts, page_ids,
+                                 token_begin, n_tokens, stream=None):
+    """Every layer of the cache in one call: k_wires / v_wires are lists (one per shard) of layer 0's wire tensors; layer l's
+    wire starts l * layer_stride_bytes further on in the same allocation."""
+    n = len(k_wires)
+    kp = (ctypes.c_void_p * n)(*[t.data_ptr() for t in k_wires])
+    vp_ = (ctypes.c_void_p * n)(*[t.data_ptr() for t in v_wires])
+    hb = (ctypes.c_int32 * n)(*head_begins)
+    hc = (ctypes.c_int32 * n)(*head_counts)
+    _check(lib().hma_kv_ingest_request_shards(cache.handle, n, kp, vp_, layer_stride_bytes, wire_layout, hb, hc, _ptr(page_ids),
+                                              token_begin, n_tokens, _stream(stream)), "hma_kv_ingest_request_shards")
 
 
 def hma_decode_attention_workspace_bytes(desc, batch):

@@ -190,6 +190,39 @@ def test_bfp8_cache_holds_the_wire_bytes_unchanged():
             assert np.array_equal(np.sort(rec[p, h]), np.sort(wire))
 
 
+@pytest.mark.parametrize("layout,T", [(hma.HMA_WIRE_TILE32, 112), (hma.HMA_WIRE_TILE32, 75), (hma.HMA_WIRE_ROWMAJOR, 50)])
+def test_whole_request_ingest_equals_layer_by_layer(layout, T):
+    """hma_kv_ingest_request_shards (every layer in one call) leaves the cache that layer-by-layer ingest leaves."""
+    L, H, shards = 3, 4, 2
+    sc = Scenario([T], 8, H, seed=31, layers=L, wire_layout=layout, shards=shards, one_launch=True, permute=True)
+    want = [t.clone() for t in sc.cache.layers]
+    for t in sc.cache.layers:
+        t.fill_(0xA5)
+    hs = H // shards
+    pages = sc.table[0, :(T + 15) // 16].contiguous()
+    # [layer][tensor][shard] wire pieces in one allocation, a fixed stride between layers
+    pieces = []
+    for l in range(L):
+        for w in (sc.k_wires[l][0], sc.v_wires[l][0]):
+            for s in range(shards):
+                x = torch.from_numpy(w[s * hs:(s + 1) * hs].copy())
+                pieces.append(synth.rowmajor_to_tile32(x).reshape(-1) if layout == hma.HMA_WIRE_TILE32 else x.reshape(-1))
+    n = pieces[0].numel()
+    pad = (n + 15) // 16 * 16
+    buf = torch.zeros((L, 2, shards, pad), dtype=torch.uint8, device="cuda")
+    it = iter(pieces)
+    for l in range(L):
+        for t in range(2):
+            for s in range(shards):
+                buf[l, t, s, :n] = next(it).cuda()
+    hma.hma_kv_ingest_request_shards(sc.cache, [buf[0, 0, s] for s in range(shards)], [buf[0, 1, s] for s in range(shards)],
+                                     2 * shards * pad, layout, [s * hs for s in range(shards)], [hs] * shards, pages, 0, T)
+    torch.cuda.synchronize()
+    assert hma.hma_error_flags(sc.cache) == 0
+    for l in range(L):
+        assert torch.equal(sc.cache.layers[l], want[l]), l
+
+
 def test_rowmajor_wire_needs_only_the_encoders_alignment():
     """hma_bfp8_encode_rows promises 8-byte aligned rows; a wire that starts 8 bytes off a 16-byte boundary is ingested as it is."""
     sc = Scenario([48], 8, 2, seed=21, layers=1)
