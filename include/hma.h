@@ -264,7 +264,10 @@ hma_status_t hma_decode_attention_simple(const hma_cache_t *cache, int32_t layer
  *                made for another launch shape is detected and the call computes nothing; page counts that no longer
  *                match are detected while the call runs and its results are void; both raise HMA_FLAG_BAD_PLAN.  Changed
  *                table entries under unchanged page counts are not detectable.
- *   results      identical, bit for bit, to hma_decode_attention_multi with the same arguments.
+ *   results      identical, bit for bit, to hma_decode_attention_multi with the same arguments, except when no sequence
+ *                is longer than 8 pages: such a plan gives every (sequence, kv head) to one warp (nothing to combine at
+ *                the end of the kernel), the softmax weights (FP16) are rounded against other
+ *                running maxima and the sums are formed in another order: the results agree within the kernel's own error.
  * The plan call is ordinary stream work: later planned calls on the same stream see it without further synchronisation.
  */
 size_t hma_decode_attention_plan_bytes(int32_t rows);
@@ -296,8 +299,9 @@ hma_status_t hma_decode_attention_mixed(const hma_cache_t *prefix, const hma_cac
                                         int32_t batch, float sm_scale, void *workspace, size_t workspace_bytes,
                                         void *stream);
 /* The same with both launches' set-up taken from plans: prefix_plan from hma_decode_attention_plan(prefix, prefix_table,
- * prefix_max_pages, prefix_lens, batch, 1, ..), tail_plan likewise for the tail cache (two plan buffers).  Same results bit
- * for bit; the rules for a plan's lifetime are those of hma_decode_attention_planned. */
+ * prefix_max_pages, prefix_lens, batch, 1, ..), tail_plan likewise for the tail cache (two plan buffers).  Same results (to
+ * the bit, or within the kernel's own error where a plan of short segments cuts the work differently); the rules for a plan's lifetime
+ * are those of hma_decode_attention_planned. */
 hma_status_t hma_decode_attention_mixed_planned(const hma_cache_t *prefix, const hma_cache_t *tail, int32_t layer,
                                                 const void *q, void *out, int32_t out_dtype,
                                                 const int32_t *prefix_table, int32_t prefix_max_pages, const int32_t *prefix_lens,

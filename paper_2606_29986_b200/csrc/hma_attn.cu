@@ -54,6 +54,7 @@ constexpr int kMaxBatch = 1024;
 constexpr int kSegCost = 2;                        // what starting a segment costs a warp, in records (Q load, partial tile)
 constexpr int kMaxCtas = 192;                       // CTAs launched = min(SM count, kMaxCtas); sizes the workspace
 constexpr int kMinRecords = 4;                    // fewest records a worker takes
+constexpr int kAlignedMaxPages = 8;               // a plan gives every segment to one warp when none is longer than this
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGroups = 32;       // more than a CTA can have: a group holds a boundary between two of its (at most 16) warps, or one of its own ends
 constexpr int kGroupInts = 6;        // sequence, kv head, member mask, flags (1 whole segment, 2 has tail, tail warp << 8), parts, first CTA
@@ -749,7 +750,22 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
     // Small batches use fewer workers, at least kMinRecords units each, so that a segment is never cut into more
     // partials than it is worth.  Workers are dealt to the CTAs in contiguous runs (CTA c holds workers
     // [c * NWK / C, (c + 1) * NWK / C) of the C CTAs in use), so a CTA owns one contiguous range of records.
-    const Split sp = make_split(WX, (int)gridDim.x, kWarps);
+    Split sp = make_split(WX, (int)gridDim.x, kWarps);
+    // A plan for short segments (the decode-side tail of two-cache attention: a few pages per sequence) gives every
+    // (sequence, kv head) segment to one warp, worker u = sequence * Hkv + head: no segment is shared, so the kernel that
+    // follows the plan has no CTA-level reduction and no cross-CTA merge to do at its end.  (Its loop over empty sequences
+    // steps by the cost-based worker count; with this numbering worker u = b covers sequence b, and a second visit writes
+    // the same bytes.)
+    bool aligned = false;
+    if constexpr (kPlanOnly) {
+        int maxnp = 0;
+        for (int bb = 0; bb < B; ++bb) maxnp = max(maxnp, cum[bb + 1] - cum[bb]);
+        aligned = maxnp > 0 && maxnp <= kAlignedMaxPages && (int64_t)B * Hkv <= (int64_t)gridDim.x * kWarps;
+        if (aligned) {
+            sp.nwk = (int64_t)B * Hkv;
+            sp.ctas = sp.nwk < (int64_t)gridDim.x ? sp.nwk : (int64_t)gridDim.x;
+        }
+    }
     const int64_t NWK = sp.nwk;
     int64_t u;                                                      // this warp's worker index (if it is a worker)
     bool worker;
@@ -826,8 +842,14 @@ __global__ void __launch_bounds__(Geo<kFmt, kQ>::threads, 1) attn_kernel(const A
         wlo = pw.wlo;
         whi = pw.whi;
     } else {
-        wlo = records_before(u * WX / NWK);
-        whi = records_before((u + 1) * WX / NWK);
+        if (kPlanOnly && aligned) {
+            const int bb = (int)(u / Hkv), gg = (int)(u - (int64_t)bb * Hkv), npb = cum[bb + 1] - cum[bb];
+            wlo = (int64_t)Hkv * cum[bb] + (int64_t)gg * npb;
+            whi = wlo + npb;
+        } else {
+            wlo = records_before(u * WX / NWK);
+            whi = records_before((u + 1) * WX / NWK);
+        }
     }
     if (wlo >= whi) { publish(); break; }
     const int Rw = (int)(whi - wlo);
